@@ -1,0 +1,418 @@
+"""Pins of the CPU checker against things other than itself.
+
+* the paper's worked example (Section 3.2 listing) against a hand-written standard-library
+  regular expression of the pattern the paper says it represents;
+* the non-greedy rule (Section 6);
+* masks against an independent partial matcher (``regex_ref``) and against brute-force
+  prefix viability on tiny vocabularies;
+* closed forms: single-byte tokens, pure literals, one free-text slot;
+* the invariants the method promises: the EOS rule, non-empty masks on a valid trajectory,
+  the decoded trajectory being a member of the language;
+* apply / argmax against their plain definitions in numpy.
+"""
+import itertools
+import re
+
+import numpy as np
+import pytest
+
+import oracle
+import regex_ref
+from wg_workloads import (ALL_BYTES, DIGITS, EOS, Cond, DoWhile, IfElse, Sequence, Switch, SymSet,
+                          Wait, Write, bf16_bits_to_f32, enum_trie, flatten, grammars,
+                          make_logits, make_vocab, vocab_from_tokens)
+
+
+def tree_of(op):
+    return oracle.Tree(flatten(op))
+
+
+def bit(words, t):
+    return (int(words[t >> 5]) >> (t & 31)) & 1
+
+
+def unpack(words, V):
+    return np.unpackbits(words.view(np.uint8), bitorder="little")[:V].astype(bool)
+
+
+# ---------------------------------------------------------------------------------------
+# Section 3.2 listing: said to represent \d+(\.\d+)* followed by <eos>
+# ---------------------------------------------------------------------------------------
+def test_paper_listing_language_exhaustive():
+    tree = tree_of(grammars.paper_listing_example())
+    hand = re.compile(rb"[0-9]+(\.[0-9]+)*\x02+")
+    alphabet = [ord("0"), ord("7"), ord("."), ord("x"), EOS]
+    n_accept = 0
+
+    def dfs(cursor, symbols):
+        nonlocal n_accept
+        data = regex_ref.to_bytes(symbols)
+        accepted = cursor == oracle.DONE
+        assert accepted == (hand.fullmatch(data) is not None), data
+        n_accept += accepted
+        if len(symbols) == 7:
+            return
+        for s in alphabet:
+            nxt = tree.step(cursor, s)
+            if oracle.is_dead(nxt):
+                # everything below a refused symbol must be a non-member as well
+                assert hand.fullmatch(regex_ref.to_bytes(symbols + [s])) is None
+                if len(symbols) < 5:
+                    for tail in itertools.product(alphabet, repeat=2):
+                        assert hand.fullmatch(regex_ref.to_bytes(symbols + [s] + list(tail))) is None
+                continue
+            dfs(nxt, symbols + [s])
+
+    dfs(tree.start(), [])
+    assert n_accept > 100
+
+
+def test_paper_listing_keeps_digit_runs_and_needs_a_digit_after_the_dot():
+    tree = tree_of(grammars.paper_listing_example())
+    ok = lambda s: tree.accepts([ord(c) for c in s] + [EOS])  # noqa: E731
+    assert ok("7") and ok("2025") and ok("3.14") and ok("10.0.0.255")
+    assert not ok("") and not ok(".5") and not ok("5.") and not ok("1..2") and not ok("1.x")
+    # without the end-of-sequence symbol the program has not completed
+    assert not tree.accepts([ord("7")])
+
+
+def test_non_greedy_wait_ends_at_first_wait_symbol():
+    tree = tree_of(Sequence(Wait(allow=SymSet(b"ab"), wait=SymSet(b"b")), Write(b"c")))
+    assert tree.accepts(list(b"aabc") + [EOS])
+    assert tree.accepts(list(b"bc") + [EOS])
+    assert not tree.accepts(list(b"abbc") + [EOS])
+    assert not tree.accepts(list(b"aac") + [EOS])
+
+
+def test_wait_symbol_outside_allow_is_still_accepted_and_deny_wins_over_allow():
+    tree = tree_of(Wait(allow=SymSet(b"abc"), deny=SymSet(b"c"), wait=SymSet(b";")))
+    assert tree.accepts(list(b"abab;") + [EOS])
+    assert not tree.accepts(list(b"abc;") + [EOS])
+
+
+def test_wait_body_runs_after_the_wait_symbol():
+    tree = tree_of(Sequence(Wait(allow=SymSet(b"x"), wait=SymSet(b"("), body=Write(b"in")),
+                            Write(b")")))
+    assert tree.accepts(list(b"xx(in)") + [EOS])
+    assert not tree.accepts(list(b"xx()") + [EOS])
+
+
+def test_switch_three_way_and_absent_bodies():
+    sw = Switch(allow=SymSet(b" abc"), cases=[SymSet(b"a"), SymSet(b"b"), SymSet(b"c")],
+                bodies=[Write(b"1"), None, Sequence(Write(b"3"), Write(b"3"))])
+    tree = tree_of(Sequence(sw, Write(b".")))
+    for s, want in [(b"a1.", True), (b"  b.", True), (b"c33.", True), (b"a.", False),
+                    (b"b1.", False), (b"c3.", False), (b"d.", False)]:
+        assert tree.accepts(list(s) + [EOS]) is want, s
+
+
+def test_dowhile_repeats_on_true_and_leaves_on_false():
+    loop = DoWhile(body=Write(b"ab"), condition=Cond(allow=SymSet(b" ,;"), true_waits=SymSet(b","),
+                                                     false_waits=SymSet(b";")))
+    tree = tree_of(Sequence(Write(b"["), loop, Write(b"]")))
+    for s, want in [(b"[ab;]", True), (b"[ab,ab;]", True), (b"[ab ,ab  ;]", True),
+                    (b"[;]", False), (b"[ab,;]", False), (b"[ab,ab]", False), (b"[abab;]", False)]:
+        assert tree.accepts(list(s) + [EOS]) is want, s
+
+
+def test_done_accepts_only_eos_and_stays_done():
+    tree = tree_of(Write(b"hi"))
+    c = tree.walk(tree.start(), list(b"hi"))
+    assert c == (-3, 0)                        # the implicit trailing EOS wait
+    assert oracle.is_dead(tree.step(c, ord("x")))
+    c = tree.step(c, EOS)
+    assert c == oracle.DONE
+    assert tree.step(c, EOS) == oracle.DONE
+    assert oracle.is_dead(tree.step(c, ord("h")))
+
+
+def test_explicit_eos_suppresses_the_implicit_one():
+    tree = tree_of(Sequence(Write(b"a"), Wait(allow=SymSet([EOS]), wait=SymSet([EOS]))))
+    assert tree.walk(tree.start(), [ord("a"), EOS]) == oracle.DONE
+
+
+@pytest.mark.parametrize("bad", [
+    Wait(allow=SymSet(b"a"), wait=SymSet()),                                   # empty wait set
+    Wait(allow=SymSet(b"ab"), wait=SymSet(b"b"), deny=SymSet(b"b")),           # wait meets deny
+    IfElse(Cond(allow=SymSet(b"ab"), true_waits=SymSet(b"ab"), false_waits=SymSet(b"b")),
+           None, None),                                                         # overlapping cases
+    DoWhile(Write(b"x"), Cond(allow=SymSet(b"a"), true_waits=SymSet(b"a"), false_waits=SymSet())),
+])
+def test_rejected_trees(bad):
+    with pytest.raises(oracle.OracleError) as e:
+        tree_of(bad)
+    assert e.value.code == oracle.ERR_GRAMMAR
+
+
+def test_shared_subtree_is_rejected():
+    flat = flatten(Sequence(Write(b"a"), Write(b"b")))
+    flat.children[1] = flat.children[0]        # both parts point at the same node
+    with pytest.raises(oracle.OracleError):
+        oracle.Tree(flat)
+
+
+# ---------------------------------------------------------------------------------------
+# masks against the independent partial matcher
+# ---------------------------------------------------------------------------------------
+SMALL_GRAMMARS = {
+    "listing": grammars.paper_listing_example,
+    "html": grammars.html_template,
+    "json": grammars.json_reference_lookup,
+    "template0": lambda: grammars.random_template(0, 4, 6),
+    "template5": lambda: grammars.random_template(5, 4, 6),
+    "snippets": lambda: grammars.dynamic_snippet_template(3, n_args=2, enum_size=7),
+}
+
+
+def greedy_random_walk(tree, vocab, rng, steps, prefer=None):
+    """Yield (cursor, emitted symbols so far) along a random valid trajectory."""
+    cursor, emitted = tree.start(), []
+    for _ in range(steps):
+        yield cursor, list(emitted)
+        allowed = np.flatnonzero(unpack(oracle.mask(tree, vocab, cursor), vocab.size))
+        assert allowed.size > 0
+        pool = allowed
+        if prefer is not None and rng.random() < 0.7:
+            good = allowed[prefer[allowed]]
+            if good.size:
+                pool = good
+        t = int(rng.choice(pool))
+        rc, cursor = oracle.advance(tree, vocab, cursor, t)
+        assert rc == 0
+        emitted += [EOS] if t == vocab.eos_id else list(vocab.token(t))
+
+
+@pytest.mark.parametrize("name", sorted(SMALL_GRAMMARS))
+def test_masks_equal_partial_regex_matching(name):
+    from wg_workloads import has_structural_byte
+    op = SMALL_GRAMMARS[name]()
+    tree = tree_of(op)
+    prog = regex_ref.program(op)
+    vocab = make_vocab(1500, seed=11)
+    toks = vocab.tokens()
+    rng = np.random.default_rng(7)
+    prefer = has_structural_byte(vocab)
+    n_points = 0
+    for cursor, emitted in greedy_random_walk(tree, vocab, rng, 40, prefer):
+        prefix = regex_ref.to_bytes(emitted)
+        got = unpack(oracle.mask(tree, vocab, cursor), vocab.size)
+        for t in range(vocab.size):
+            if t == vocab.eos_id:
+                want = regex_ref.viable(prog, prefix + bytes([regex_ref.EOS_BYTE]))
+            elif len(toks[t]) == 0:
+                want = False
+            else:
+                want = regex_ref.viable(prog, prefix + toks[t])
+            assert bool(got[t]) == want, (name, t, toks[t], prefix[-20:])
+        n_points += 1
+    assert n_points == 40
+
+
+def test_mask_is_prefix_viability_by_brute_force_on_a_tiny_vocabulary():
+    # [TEXT</] with TEXT free of '<'; membership decided by a hand-written stdlib pattern
+    op = Sequence(Write(b"["), Wait(allow=ALL_BYTES, wait=SymSet(b"<")), Write(b"/]"))
+    hand = re.compile(rb"\[[^<\x02]*</\]\x02+", re.S)
+    tree = tree_of(op)
+    alphabet = [b"<", b"[", b"]", b"/", b"x", b"\x02"]
+    tokens = [b"<", b"[", b"", b"]", b"/", b"x", b"[<", b"/]", b"[x", b"x<", b"</", b"</]",
+              b"xx", b"<<", b"[</]", b"]x</", b"</]x", b"[[", b"x]/", b"[x</]", b"/]x", b"<]"]
+    vocab = vocab_from_tokens(tokens, eos_id=2)
+
+    def viable(data):
+        for n in range(0, 7):
+            for z in itertools.product(alphabet, repeat=n):
+                if hand.fullmatch(data + b"".join(z)):
+                    return True
+        return False
+
+    prefixes = [b"", b"[", b"[x", b"[x]x/", b"[<", b"[xx<", b"[x</", b"[x</]"]
+    for p in prefixes:
+        cursor = tree.walk(tree.start(), list(p))
+        assert not oracle.is_dead(cursor)
+        got = unpack(oracle.mask(tree, vocab, cursor), vocab.size)
+        for t, tok in enumerate(tokens):
+            data = p + (b"\x02" if t == 2 else tok)
+            want = False if (t != 2 and not tok) else viable(data)
+            assert bool(got[t]) == want, (p, tok)
+
+
+# ---------------------------------------------------------------------------------------
+# closed forms on the config-1 vocabulary
+# ---------------------------------------------------------------------------------------
+@pytest.fixture(scope="module")
+def vocab32k():
+    return make_vocab(32000, seed=1)
+
+
+def test_bit_order_and_zero_tail():
+    tokens = [bytes([65 + (i % 26)]) * (1 + i // 26) for i in range(70)]
+    tokens[2] = b""
+    vocab = vocab_from_tokens(tokens, eos_id=2)
+    tree = tree_of(Write(b"HH"))              # allowed: "H" (id 7) and "HH" (id 33)
+    words = oracle.mask(tree, vocab, tree.start())
+    assert words.shape == (3,)
+    assert words.tolist() == [1 << 7, 1 << (33 - 32), 0]
+    every = tree_of(Wait(allow=ALL_BYTES, wait=SymSet(b"!")))
+    words = oracle.mask(every, vocab, every.start())
+    assert words.tolist() == [0xFFFFFFFF & ~(1 << 2), 0xFFFFFFFF, (1 << 6) - 1]  # ids 64..69 only
+
+
+def test_single_byte_tokens_follow_the_active_primitive(vocab32k):
+    op = grammars.json_reference_lookup()
+    tree = tree_of(op)
+    prog = regex_ref.program(op)
+    prefix = b'[{"topic": 1'
+    cursor = tree.walk(tree.start(), list(prefix))
+    words = oracle.mask(tree, vocab32k, cursor)
+    for t in range(256):
+        want = t != 2 and (chr(t) in "0123456789,")
+        assert bit(words, t) == int(want), t
+    assert regex_ref.viable(prog, prefix + b",")
+
+
+def test_pure_literal_allows_exactly_the_prefixes_of_the_rest(vocab32k):
+    lit = b'he said: "<p>ok</p>", twice'
+    tree = tree_of(Write(lit))
+    toks = vocab32k.tokens()
+    for done in (0, 3, 10, len(lit) - 2):
+        cursor = tree.walk(tree.start(), list(lit[:done]))
+        got = unpack(oracle.mask(tree, vocab32k, cursor), vocab32k.size)
+        rest = lit[done:]
+        want = np.array([len(t) > 0 and rest.startswith(t) for t in toks])
+        assert (got == want).all()
+        assert got.sum() >= 1
+
+
+def test_free_text_slot_closed_form(vocab32k):
+    closing = b"/h1>"
+    op = Sequence(Write(b"<h1>"), Wait(allow=ALL_BYTES, wait=SymSet(b"<")), Write(closing),
+                  Write(b"<p>"))
+    tree = tree_of(op)
+    cursor = tree.walk(tree.start(), list(b"<h1>some text"))
+    got = unpack(oracle.mask(tree, vocab32k, cursor), vocab32k.size)
+    after = closing + b"<p>"
+    for t, tok in enumerate(vocab32k.tokens()):
+        if t == 2 or not tok:
+            want = False
+        elif b"<" not in tok:
+            want = True
+        else:
+            want = after.startswith(tok[tok.index(b"<") + 1:])
+        assert bool(got[t]) == want, tok
+    assert 0.5 < got.mean() < 1.0
+
+
+# ---------------------------------------------------------------------------------------
+# invariants along decoded trajectories
+# ---------------------------------------------------------------------------------------
+@pytest.mark.parametrize("name", ["html", "json", "template0", "snippets"])
+def test_trajectory_invariants(name):
+    from wg_workloads import has_structural_byte
+    op = SMALL_GRAMMARS[name]()
+    tree = tree_of(op)
+    prog = regex_ref.program(op)
+    vocab = make_vocab(4000, seed=3)
+    bonus = has_structural_byte(vocab)
+    cursor, emitted, finished = tree.start(), [], False
+    for step in range(400):
+        words = oracle.mask(tree, vocab, cursor)
+        assert words.any(), "empty mask on a valid trajectory"
+        # EOS rule: the EOS bit is set iff the EOS symbol is accepted here
+        assert bit(words, vocab.eos_id) == int(not oracle.is_dead(tree.step(cursor, EOS)))
+        logits = make_logits(1, vocab.size, "fp32", [99, 0], step, bonus, steer=6.0)
+        t = int(oracle.argmax(logits, words[None, :], vocab.size)[0])
+        assert bit(words, t) == 1
+        rc, cursor = oracle.advance(tree, vocab, cursor, t)
+        assert rc == 0
+        emitted += [EOS] if t == vocab.eos_id else list(vocab.token(t))
+        assert regex_ref.viable(prog, regex_ref.to_bytes(emitted))
+        if cursor == oracle.DONE:
+            finished = True
+            break
+    if finished:
+        assert regex_ref.member(prog, regex_ref.to_bytes(emitted))
+        # a finished request can only emit EOS
+        words = oracle.mask(tree, vocab, cursor)
+        assert unpack(words, vocab.size).sum() == 1 and bit(words, vocab.eos_id) == 1
+    if name in ("json", "html"):
+        assert finished, "steered greedy decoding should finish these templates"
+
+
+def test_advance_rejects_and_keeps_the_cursor(vocab32k):
+    tree = tree_of(Write(b"abc"))
+    start = tree.start()
+    rc, c = oracle.advance(tree, vocab32k, start, ord("b"))
+    assert rc == oracle.ERR_REJECTED and c == start
+    rc, c = oracle.advance(tree, vocab32k, start, vocab32k.size)
+    assert rc == oracle.ERR_REJECTED and c == start
+    rc, c = oracle.advance(tree, vocab32k, start, ord("a"))
+    assert rc == 0 and c == (0, 1)
+
+
+# ---------------------------------------------------------------------------------------
+# apply and argmax against their definitions
+# ---------------------------------------------------------------------------------------
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+def test_apply_matches_numpy_definition(dtype):
+    V, B = 1003, 5
+    rng = np.random.default_rng(5)
+    logits = make_logits(B, V, dtype, 1)
+    words = rng.integers(0, 1 << 32, size=(B, (V + 31) // 32), dtype=np.uint64).astype(np.uint32)
+    words[0] = 0xFFFFFFFF
+    words[1] = 0
+    keep = np.stack([unpack(words[r], V) for r in range(B)])
+    before = logits.copy()
+    oracle.apply_mask(logits, words, V)
+    raw = logits.view(np.uint32) if dtype == "fp32" else logits
+    raw_before = before.view(np.uint32) if dtype == "fp32" else before
+    ninf = 0xFF800000 if dtype == "fp32" else 0xFF80
+    assert (raw[keep] == raw_before[keep]).all()
+    assert (raw[~keep] == ninf).all()
+    assert (raw[0] == raw_before[0]).all() and (raw[1] == ninf).all()
+    as_float = logits if dtype == "fp32" else bf16_bits_to_f32(logits)
+    assert np.isneginf(as_float[~keep]).all()
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+def test_argmax_is_first_maximum_over_allowed(dtype):
+    V, B = 5000, 6
+    rng = np.random.default_rng(9)
+    logits = make_logits(B, V, dtype, 2)
+    words = rng.integers(0, 1 << 32, size=(B, (V + 31) // 32), dtype=np.uint64).astype(np.uint32)
+    words[5] = 0
+    got = oracle.argmax(logits, words, V)
+    vals = logits if dtype == "fp32" else bf16_bits_to_f32(logits)
+    for r in range(B - 1):
+        keep = unpack(words[r], V)
+        masked = np.where(keep, vals[r], -np.inf)
+        assert got[r] == int(np.argmax(masked))     # numpy returns the first maximum
+    assert got[5] == -1
+
+
+def test_argmax_ties_signed_zero_and_all_minus_inf():
+    V = 64
+    words = np.array([[0xFFFFFFF0, 0xFFFFFFFF]], np.uint32)     # ids 0..3 are masked out
+    x = np.full((1, V), -1.0, np.float32)
+    x[0, 2] = 9.0                     # masked: must not win
+    x[0, 10] = -0.0
+    x[0, 20] = 0.0                    # equal to -0.0: the lower id stays
+    assert oracle.argmax(x, words, V)[0] == 10
+    x[0, 30] = 0.5
+    x[0, 40] = 0.5
+    assert oracle.argmax(x, words, V)[0] == 30
+    x[:] = -np.inf
+    assert oracle.argmax(x, words, V)[0] == 4
+    bf = np.full((1, V), 0xBF80, np.uint16)                    # -1.0
+    bf[0, 50] = 0x3F80                                          # +1.0
+    bf[0, 60] = 0x3F80
+    assert oracle.argmax(bf, words, V)[0] == 50
+
+
+def test_enum_trie_accepts_exactly_its_strings():
+    names = [b'alpha"', b'alps"', b'beta"', b'be"', b'gamma-1"', b'gamma-2"', b'g"']
+    op = Sequence(Write(b'"'), enum_trie(names), Write(b";"))
+    tree = tree_of(op)
+    for n in names:
+        assert tree.accepts(list(b'"' + n + b";") + [EOS])
+    for bad in [b'alp"', b'alphas"', b'bet"', b'gamma-3"', b'"']:
+        assert not tree.accepts(list(b'"' + bad + b";") + [EOS])
