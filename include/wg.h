@@ -1,0 +1,270 @@
+/*
+ * wg.h -- C ABI of the allowed-token mask path for operator-automaton structured decoding.
+ *
+ * What the path computes (paper Section 1: the mask is a vocabulary-sized binary tensor,
+ * ones = allowed, applied to the logits before sampling; Section 3.2: Wait / Write / IfElse /
+ * DoWhile / Sequence operators tracked by a finite state machine, one transition per
+ * generated token; Section 3.3: masks depend on the operator state only, so they are cached
+ * globally across steps and requests):
+ *
+ *   for every request r of a batch, with grammar id gid[r] and automaton state sid[r]:
+ *     bitmask[r, t>>5] bit (t&31) = 1  iff  the bytes of token t, walked from sid[r] through
+ *                                       the grammar's byte-level transition table, never
+ *                                       reach the DEAD state           (wg_build_masks)
+ *     masks of states seen before are served from a device cache       (wg_mask_cache_lookup)
+ *     logits[r, t] = -inf where the bit is clear, in place             (wg_apply_mask)
+ *     optionally token[r] = lowest id among the maxima of the allowed logits
+ *     sid[r] = state after the chosen token's bytes                    (wg_advance)
+ *
+ * Conventions
+ *   - Every call returns WG_OK (0) or a negative wg_status.  Nothing aborts or throws.
+ *   - "host" pointers are read during the call and may be freed afterwards.  "device"
+ *     pointers are owned by the caller, must belong to the CUDA device that was current when
+ *     the wg_ctx was created, and must stay valid until the work queued on `stream` is done.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Device
+ *     calls only enqueue work; they do not synchronise unless stated.
+ *   - Per-row problems found on the device (a refused token, an empty mask, an unknown
+ *     state) are written to the optional per-row status array and counted in wg_stats; they
+ *     never fault the GPU.
+ *   - Alphabet: symbols 0..255 are byte values, symbol 256 is end-of-sequence (EOS).  The EOS
+ *     token (id `eos_id`) stands for the one-symbol string [EOS]; any other token is its byte
+ *     string.  A zero-length token other than EOS is never allowed.
+ *   - State 0 of every compiled grammar is DEAD.  State ids are dense, 0 .. n_states-1.
+ *   - Packed masks: uint32 words, bit (t & 31) of word (t >> 5) belongs to token t, 1 =
+ *     allowed, bits at and beyond V are 0.  W = ceil(V / 32) words per row.
+ */
+#ifndef WG_H_
+#define WG_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum wg_status {
+    WG_OK = 0,
+    WG_ERR_ARG = -1,            /* null pointer, bad size, bad stride, unknown id            */
+    WG_ERR_GRAMMAR = -2,        /* the operator tree breaks a rule listed at wg_compile_grammar */
+    WG_ERR_CAPACITY = -3,       /* a fixed-size table of the library is full                 */
+    WG_ERR_TOKEN_REJECTED = -4, /* per row: the token is not allowed in the row's state      */
+    WG_ERR_CUDA = -5,           /* a CUDA runtime call failed; see wg_last_cuda_error        */
+    WG_ERR_EMPTY_MASK = -6,     /* per row: no token is allowed, so there is no argmax       */
+    WG_ERR_STATE = -7           /* per row: grammar id or state id out of range              */
+} wg_status;
+
+/* Logit element types of wg_apply_mask / wg_decode_step. */
+enum { WG_DTYPE_BF16 = 0, WG_DTYPE_FP32 = 1 };
+
+/* Flags of wg_build_masks and wg_decode_step. */
+enum {
+    WG_USE_CACHE = 0u, /* look up (gid, sid); build and insert the misses; copy rows out   */
+    WG_NO_CACHE = 1u   /* build every row, duplicates included; the cache is not touched   */
+};
+
+/* Flags of wg_advance and wg_decode_step. */
+enum {
+    WG_RESTART_ON_DONE = 2u /* a row that reaches the DONE state starts over at the grammar's
+                               start state (a finished request is replaced by a new one)   */
+};
+
+/* Operator kinds of wg_op_node (paper Section 3.2). */
+enum {
+    WG_OP_SEQUENCE = 0,
+    WG_OP_WRITE = 1,
+    WG_OP_WAIT = 2,
+    WG_OP_SWITCH = 3, /* IfElse and its k-way generalisation */
+    WG_OP_DOWHILE = 4
+};
+
+/* One node of a flattened operator tree.  Children, symbol sets and literal bytes live in
+ * three side arrays; a node names its slice of each.  A symbol set is 9 uint32 words, bit
+ * (s & 31) of word (s >> 5) for symbol s, symbol 256 = EOS.
+ *   SEQUENCE  children = the parts, in order
+ *   WRITE     data     = the literal bytes
+ *   WAIT      sets     = [allow, deny, wait],               children = [body or -1]
+ *   SWITCH    sets     = [allow, deny, case_0 .. case_k-1], children = [body_0 .. body_k-1]
+ *             (IfElse: case_0 = true_waits -> if_body, case_1 = false_waits -> else_body)
+ *   DOWHILE   sets     = [allow, deny, true_waits, false_waits], children = [body or -1] */
+typedef struct wg_op_node {
+    int32_t kind;
+    int32_t n_child, child_off;
+    int32_t n_set, set_off;
+    int32_t data_off, data_len;
+    int32_t reserved;
+} wg_op_node;
+
+typedef struct wg_vocab wg_vocab;     /* token byte strings, resident on one device */
+typedef struct wg_grammar wg_grammar; /* a compiled transition table, host side     */
+typedef struct wg_ctx wg_ctx;         /* device tables, mask cache and scratch      */
+
+typedef struct wg_stats {
+    int64_t cache_hits;      /* rows served from the cache                                  */
+    int64_t cache_misses;    /* rows whose mask had to be built (first sight of the state)  */
+    int64_t masks_built;     /* masks produced by the build kernel                          */
+    int64_t rows_uncached;   /* rows built outside the cache because it was full            */
+    int64_t tokens_rejected; /* rows of wg_advance whose token was refused                  */
+    int64_t empty_masks;     /* rows whose argmax found no allowed token                    */
+    int64_t bad_states;      /* rows with a grammar or state id out of range                */
+    int64_t cache_entries;   /* states held by the cache now                                */
+} wg_stats;
+
+/* ---- setup ------------------------------------------------------------------------- */
+
+/* Copies a vocabulary to the current device.  The tokens are given in CSR form (paper
+ * Section 3.1 keeps a token-to-id map in the structure factory; here the map is the byte
+ * string of every id): token t is bytes[offsets[t] .. offsets[t+1]).
+ *   offsets  host, V + 1 entries, non-decreasing, offsets[0] = 0
+ *   bytes    host, offsets[V] bytes (may be NULL when that is 0)
+ *   eos_id   0 <= eos_id < V; the bytes given for it are ignored
+ * The library keeps its own device copy: the first 16 bytes of every token in fixed-size
+ * records, the lengths, and the CSR arrays for longer tokens.  Free with wg_vocab_free.
+ * Errors: WG_ERR_ARG (null, V <= 0, bad offsets, eos_id out of range), WG_ERR_CUDA. */
+int32_t wg_load_vocab(const uint32_t *offsets, const uint8_t *bytes, int32_t V, int32_t eos_id,
+                      wg_vocab **out);
+void wg_vocab_free(wg_vocab *vocab);
+
+/* Lowers an operator tree to a byte-level deterministic transition table, on the host
+ * (paper Section 3.2: operator composition; the paper tracks operators per token, this
+ * library walks token BYTES, so a literal may be produced by any tokens whose bytes spell it).
+ * All pointers are host arrays in the layout described at wg_op_node.
+ * Languages: Write = its literal; Wait = stay* w body (ends at the first wait symbol, paper
+ * Section 6); Switch = stay* (s_i body_i); DoWhile = (body stay* t)* body stay* f; Sequence =
+ * concatenation; stay = (allow \ deny) \ deciding symbols; an absent body is empty.  If no
+ * set mentions EOS, the program is followed by one EOS.  After the program comes the DONE
+ * state, which accepts EOS only and stays DONE.
+ * Errors: WG_ERR_ARG for malformed arrays; WG_ERR_GRAMMAR for an empty deciding set,
+ * deciding sets that overlap each other or the deny set, or a node used twice (not a tree). */
+int32_t wg_compile_grammar(const wg_op_node *nodes, int32_t n_nodes, const int32_t *children,
+                           int32_t n_children, const uint32_t *sets, int32_t n_sets,
+                           const uint8_t *data, int32_t n_data, int32_t root, wg_grammar **out);
+void wg_grammar_free(wg_grammar *grammar);
+
+/* Host-side facts about a compiled grammar.  Any output pointer may be NULL.
+ * content_hash identifies the table: two compilations with equal tables hash equally. */
+int32_t wg_grammar_info(const wg_grammar *grammar, int32_t *n_states, int32_t *start_state,
+                        int32_t *done_state, int32_t *n_classes, uint64_t *content_hash);
+
+/* Host-side single transition: the state after `symbol` (0..256) in `state`, 0 = DEAD.
+ * Out-of-range arguments give 0.  For tests and tooling; not on the decode path. */
+int32_t wg_grammar_step(const wg_grammar *grammar, int32_t state, int32_t symbol);
+
+/* Creates the device context on the current device: grammar table registry, the mask cache
+ * (a hash table keyed by (grammar id, state id) plus a pool of `cache_capacity` mask rows,
+ * paper Section 3.3) and per-batch scratch for up to `max_batch` rows per call.
+ * cache_capacity may be 0 (every WG_USE_CACHE row is then built uncached).
+ * The vocabulary must outlive the context.  Errors: WG_ERR_ARG, WG_ERR_CUDA. */
+int32_t wg_ctx_create(const wg_vocab *vocab, int32_t cache_capacity, int32_t max_batch,
+                      wg_ctx **out);
+void wg_ctx_free(wg_ctx *ctx);
+
+/* Uploads a compiled grammar's table and returns its id in this context.  A grammar whose
+ * content_hash and tables equal one already added gets that grammar's id, so requests
+ * instantiated with the same arguments share cache entries.  Synchronous (small copies).
+ * Errors: WG_ERR_ARG, WG_ERR_CAPACITY (more than 65535 grammars), WG_ERR_CUDA. */
+int32_t wg_ctx_add_grammar(wg_ctx *ctx, const wg_grammar *grammar, int32_t *grammar_id);
+
+/* Builds and caches the mask of every state of grammar `grammar_id` (states 1..n_states-1).
+ * Stops with WG_ERR_CAPACITY if the pool cannot hold them all.  Synchronises `stream`. */
+int32_t wg_cache_prewarm(wg_ctx *ctx, int32_t grammar_id, void *stream);
+
+/* Forgets every cached mask (enqueued on `stream`). */
+int32_t wg_cache_clear(wg_ctx *ctx, void *stream);
+
+/* Copies the device counters to *out.  Synchronises `stream`. */
+int32_t wg_get_stats(wg_ctx *ctx, wg_stats *out, void *stream);
+int32_t wg_reset_stats(wg_ctx *ctx, void *stream);
+
+/* ---- the decode path --------------------------------------------------------------- */
+
+/* Cache probe (paper Section 3.3, global cache keyed by the operator state).
+ *   gid, sid  device, B entries
+ *   slot      device, B entries: pool row holding the mask of (gid[r], sid[r]), or -1
+ * Read-only: nothing is inserted.  1 <= B <= max_batch. */
+int32_t wg_mask_cache_lookup(wg_ctx *ctx, const int32_t *gid, const int32_t *sid, int32_t B,
+                             int32_t *slot, void *stream);
+
+/* Mask creation (paper Section 1 "mask creation", Section 3.3).
+ *   gid, sid          device, B entries
+ *   bitmask           device, B rows of W words, row r at bitmask + r * row_stride_words
+ *   row_stride_words  >= W
+ *   flags             WG_USE_CACHE: rows whose state is cached are copied from the pool; the
+ *                     others are built once per distinct state, inserted, then copied.  When
+ *                     the pool is full the remaining rows are built straight into `bitmask`.
+ *                     WG_NO_CACHE: every row is built, duplicates included.
+ * Rows with an unknown grammar or state get an all-zero mask and count as bad_states. */
+int32_t wg_build_masks(wg_ctx *ctx, const int32_t *gid, const int32_t *sid, int32_t B,
+                       uint32_t *bitmask, int64_t row_stride_words, uint32_t flags, void *stream);
+
+/* Mask application (paper Section 1: applied to the logits prior to sampling), in place.
+ *   logits            device, B rows of V elements, row r at logits + r * row_stride_elems
+ *   dtype             WG_DTYPE_BF16 or WG_DTYPE_FP32
+ *   bitmask           device, as written by wg_build_masks
+ *   argmax_out        device, B entries, or NULL.  When given, token[r] = the lowest id among
+ *                     the maxima of the allowed logits (-0.0 equals +0.0), or -1 for an
+ *                     empty mask.  NaN logits are outside the contract.
+ *   workspace         device scratch of wg_apply_workspace_bytes(B) bytes, 8-byte aligned;
+ *                     needed only with argmax_out, may be NULL otherwise.  Contents are
+ *                     overwritten.
+ * Disallowed elements become -inf (bf16 0xFF80, fp32 0xFF800000); all others keep their bits.
+ * Fastest when logits is 32-byte aligned and row_stride_elems * element size is a multiple
+ * of 32 bytes; other layouts take a slower element-wise kernel with identical results. */
+int32_t wg_apply_mask(void *logits, int32_t dtype, int64_t row_stride_elems,
+                      const uint32_t *bitmask, int64_t mask_stride_words, int32_t B, int32_t V,
+                      int32_t *argmax_out, void *workspace, void *stream);
+size_t wg_apply_workspace_bytes(int32_t B);
+
+/* State tracking (paper Section 3.2: the current token id updates the state machine).
+ *   gid     device, B entries
+ *   sid     device, B entries, updated in place
+ *   token   device, B entries
+ *   status  device, B entries, or NULL: WG_OK, WG_ERR_TOKEN_REJECTED (state unchanged; also
+ *           for token ids outside 0..V-1) or WG_ERR_STATE
+ *   flags   0 or WG_RESTART_ON_DONE */
+int32_t wg_advance(wg_ctx *ctx, const int32_t *gid, int32_t *sid, const int32_t *token,
+                   int32_t B, int32_t *status, uint32_t flags, void *stream);
+
+/* One whole decode step on device buffers: cache lookup, build of the misses, mask rows out,
+ * apply with greedy argmax, state advance.  Same results as the four calls above in that
+ * order, in fewer kernel launches (the rows are copied from the cache pool inside the apply
+ * kernel).  flags: WG_USE_CACHE or WG_NO_CACHE, optionally | WG_RESTART_ON_DONE.
+ *   token_out  device, B entries (the greedy choice, -1 for an empty mask)
+ *   status     device, B entries, or NULL (WG_OK, WG_ERR_EMPTY_MASK, WG_ERR_STATE) */
+int32_t wg_decode_step(wg_ctx *ctx, const int32_t *gid, int32_t *sid, int32_t B, void *logits,
+                       int32_t dtype, int64_t row_stride_elems, uint32_t *bitmask,
+                       int64_t mask_stride_words, int32_t *token_out, int32_t *status,
+                       uint32_t flags, void *stream);
+
+/* The same step for a caller whose logits live in HOST memory (pinned memory makes the
+ * copies asynchronous): copies logits_host to the device buffer `logits_dev`, runs
+ * wg_decode_step, copies the chosen tokens back to token_host and synchronises `stream`.
+ *   logits_host  host, B * V elements, rows contiguous
+ *   logits_dev   device staging, B rows of row_stride_elems elements
+ *   token_dev    device, B entries; token_host host, B entries */
+int32_t wg_decode_step_host(wg_ctx *ctx, const int32_t *gid, int32_t *sid, int32_t B,
+                            const void *logits_host, void *logits_dev, int32_t dtype,
+                            int64_t row_stride_elems, uint32_t *bitmask,
+                            int64_t mask_stride_words, int32_t *token_dev, int32_t *token_host,
+                            int32_t *status, uint32_t flags, void *stream);
+
+/* ---- diagnostics ------------------------------------------------------------------- */
+
+/* Per-kernel timing for benchmarks.  While enabled, wg_decode_step records CUDA events on the
+ * caller's stream around its mask-build kernel and around its apply kernel (at most 8192
+ * steps are kept between two reads).  wg_ctx_get_timing waits for the recorded events, adds
+ * up the elapsed milliseconds of each kernel over the recorded steps, and forgets them.
+ * Any output pointer may be NULL. */
+int32_t wg_ctx_set_timing(wg_ctx *ctx, int32_t enable);
+int32_t wg_ctx_get_timing(wg_ctx *ctx, double *build_ms, double *apply_ms, int64_t *steps);
+
+const char *wg_strerror(int32_t status);
+/* cudaError_t of the last failed CUDA call on this thread (0 if none). */
+int32_t wg_last_cuda_error(void);
+/* Number of kernels this library has launched since load (all contexts, all threads). */
+int64_t wg_kernel_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* WG_H_ */

@@ -1,0 +1,329 @@
+"""Thin ctypes binding of the C ABI in ``include/wg.h``.
+
+Argument marshalling only: every step of the path runs in the library's CUDA kernels.
+Device buffers are ``torch`` tensors (PyTorch is used for device memory and streams); host
+arrays are numpy.  There is no CPU fallback: if ``libwg.so`` has not been built, importing
+this module fails.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional
+
+import numpy as np
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libwg.so")
+
+WG_OK = 0
+WG_ERR_ARG = -1
+WG_ERR_GRAMMAR = -2
+WG_ERR_CAPACITY = -3
+WG_ERR_TOKEN_REJECTED = -4
+WG_ERR_CUDA = -5
+WG_ERR_EMPTY_MASK = -6
+WG_ERR_STATE = -7
+
+WG_DTYPE_BF16 = 0
+WG_DTYPE_FP32 = 1
+WG_USE_CACHE = 0
+WG_NO_CACHE = 1
+WG_RESTART_ON_DONE = 2
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        f"{LIB_PATH} is missing: build it with `python -m paper_2507_16768_b200.build` "
+        "(nvcc, sm_100a). This package has no CPU fallback.")
+
+_lib = C.CDLL(LIB_PATH)
+
+
+class WgStats(C.Structure):
+    _fields_ = [(n, C.c_int64) for n in (
+        "cache_hits", "cache_misses", "masks_built", "rows_uncached", "tokens_rejected",
+        "empty_masks", "bad_states", "cache_entries")]
+
+    def as_dict(self):
+        return {n: int(getattr(self, n)) for n, _ in self._fields_}
+
+
+_vp, _i32, _i64, _u32 = C.c_void_p, C.c_int32, C.c_int64, C.c_uint32
+_SIGNATURES = {
+    "wg_load_vocab": (_i32, [_vp, _vp, _i32, _i32, C.POINTER(_vp)]),
+    "wg_vocab_free": (None, [_vp]),
+    "wg_compile_grammar": (_i32, [_vp, _i32, _vp, _i32, _vp, _i32, _vp, _i32, _i32, C.POINTER(_vp)]),
+    "wg_grammar_free": (None, [_vp]),
+    "wg_grammar_info": (_i32, [_vp, C.POINTER(_i32), C.POINTER(_i32), C.POINTER(_i32),
+                               C.POINTER(_i32), C.POINTER(C.c_uint64)]),
+    "wg_grammar_step": (_i32, [_vp, _i32, _i32]),
+    "wg_ctx_create": (_i32, [_vp, _i32, _i32, C.POINTER(_vp)]),
+    "wg_ctx_free": (None, [_vp]),
+    "wg_ctx_add_grammar": (_i32, [_vp, _vp, C.POINTER(_i32)]),
+    "wg_cache_prewarm": (_i32, [_vp, _i32, _vp]),
+    "wg_cache_clear": (_i32, [_vp, _vp]),
+    "wg_get_stats": (_i32, [_vp, C.POINTER(WgStats), _vp]),
+    "wg_reset_stats": (_i32, [_vp, _vp]),
+    "wg_mask_cache_lookup": (_i32, [_vp, _vp, _vp, _i32, _vp, _vp]),
+    "wg_build_masks": (_i32, [_vp, _vp, _vp, _i32, _vp, _i64, _u32, _vp]),
+    "wg_apply_mask": (_i32, [_vp, _i32, _i64, _vp, _i64, _i32, _i32, _vp, _vp, _vp]),
+    "wg_apply_workspace_bytes": (C.c_size_t, [_i32]),
+    "wg_advance": (_i32, [_vp, _vp, _vp, _vp, _i32, _vp, _u32, _vp]),
+    "wg_decode_step": (_i32, [_vp, _vp, _vp, _i32, _vp, _i32, _i64, _vp, _i64, _vp, _vp, _u32, _vp]),
+    "wg_decode_step_host": (_i32, [_vp, _vp, _vp, _i32, _vp, _vp, _i32, _i64, _vp, _i64, _vp, _vp,
+                                   _vp, _u32, _vp]),
+    "wg_ctx_set_timing": (_i32, [_vp, _i32]),
+    "wg_ctx_get_timing": (_i32, [_vp, C.POINTER(C.c_double), C.POINTER(C.c_double),
+                                 C.POINTER(_i64)]),
+    "wg_strerror": (C.c_char_p, [_i32]),
+    "wg_last_cuda_error": (_i32, []),
+    "wg_kernel_launch_count": (_i64, []),
+}
+for _name, (_res, _args) in _SIGNATURES.items():
+    _f = getattr(_lib, _name)
+    _f.restype = _res
+    _f.argtypes = _args
+
+EXPORTED = tuple(_SIGNATURES)
+
+
+class WgError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        msg = _lib.wg_strerror(int(status)).decode()
+        if status == WG_ERR_CUDA:
+            msg += f" (cudaError {_lib.wg_last_cuda_error()})"
+        super().__init__(f"{where}: {msg} [{status}]")
+        self.status = int(status)
+
+
+def _check(status: int, where: str) -> None:
+    if status != WG_OK:
+        raise WgError(status, where)
+
+
+def _np_ptr(a: Optional[np.ndarray]):
+    return None if a is None else a.ctypes.data_as(C.c_void_p)
+
+
+def _dev_ptr(t, dtype=None, what: str = "tensor"):
+    """Raw device pointer of a torch CUDA tensor (None passes through)."""
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise TypeError(f"{what} must be a CUDA tensor")
+    if dtype is not None and t.dtype not in (dtype if isinstance(dtype, tuple) else (dtype,)):
+        raise TypeError(f"{what} has dtype {t.dtype}")
+    return C.c_void_p(t.data_ptr())
+
+
+def _stream_ptr(stream):
+    if stream is None:
+        import torch
+        stream = torch.cuda.current_stream()
+    return C.c_void_p(stream.cuda_stream)
+
+
+def kernel_launch_count() -> int:
+    return int(_lib.wg_kernel_launch_count())
+
+
+class Vocab:
+    """wg_load_vocab: copies a CSR vocabulary (numpy, host) to the current device."""
+
+    def __init__(self, offsets: np.ndarray, data: np.ndarray, eos_id: int):
+        self._offsets = np.ascontiguousarray(offsets, np.uint32)
+        self._data = np.ascontiguousarray(data, np.uint8)
+        self.V = int(self._offsets.shape[0] - 1)
+        self.W = (self.V + 31) // 32
+        self.eos_id = int(eos_id)
+        h = _vp()
+        _check(_lib.wg_load_vocab(_np_ptr(self._offsets), _np_ptr(self._data), self.V, self.eos_id,
+                                  C.byref(h)), "wg_load_vocab")
+        self.handle = h
+
+    def close(self):
+        if getattr(self, "handle", None):
+            _lib.wg_vocab_free(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        self.close()
+
+
+class Grammar:
+    """wg_compile_grammar: lowers a flat operator tree to a byte-level table (host side)."""
+
+    def __init__(self, flat):
+        nodes = np.ascontiguousarray(flat.nodes, np.int32)
+        children = np.ascontiguousarray(flat.children, np.int32)
+        sets = np.ascontiguousarray(flat.sets, np.uint32)
+        data = np.ascontiguousarray(flat.data, np.uint8)
+        h = _vp()
+        _check(_lib.wg_compile_grammar(_np_ptr(nodes), nodes.shape[0], _np_ptr(children),
+                                       children.shape[0], _np_ptr(sets), sets.shape[0],
+                                       _np_ptr(data), data.shape[0], int(flat.root), C.byref(h)),
+               "wg_compile_grammar")
+        self.handle = h
+        n, s, d, c, hs = _i32(), _i32(), _i32(), _i32(), C.c_uint64()
+        _check(_lib.wg_grammar_info(h, C.byref(n), C.byref(s), C.byref(d), C.byref(c), C.byref(hs)),
+               "wg_grammar_info")
+        self.n_states, self.start_state, self.done_state = n.value, s.value, d.value
+        self.n_classes, self.content_hash = c.value, hs.value
+
+    def step(self, state: int, symbol: int) -> int:
+        return int(_lib.wg_grammar_step(self.handle, int(state), int(symbol)))
+
+    def walk(self, state: int, symbols) -> int:
+        for s in symbols:
+            state = self.step(state, s)
+        return state
+
+    def close(self):
+        if getattr(self, "handle", None):
+            _lib.wg_grammar_free(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        self.close()
+
+
+class Context:
+    """wg_ctx: device tables, the mask cache and per-batch scratch."""
+
+    def __init__(self, vocab: Vocab, cache_capacity: int, max_batch: int):
+        self.vocab = vocab
+        self.max_batch = int(max_batch)
+        h = _vp()
+        _check(_lib.wg_ctx_create(vocab.handle, int(cache_capacity), int(max_batch), C.byref(h)),
+               "wg_ctx_create")
+        self.handle = h
+
+    def close(self):
+        if getattr(self, "handle", None):
+            _lib.wg_ctx_free(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        self.close()
+
+    def add_grammar(self, grammar: Grammar) -> int:
+        gid = _i32()
+        _check(_lib.wg_ctx_add_grammar(self.handle, grammar.handle, C.byref(gid)),
+               "wg_ctx_add_grammar")
+        return gid.value
+
+    def cache_prewarm(self, grammar_id: int, stream=None) -> None:
+        _check(_lib.wg_cache_prewarm(self.handle, int(grammar_id), _stream_ptr(stream)),
+               "wg_cache_prewarm")
+
+    def cache_clear(self, stream=None) -> None:
+        _check(_lib.wg_cache_clear(self.handle, _stream_ptr(stream)), "wg_cache_clear")
+
+    def stats(self, stream=None) -> dict:
+        st = WgStats()
+        _check(_lib.wg_get_stats(self.handle, C.byref(st), _stream_ptr(stream)), "wg_get_stats")
+        return st.as_dict()
+
+    def set_timing(self, enable: bool) -> None:
+        _check(_lib.wg_ctx_set_timing(self.handle, int(bool(enable))), "wg_ctx_set_timing")
+
+    def get_timing(self) -> dict:
+        """Summed kernel milliseconds of the steps recorded since the last read."""
+        b, a, n = C.c_double(), C.c_double(), _i64()
+        _check(_lib.wg_ctx_get_timing(self.handle, C.byref(b), C.byref(a), C.byref(n)),
+               "wg_ctx_get_timing")
+        return {"build_ms": b.value, "apply_ms": a.value, "steps": int(n.value)}
+
+    def reset_stats(self, stream=None) -> None:
+        _check(_lib.wg_reset_stats(self.handle, _stream_ptr(stream)), "wg_reset_stats")
+
+
+def _logits_dtype(logits) -> int:
+    import torch
+    if logits.dtype == torch.bfloat16:
+        return WG_DTYPE_BF16
+    if logits.dtype == torch.float32:
+        return WG_DTYPE_FP32
+    raise TypeError(f"logits must be bfloat16 or float32, not {logits.dtype}")
+
+
+def _rows(t, what: str):
+    if t.dim() != 2 or t.stride(1) != 1:
+        raise ValueError(f"{what} must be 2-D with unit inner stride")
+    return t.shape[0], t.stride(0)
+
+
+def wg_mask_cache_lookup(ctx: Context, gid, sid, slot, stream=None) -> None:
+    import torch
+    B = gid.shape[0]
+    _check(_lib.wg_mask_cache_lookup(ctx.handle, _dev_ptr(gid, torch.int32, "gid"),
+                                     _dev_ptr(sid, torch.int32, "sid"), B,
+                                     _dev_ptr(slot, torch.int32, "slot"), _stream_ptr(stream)),
+           "wg_mask_cache_lookup")
+
+
+def wg_build_masks(ctx: Context, gid, sid, bitmask, flags: int = WG_USE_CACHE, stream=None) -> None:
+    import torch
+    B, stride = _rows(bitmask, "bitmask")
+    _check(_lib.wg_build_masks(ctx.handle, _dev_ptr(gid, torch.int32, "gid"),
+                               _dev_ptr(sid, torch.int32, "sid"), B,
+                               _dev_ptr(bitmask, (torch.int32, torch.uint32), "bitmask"), stride,
+                               int(flags), _stream_ptr(stream)), "wg_build_masks")
+
+
+def wg_apply_mask(logits, bitmask, V: int, argmax_out=None, workspace=None, stream=None) -> None:
+    import torch
+    B, stride = _rows(logits, "logits")
+    Bm, mstride = _rows(bitmask, "bitmask")
+    if Bm != B:
+        raise ValueError("logits and bitmask disagree on the batch size")
+    _check(_lib.wg_apply_mask(_dev_ptr(logits, None, "logits"), _logits_dtype(logits), stride,
+                              _dev_ptr(bitmask, (torch.int32, torch.uint32), "bitmask"), mstride,
+                              B, int(V), _dev_ptr(argmax_out, torch.int32, "argmax_out"),
+                              _dev_ptr(workspace, None, "workspace"), _stream_ptr(stream)),
+           "wg_apply_mask")
+
+
+def wg_apply_workspace_bytes(B: int) -> int:
+    return int(_lib.wg_apply_workspace_bytes(int(B)))
+
+
+def wg_advance(ctx: Context, gid, sid, token, status=None, flags: int = 0, stream=None) -> None:
+    import torch
+    B = gid.shape[0]
+    _check(_lib.wg_advance(ctx.handle, _dev_ptr(gid, torch.int32, "gid"),
+                           _dev_ptr(sid, torch.int32, "sid"), _dev_ptr(token, torch.int32, "token"),
+                           B, _dev_ptr(status, torch.int32, "status"), int(flags),
+                           _stream_ptr(stream)), "wg_advance")
+
+
+def wg_decode_step(ctx: Context, gid, sid, logits, bitmask, token_out, status=None,
+                   flags: int = WG_USE_CACHE, stream=None) -> None:
+    import torch
+    B, stride = _rows(logits, "logits")
+    _, mstride = _rows(bitmask, "bitmask")
+    _check(_lib.wg_decode_step(ctx.handle, _dev_ptr(gid, torch.int32, "gid"),
+                               _dev_ptr(sid, torch.int32, "sid"), B,
+                               _dev_ptr(logits, None, "logits"), _logits_dtype(logits), stride,
+                               _dev_ptr(bitmask, (torch.int32, torch.uint32), "bitmask"), mstride,
+                               _dev_ptr(token_out, torch.int32, "token_out"),
+                               _dev_ptr(status, torch.int32, "status"), int(flags),
+                               _stream_ptr(stream)), "wg_decode_step")
+
+
+def wg_decode_step_host(ctx: Context, gid, sid, logits_host, logits_dev, bitmask, token_dev,
+                        token_host, status=None, flags: int = WG_USE_CACHE, stream=None) -> None:
+    """logits_host / token_host are CPU tensors (pinned for asynchronous copies)."""
+    import torch
+    B, stride = _rows(logits_dev, "logits_dev")
+    _, mstride = _rows(bitmask, "bitmask")
+    if logits_host.is_cuda or token_host.is_cuda or not logits_host.is_contiguous():
+        raise TypeError("logits_host and token_host must be contiguous CPU tensors")
+    _check(_lib.wg_decode_step_host(
+        ctx.handle, _dev_ptr(gid, torch.int32, "gid"), _dev_ptr(sid, torch.int32, "sid"), B,
+        C.c_void_p(logits_host.data_ptr()), _dev_ptr(logits_dev, None, "logits_dev"),
+        _logits_dtype(logits_dev), stride,
+        _dev_ptr(bitmask, (torch.int32, torch.uint32), "bitmask"), mstride,
+        _dev_ptr(token_dev, torch.int32, "token_dev"), C.c_void_p(token_host.data_ptr()),
+        _dev_ptr(status, torch.int32, "status"), int(flags), _stream_ptr(stream)),
+        "wg_decode_step_host")

@@ -1,0 +1,605 @@
+// Host side of the C ABI declared in wg.h: object lifetimes, uploads and kernel launches.
+#include <atomic>
+#include <cstdio>
+#include <cstring>
+#include <mutex>
+#include <new>
+#include <vector>
+
+#include "wg_kernels.cuh"
+
+namespace {
+
+thread_local int32_t g_last_cuda_error = 0;
+std::atomic<int64_t> g_launches{0};
+
+#define WG_CUDA(expr)                                   \
+    do {                                                \
+        cudaError_t e__ = (expr);                       \
+        if (e__ != cudaSuccess) {                       \
+            g_last_cuda_error = (int32_t)e__;           \
+            return WG_ERR_CUDA;                         \
+        }                                               \
+    } while (0)
+
+// after a <<< >>> launch: count it and pick up a launch-configuration error
+#define WG_LAUNCHED()                                   \
+    do {                                                \
+        g_launches.fetch_add(1, std::memory_order_relaxed); \
+        WG_CUDA(cudaGetLastError());                    \
+    } while (0)
+
+int g_sm_count = 0;
+int sm_count() {
+    if (g_sm_count == 0) {
+        int dev = 0, n = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess &&
+            cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0)
+            g_sm_count = n;
+        else
+            g_sm_count = 148;
+    }
+    return g_sm_count;
+}
+
+template <typename T>
+int32_t dev_alloc(T **p, size_t n) {
+    *p = nullptr;
+    WG_CUDA(cudaMalloc((void **)p, (n ? n : 1) * sizeof(T)));
+    return WG_OK;
+}
+
+}  // namespace
+
+struct wg_vocab {
+    VocabDev dev{};
+    void *d_rec = nullptr, *d_len = nullptr, *d_offsets = nullptr, *d_bytes = nullptr;
+    int device = 0;
+};
+
+struct GrammarSlot {
+    uint64_t hash;
+    std::vector<int32_t> table;  // host copy, for exact comparison on hash equality
+    int32_t n_states, n_classes;
+    void *d_table, *d_cls;
+};
+
+struct wg_ctx {
+    const wg_vocab *vocab = nullptr;
+    CtxDev dev{};
+    std::vector<GrammarDev> grammars;  // host mirror of dev.grammars
+    std::vector<GrammarSlot> slots;
+    GrammarDev *d_grammars = nullptr;
+    int32_t grammar_cap = 0;
+    int32_t max_batch = 0;
+    int32_t *d_stage_gid = nullptr, *d_stage_sid = nullptr;  // prewarm staging
+    std::vector<void *> owned;  // every other device allocation
+    std::mutex mu;
+    // optional per-kernel timing: events[4 * i + {0,1,2,3}] = build begin/end, apply begin/end
+    bool timing = false;
+    std::vector<cudaEvent_t> events;
+    size_t timed_steps = 0;
+};
+
+namespace {
+constexpr size_t MAX_TIMED_STEPS = 8192;
+
+// Records event `which` (0..3) of the current timed step; grows the event pool on demand.
+int32_t timing_mark(wg_ctx *c, int which, cudaStream_t st) {
+    if (!c->timing || c->timed_steps >= MAX_TIMED_STEPS) return WG_OK;
+    const size_t idx = 4 * c->timed_steps + (size_t)which;
+    while (c->events.size() <= idx) {
+        cudaEvent_t e;
+        WG_CUDA(cudaEventCreate(&e));
+        c->events.push_back(e);
+    }
+    WG_CUDA(cudaEventRecord(c->events[idx], st));
+    if (which == 3) ++c->timed_steps;
+    return WG_OK;
+}
+}  // namespace
+
+extern "C" {
+
+const char *wg_strerror(int32_t status) {
+    switch (status) {
+    case WG_OK: return "ok";
+    case WG_ERR_ARG: return "bad argument";
+    case WG_ERR_GRAMMAR: return "operator tree breaks a grammar rule";
+    case WG_ERR_CAPACITY: return "capacity exhausted";
+    case WG_ERR_TOKEN_REJECTED: return "token not allowed in this state";
+    case WG_ERR_CUDA: return "CUDA runtime error";
+    case WG_ERR_EMPTY_MASK: return "no token allowed";
+    case WG_ERR_STATE: return "grammar or state id out of range";
+    default: return "unknown status";
+    }
+}
+
+int32_t wg_last_cuda_error(void) { return g_last_cuda_error; }
+int64_t wg_kernel_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+// ---- vocabulary ---------------------------------------------------------------------
+
+int32_t wg_load_vocab(const uint32_t *offsets, const uint8_t *bytes, int32_t V, int32_t eos_id,
+                      wg_vocab **out) {
+    if (!out) return WG_ERR_ARG;
+    *out = nullptr;
+    if (!offsets || V <= 0 || eos_id < 0 || eos_id >= V || offsets[0] != 0) return WG_ERR_ARG;
+    for (int32_t t = 0; t < V; ++t)
+        if (offsets[t + 1] < offsets[t]) return WG_ERR_ARG;
+    const uint32_t total = offsets[V];
+    if (total > 0 && !bytes) return WG_ERR_ARG;
+
+    std::vector<uint8_t> rec((size_t)V * WG_REC_BYTES, 0), len(V, 0);
+    for (int32_t t = 0; t < V; ++t) {
+        const uint32_t n = (t == eos_id) ? 0u : offsets[t + 1] - offsets[t];
+        len[t] = (uint8_t)(n > 255u ? 255u : n);
+        if (n) memcpy(&rec[(size_t)t * WG_REC_BYTES], bytes + offsets[t], n < WG_REC_BYTES ? n : WG_REC_BYTES);
+    }
+    wg_vocab *v = new (std::nothrow) wg_vocab();
+    if (!v) return WG_ERR_ARG;
+    auto fail = [&](int32_t rc) { wg_vocab_free(v); return rc; };
+    if (cudaGetDevice(&v->device) != cudaSuccess) return fail(WG_ERR_CUDA);
+    if (cudaMalloc(&v->d_rec, rec.size()) != cudaSuccess ||
+        cudaMalloc(&v->d_len, len.size()) != cudaSuccess ||
+        cudaMalloc(&v->d_offsets, sizeof(uint32_t) * ((size_t)V + 1)) != cudaSuccess ||
+        cudaMalloc(&v->d_bytes, total ? total : 1) != cudaSuccess)
+        return fail(WG_ERR_CUDA);
+    if (cudaMemcpy(v->d_rec, rec.data(), rec.size(), cudaMemcpyHostToDevice) != cudaSuccess ||
+        cudaMemcpy(v->d_len, len.data(), len.size(), cudaMemcpyHostToDevice) != cudaSuccess ||
+        cudaMemcpy(v->d_offsets, offsets, sizeof(uint32_t) * ((size_t)V + 1),
+                   cudaMemcpyHostToDevice) != cudaSuccess ||
+        (total && cudaMemcpy(v->d_bytes, bytes, total, cudaMemcpyHostToDevice) != cudaSuccess))
+        return fail(WG_ERR_CUDA);
+    v->dev.rec = static_cast<const uint4 *>(v->d_rec);
+    v->dev.len = static_cast<const uint8_t *>(v->d_len);
+    v->dev.offsets = static_cast<const uint32_t *>(v->d_offsets);
+    v->dev.bytes = static_cast<const uint8_t *>(v->d_bytes);
+    v->dev.V = V;
+    v->dev.W = (V + 31) / 32;
+    v->dev.eos_id = eos_id;
+    *out = v;
+    return WG_OK;
+}
+
+void wg_vocab_free(wg_vocab *v) {
+    if (!v) return;
+    cudaFree(v->d_rec);
+    cudaFree(v->d_len);
+    cudaFree(v->d_offsets);
+    cudaFree(v->d_bytes);
+    delete v;
+}
+
+// ---- grammars -----------------------------------------------------------------------
+
+int32_t wg_compile_grammar(const wg_op_node *nodes, int32_t n_nodes, const int32_t *children,
+                           int32_t n_children, const uint32_t *sets, int32_t n_sets,
+                           const uint8_t *data, int32_t n_data, int32_t root, wg_grammar **out) {
+    if (!out) return WG_ERR_ARG;
+    *out = nullptr;
+    wg_grammar *g = new (std::nothrow) wg_grammar();
+    if (!g) return WG_ERR_ARG;
+    int32_t rc;
+    try {
+        rc = wg_lower_tree(nodes, n_nodes, children, n_children, sets, n_sets, data, n_data, root, g);
+    } catch (const std::bad_alloc &) {
+        rc = WG_ERR_CAPACITY;
+    }
+    if (rc != WG_OK) {
+        delete g;
+        return rc;
+    }
+    *out = g;
+    return WG_OK;
+}
+
+void wg_grammar_free(wg_grammar *g) { delete g; }
+
+int32_t wg_grammar_info(const wg_grammar *g, int32_t *n_states, int32_t *start_state,
+                        int32_t *done_state, int32_t *n_classes, uint64_t *content_hash) {
+    if (!g) return WG_ERR_ARG;
+    if (n_states) *n_states = g->n_states;
+    if (start_state) *start_state = g->start;
+    if (done_state) *done_state = g->done;
+    if (n_classes) *n_classes = g->n_classes;
+    if (content_hash) *content_hash = g->hash;
+    return WG_OK;
+}
+
+int32_t wg_grammar_step(const wg_grammar *g, int32_t state, int32_t symbol) {
+    if (!g || state < 0 || state >= g->n_states || symbol < 0 || symbol >= WG_N_SYMBOLS) return 0;
+    const int c = symbol == WG_SYM_EOS ? g->eos_class : g->byte_class[symbol];
+    return g->table[(size_t)state * g->n_classes + c];
+}
+
+// ---- context ------------------------------------------------------------------------
+
+int32_t wg_ctx_create(const wg_vocab *vocab, int32_t cache_capacity, int32_t max_batch,
+                      wg_ctx **out) {
+    if (!out) return WG_ERR_ARG;
+    *out = nullptr;
+    if (!vocab || cache_capacity < 0 || max_batch <= 0 || cache_capacity > (1 << 28))
+        return WG_ERR_ARG;
+    wg_ctx *c = new (std::nothrow) wg_ctx();
+    if (!c) return WG_ERR_ARG;
+    c->vocab = vocab;
+    c->max_batch = max_batch;
+    CtxDev &d = c->dev;
+    d.capacity = cache_capacity;
+    d.pool_stride = ((int64_t)vocab->dev.W + 31) / 32 * 32;  // rows start on 128-byte lines
+    d.hash_size = 0;
+    if (cache_capacity > 0) {
+        int32_t h = 64;
+        while (h < 2 * cache_capacity) h <<= 1;
+        d.hash_size = h;
+    }
+    int32_t rc = WG_OK;
+    auto take = [&](auto **p, size_t n) {
+        if (rc != WG_OK) return;
+        rc = dev_alloc(p, n);
+        if (rc == WG_OK) c->owned.push_back((void *)*p);
+    };
+    take(&d.keys, (size_t)d.hash_size);
+    take(&d.vals, (size_t)d.hash_size);
+    take(&d.pool, (size_t)d.capacity * (size_t)d.pool_stride);
+    take(&d.n_slots, 1);
+    take(&d.ent, (size_t)max_batch);
+    take(&d.slot, (size_t)max_batch);
+    take(&d.bl_gid, (size_t)max_batch);
+    take(&d.bl_sid, (size_t)max_batch);
+    take(&d.bl_dst, (size_t)max_batch);
+    take(&d.bl_count, 1);
+    take(&d.argkey, (size_t)max_batch);
+    take(&d.stats, (size_t)ST_COUNT);
+    take(&c->d_stage_gid, (size_t)max_batch);
+    take(&c->d_stage_sid, (size_t)max_batch);
+    c->grammar_cap = 64;
+    take(&c->d_grammars, (size_t)c->grammar_cap);
+    if (rc == WG_OK) {
+        d.grammars = c->d_grammars;
+        d.n_grammars = 0;
+        if (cudaMemset(d.keys, 0, sizeof(unsigned long long) * (size_t)(d.hash_size ? d.hash_size : 1)) != cudaSuccess ||
+            cudaMemset(d.vals, 0xFF, sizeof(int32_t) * (size_t)(d.hash_size ? d.hash_size : 1)) != cudaSuccess ||
+            cudaMemset(d.n_slots, 0, sizeof(int32_t)) != cudaSuccess ||
+            cudaMemset(d.bl_count, 0, sizeof(int32_t)) != cudaSuccess ||
+            cudaMemset(d.argkey, 0, sizeof(unsigned long long) * (size_t)max_batch) != cudaSuccess ||
+            cudaMemset(d.stats, 0, sizeof(unsigned long long) * ST_COUNT) != cudaSuccess)
+            rc = WG_ERR_CUDA;
+    }
+    if (rc != WG_OK) {
+        wg_ctx_free(c);
+        return rc;
+    }
+    *out = c;
+    return WG_OK;
+}
+
+void wg_ctx_free(wg_ctx *c) {
+    if (!c) return;
+    cudaDeviceSynchronize();
+    for (void *p : c->owned) cudaFree(p);
+    for (cudaEvent_t e : c->events) cudaEventDestroy(e);
+    for (GrammarSlot &s : c->slots) {
+        cudaFree(s.d_table);
+        cudaFree(s.d_cls);
+    }
+    delete c;
+}
+
+int32_t wg_ctx_add_grammar(wg_ctx *c, const wg_grammar *g, int32_t *grammar_id) {
+    if (!c || !g || !grammar_id) return WG_ERR_ARG;
+    std::lock_guard<std::mutex> lock(c->mu);
+    for (size_t i = 0; i < c->slots.size(); ++i) {
+        const GrammarSlot &s = c->slots[i];
+        if (s.hash == g->hash && s.n_states == g->n_states && s.n_classes == g->n_classes &&
+            s.table == g->table) {
+            *grammar_id = (int32_t)i;
+            return WG_OK;
+        }
+    }
+    if (c->slots.size() >= 65535) return WG_ERR_CAPACITY;
+    const bool wide = g->n_states > 65535;
+    GrammarSlot slot{g->hash, g->table, g->n_states, g->n_classes, nullptr, nullptr};
+    const size_t n = g->table.size();
+    if (wide) {
+        WG_CUDA(cudaMalloc(&slot.d_table, n * sizeof(uint32_t)));
+        WG_CUDA(cudaMemcpy(slot.d_table, g->table.data(), n * sizeof(uint32_t), cudaMemcpyHostToDevice));
+    } else {
+        std::vector<uint16_t> narrow(n);
+        for (size_t i = 0; i < n; ++i) narrow[i] = (uint16_t)g->table[i];
+        WG_CUDA(cudaMalloc(&slot.d_table, n * sizeof(uint16_t)));
+        WG_CUDA(cudaMemcpy(slot.d_table, narrow.data(), n * sizeof(uint16_t), cudaMemcpyHostToDevice));
+    }
+    WG_CUDA(cudaMalloc(&slot.d_cls, 256));
+    WG_CUDA(cudaMemcpy(slot.d_cls, g->byte_class, 256, cudaMemcpyHostToDevice));
+    GrammarDev gd{slot.d_table, static_cast<const uint8_t *>(slot.d_cls), g->n_states,
+                  g->n_classes, g->start, g->done, g->eos_class, wide ? 1 : 0};
+    const int32_t id = (int32_t)c->slots.size();
+    if (id >= c->grammar_cap) {  // grow the registry; queued kernels still read the old one
+        WG_CUDA(cudaDeviceSynchronize());
+        const int32_t cap = c->grammar_cap * 2;
+        GrammarDev *bigger = nullptr;
+        WG_CUDA(cudaMalloc((void **)&bigger, sizeof(GrammarDev) * (size_t)cap));
+        WG_CUDA(cudaMemcpy(bigger, c->grammars.data(), sizeof(GrammarDev) * c->grammars.size(),
+                           cudaMemcpyHostToDevice));
+        c->owned.push_back(bigger);  // the old array is freed with the context
+        c->d_grammars = bigger;
+        c->grammar_cap = cap;
+        c->dev.grammars = bigger;
+    }
+    WG_CUDA(cudaMemcpy(c->d_grammars + id, &gd, sizeof(GrammarDev), cudaMemcpyHostToDevice));
+    c->grammars.push_back(gd);
+    c->slots.push_back(std::move(slot));
+    c->dev.n_grammars = id + 1;
+    *grammar_id = id;
+    return WG_OK;
+}
+
+int32_t wg_cache_clear(wg_ctx *c, void *stream) {
+    if (!c) return WG_ERR_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int n = c->dev.hash_size > 0 ? c->dev.hash_size : 1;
+    cache_clear_kernel<<<(n + 255) / 256, 256, 0, st>>>(c->dev);
+    WG_LAUNCHED();
+    return WG_OK;
+}
+
+int32_t wg_get_stats(wg_ctx *c, wg_stats *out, void *stream) {
+    if (!c || !out) return WG_ERR_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    unsigned long long h[ST_COUNT];
+    int32_t n_slots = 0;
+    WG_CUDA(cudaMemcpyAsync(h, c->dev.stats, sizeof(h), cudaMemcpyDeviceToHost, st));
+    WG_CUDA(cudaMemcpyAsync(&n_slots, c->dev.n_slots, sizeof(n_slots), cudaMemcpyDeviceToHost, st));
+    WG_CUDA(cudaStreamSynchronize(st));
+    out->cache_hits = (int64_t)h[ST_HITS];
+    out->cache_misses = (int64_t)h[ST_MISSES];
+    out->masks_built = (int64_t)h[ST_BUILT];
+    out->rows_uncached = (int64_t)h[ST_UNCACHED];
+    out->tokens_rejected = (int64_t)h[ST_REJECTED];
+    out->empty_masks = (int64_t)h[ST_EMPTY];
+    out->bad_states = (int64_t)h[ST_BAD_STATE];
+    out->cache_entries = n_slots;
+    return WG_OK;
+}
+
+int32_t wg_reset_stats(wg_ctx *c, void *stream) {
+    if (!c) return WG_ERR_ARG;
+    WG_CUDA(cudaMemsetAsync(c->dev.stats, 0, sizeof(unsigned long long) * ST_COUNT,
+                            static_cast<cudaStream_t>(stream)));
+    return WG_OK;
+}
+
+}  // extern "C"
+
+// ---- launch helpers -------------------------------------------------------------------
+namespace {
+
+int32_t launch_build(wg_ctx *c, const BuildWork &work, int max_entries, cudaStream_t st) {
+    const VocabDev &v = c->vocab->dev;
+    const long long n_chunks = ((long long)v.W * 32 + BUILD_CHUNK - 1) / BUILD_CHUNK;
+    long long items = (long long)max_entries * n_chunks;
+    long long grid = (long long)sm_count() * 8;  // 8 resident blocks of 256 threads per SM
+    if (items < grid) grid = items;
+    if (grid < 1) grid = 1;
+    build_masks_kernel<<<(unsigned)grid, BUILD_THREADS, 0, st>>>(v, c->dev, work);
+    WG_LAUNCHED();
+    return WG_OK;
+}
+
+bool rows_aligned(const void *p, int64_t stride_elems, size_t elem) {
+    return ((uintptr_t)p % 16 == 0) && ((stride_elems * (int64_t)elem) % 16 == 0);
+}
+
+template <typename E, bool ARGMAX, bool GATHER>
+int32_t launch_apply_t(const ApplyArgs &a_in, const CtxDev &ctx, unsigned long long *argkey,
+                       cudaStream_t st) {
+    ApplyArgs a = a_in;
+    const int n_spans = (a.W + 31) / 32;
+    // enough blocks to fill the machine a few times over, at least 8 spans (16 KB bf16) each
+    int blocks_per_row = (sm_count() * 16 + a.B - 1) / a.B;
+    if (blocks_per_row > (n_spans + 7) / 8) blocks_per_row = (n_spans + 7) / 8;
+    if (blocks_per_row < 1) blocks_per_row = 1;
+    a.spans_per_block = (n_spans + blocks_per_row - 1) / blocks_per_row;
+    blocks_per_row = (n_spans + a.spans_per_block - 1) / a.spans_per_block;
+    dim3 grid((unsigned)blocks_per_row, (unsigned)a.B);
+    if (rows_aligned(a.logits, a.row_stride, sizeof(E)))
+        apply_mask_kernel<E, ARGMAX, GATHER><<<grid, APPLY_THREADS, 0, st>>>(a, ctx, argkey);
+    else
+        apply_mask_unaligned_kernel<E, ARGMAX, GATHER><<<grid, APPLY_THREADS, 0, st>>>(a, ctx, argkey);
+    WG_LAUNCHED();
+    return WG_OK;
+}
+
+template <bool ARGMAX, bool GATHER>
+int32_t launch_apply(int32_t dtype, const ApplyArgs &a, const CtxDev &ctx,
+                     unsigned long long *argkey, cudaStream_t st) {
+    if (dtype == WG_DTYPE_BF16) return launch_apply_t<uint16_t, ARGMAX, GATHER>(a, ctx, argkey, st);
+    return launch_apply_t<uint32_t, ARGMAX, GATHER>(a, ctx, argkey, st);
+}
+
+bool batch_ok(const wg_ctx *c, int32_t B) { return c && B >= 1 && B <= c->max_batch; }
+
+}  // namespace
+
+extern "C" {
+
+// ---- decode path ----------------------------------------------------------------------
+
+int32_t wg_mask_cache_lookup(wg_ctx *c, const int32_t *gid, const int32_t *sid, int32_t B,
+                             int32_t *slot, void *stream) {
+    if (!batch_ok(c, B) || !gid || !sid || !slot) return WG_ERR_ARG;
+    cache_lookup_kernel<<<(B + 127) / 128, 128, 0, static_cast<cudaStream_t>(stream)>>>(
+        c->dev, gid, sid, B, slot);
+    WG_LAUNCHED();
+    return WG_OK;
+}
+
+int32_t wg_build_masks(wg_ctx *c, const int32_t *gid, const int32_t *sid, int32_t B,
+                       uint32_t *bitmask, int64_t row_stride_words, uint32_t flags, void *stream) {
+    if (!batch_ok(c, B) || !gid || !sid || !bitmask) return WG_ERR_ARG;
+    const int W = c->vocab->dev.W;
+    if (row_stride_words < W || (flags & ~(uint32_t)WG_NO_CACHE)) return WG_ERR_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (flags & WG_NO_CACHE) {
+        BuildWork work{gid, sid, nullptr, bitmask, row_stride_words, nullptr, B};
+        return launch_build(c, work, B, st);
+    }
+    cache_lookup_insert_kernel<<<1, 1024, 0, st>>>(c->dev, gid, sid, B, bitmask, row_stride_words);
+    WG_LAUNCHED();
+    BuildWork work{c->dev.bl_gid, c->dev.bl_sid, c->dev.bl_dst, nullptr, 0, c->dev.bl_count, 0};
+    int32_t rc = launch_build(c, work, B, st);
+    if (rc != WG_OK) return rc;
+    dim3 grid((unsigned)((W + 1023) / 1024), (unsigned)B);
+    cache_gather_kernel<<<grid, 256, 0, st>>>(c->dev, W, bitmask, row_stride_words);
+    WG_LAUNCHED();
+    return WG_OK;
+}
+
+size_t wg_apply_workspace_bytes(int32_t B) { return B > 0 ? sizeof(unsigned long long) * (size_t)B : 0; }
+
+int32_t wg_apply_mask(void *logits, int32_t dtype, int64_t row_stride_elems,
+                      const uint32_t *bitmask, int64_t mask_stride_words, int32_t B, int32_t V,
+                      int32_t *argmax_out, void *workspace, void *stream) {
+    if (!logits || !bitmask || B < 1 || V < 1) return WG_ERR_ARG;
+    if (dtype != WG_DTYPE_BF16 && dtype != WG_DTYPE_FP32) return WG_ERR_ARG;
+    const int W = (V + 31) / 32;
+    if (row_stride_elems < V || mask_stride_words < W) return WG_ERR_ARG;
+    if (argmax_out && (!workspace || (uintptr_t)workspace % 8 != 0)) return WG_ERR_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    ApplyArgs a{logits, row_stride_elems, bitmask, nullptr, mask_stride_words, B, V, W, 0};
+    CtxDev none{};
+    if (!argmax_out) return launch_apply<false, false>(dtype, a, none, nullptr, st);
+    unsigned long long *keys = static_cast<unsigned long long *>(workspace);
+    WG_CUDA(cudaMemsetAsync(keys, 0, sizeof(unsigned long long) * (size_t)B, st));
+    int32_t rc = launch_apply<true, false>(dtype, a, none, keys, st);
+    if (rc != WG_OK) return rc;
+    argmax_finish_kernel<<<(B + 127) / 128, 128, 0, st>>>(keys, B, argmax_out);
+    WG_LAUNCHED();
+    return WG_OK;
+}
+
+int32_t wg_advance(wg_ctx *c, const int32_t *gid, int32_t *sid, const int32_t *token, int32_t B,
+                   int32_t *status, uint32_t flags, void *stream) {
+    if (!batch_ok(c, B) || !gid || !sid || !token) return WG_ERR_ARG;
+    if (flags & ~(uint32_t)WG_RESTART_ON_DONE) return WG_ERR_ARG;
+    advance_kernel<<<(B + 127) / 128, 128, 0, static_cast<cudaStream_t>(stream)>>>(
+        c->vocab->dev, c->dev, gid, sid, token, nullptr, B, status, flags, 0);
+    WG_LAUNCHED();
+    return WG_OK;
+}
+
+int32_t wg_decode_step(wg_ctx *c, const int32_t *gid, int32_t *sid, int32_t B, void *logits,
+                       int32_t dtype, int64_t row_stride_elems, uint32_t *bitmask,
+                       int64_t mask_stride_words, int32_t *token_out, int32_t *status,
+                       uint32_t flags, void *stream) {
+    if (!batch_ok(c, B) || !gid || !sid || !logits || !bitmask || !token_out) return WG_ERR_ARG;
+    if (dtype != WG_DTYPE_BF16 && dtype != WG_DTYPE_FP32) return WG_ERR_ARG;
+    if (flags & ~(uint32_t)(WG_NO_CACHE | WG_RESTART_ON_DONE)) return WG_ERR_ARG;
+    const VocabDev &v = c->vocab->dev;
+    if (row_stride_elems < v.V || mask_stride_words < v.W) return WG_ERR_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    ApplyArgs a{logits, row_stride_elems, bitmask, bitmask, mask_stride_words, B, v.V, v.W, 0};
+    int32_t rc;
+    if (flags & WG_NO_CACHE) {
+        reset_rows_kernel<<<(B + 255) / 256, 256, 0, st>>>(c->dev, B);
+        WG_LAUNCHED();
+        BuildWork work{gid, sid, nullptr, bitmask, mask_stride_words, nullptr, B};
+        if ((rc = timing_mark(c, 0, st)) != WG_OK) return rc;
+        rc = launch_build(c, work, B, st);
+        if (rc != WG_OK) return rc;
+        if ((rc = timing_mark(c, 1, st)) != WG_OK) return rc;
+        if ((rc = timing_mark(c, 2, st)) != WG_OK) return rc;
+        rc = launch_apply<true, false>(dtype, a, c->dev, c->dev.argkey, st);
+    } else {
+        cache_lookup_insert_kernel<<<1, 1024, 0, st>>>(c->dev, gid, sid, B, bitmask, mask_stride_words);
+        WG_LAUNCHED();
+        BuildWork work{c->dev.bl_gid, c->dev.bl_sid, c->dev.bl_dst, nullptr, 0, c->dev.bl_count, 0};
+        if ((rc = timing_mark(c, 0, st)) != WG_OK) return rc;
+        rc = launch_build(c, work, B, st);
+        if (rc != WG_OK) return rc;
+        if ((rc = timing_mark(c, 1, st)) != WG_OK) return rc;
+        if ((rc = timing_mark(c, 2, st)) != WG_OK) return rc;
+        rc = launch_apply<true, true>(dtype, a, c->dev, c->dev.argkey, st);
+    }
+    if (rc != WG_OK) return rc;
+    if ((rc = timing_mark(c, 3, st)) != WG_OK) return rc;
+    advance_kernel<<<(B + 127) / 128, 128, 0, st>>>(v, c->dev, gid, sid, nullptr, token_out, B,
+                                                    status, flags & WG_RESTART_ON_DONE, 1);
+    WG_LAUNCHED();
+    return WG_OK;
+}
+
+int32_t wg_decode_step_host(wg_ctx *c, const int32_t *gid, int32_t *sid, int32_t B,
+                            const void *logits_host, void *logits_dev, int32_t dtype,
+                            int64_t row_stride_elems, uint32_t *bitmask,
+                            int64_t mask_stride_words, int32_t *token_dev, int32_t *token_host,
+                            int32_t *status, uint32_t flags, void *stream) {
+    if (!c || !logits_host || !logits_dev || !token_dev || !token_host) return WG_ERR_ARG;
+    if (dtype != WG_DTYPE_BF16 && dtype != WG_DTYPE_FP32) return WG_ERR_ARG;
+    if (!batch_ok(c, B) || row_stride_elems < c->vocab->dev.V) return WG_ERR_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t e = dtype == WG_DTYPE_BF16 ? 2 : 4;
+    const size_t row_bytes = (size_t)c->vocab->dev.V * e;
+    WG_CUDA(cudaMemcpy2DAsync(logits_dev, (size_t)row_stride_elems * e, logits_host, row_bytes,
+                              row_bytes, (size_t)B, cudaMemcpyHostToDevice, st));
+    int32_t rc = wg_decode_step(c, gid, sid, B, logits_dev, dtype, row_stride_elems, bitmask,
+                                mask_stride_words, token_dev, status, flags, stream);
+    if (rc != WG_OK) return rc;
+    WG_CUDA(cudaMemcpyAsync(token_host, token_dev, sizeof(int32_t) * (size_t)B,
+                            cudaMemcpyDeviceToHost, st));
+    WG_CUDA(cudaStreamSynchronize(st));
+    return WG_OK;
+}
+
+int32_t wg_ctx_set_timing(wg_ctx *c, int32_t enable) {
+    if (!c) return WG_ERR_ARG;
+    c->timing = enable != 0;
+    c->timed_steps = 0;
+    return WG_OK;
+}
+
+int32_t wg_ctx_get_timing(wg_ctx *c, double *build_ms, double *apply_ms, int64_t *steps) {
+    if (!c) return WG_ERR_ARG;
+    double b = 0.0, a = 0.0;
+    for (size_t i = 0; i < c->timed_steps; ++i) {
+        float ms = 0.f;
+        WG_CUDA(cudaEventSynchronize(c->events[4 * i + 3]));
+        WG_CUDA(cudaEventElapsedTime(&ms, c->events[4 * i], c->events[4 * i + 1]));
+        b += ms;
+        WG_CUDA(cudaEventElapsedTime(&ms, c->events[4 * i + 2], c->events[4 * i + 3]));
+        a += ms;
+    }
+    if (build_ms) *build_ms = b;
+    if (apply_ms) *apply_ms = a;
+    if (steps) *steps = (int64_t)c->timed_steps;
+    c->timed_steps = 0;
+    return WG_OK;
+}
+
+int32_t wg_cache_prewarm(wg_ctx *c, int32_t grammar_id, void *stream) {
+    if (!c || grammar_id < 0 || grammar_id >= (int32_t)c->slots.size()) return WG_ERR_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int32_t S = c->slots[grammar_id].n_states;
+    wg_stats before{}, after{};
+    int32_t rc = wg_get_stats(c, &before, stream);
+    if (rc != WG_OK) return rc;
+    for (int32_t first = 1; first < S; first += c->max_batch) {
+        const int32_t n = (S - first < c->max_batch) ? S - first : c->max_batch;
+        iota_states_kernel<<<(n + 255) / 256, 256, 0, st>>>(c->d_stage_gid, c->d_stage_sid,
+                                                            grammar_id, first, n);
+        WG_LAUNCHED();
+        cache_lookup_insert_kernel<<<1, 1024, 0, st>>>(c->dev, c->d_stage_gid, c->d_stage_sid, n,
+                                                       nullptr, 0);
+        WG_LAUNCHED();
+        BuildWork work{c->dev.bl_gid, c->dev.bl_sid, c->dev.bl_dst, nullptr, 0, c->dev.bl_count, 0};
+        rc = launch_build(c, work, n, st);
+        if (rc != WG_OK) return rc;
+    }
+    rc = wg_get_stats(c, &after, stream);
+    if (rc != WG_OK) return rc;
+    return after.rows_uncached > before.rows_uncached ? WG_ERR_CAPACITY : WG_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,32 @@
+// Internal declarations shared by the library's translation units (not part of the ABI).
+#pragma once
+
+#include <cstdint>
+#include <vector>
+
+#include "wg.h"
+
+constexpr int WG_N_SYMBOLS = 257;
+constexpr int WG_SYM_EOS = 256;
+constexpr int WG_SET_WORDS = 9;
+constexpr int WG_REC_BYTES = 16;  // token bytes held in the fixed-size record
+
+// A compiled grammar on the host: a dense table over byte classes.
+// table[s * n_classes + c] is the state after any symbol of class c in state s; state 0 is
+// DEAD (all of its entries are 0).  byte_class maps the 256 byte values, eos_class the EOS
+// symbol.  Classes group symbols whose columns are equal in every state.
+struct wg_grammar {
+    int32_t n_states = 0;
+    int32_t n_classes = 0;
+    int32_t start = 0;
+    int32_t done = 0;
+    int32_t eos_class = 0;
+    uint8_t byte_class[256] = {};
+    std::vector<int32_t> table;
+    uint64_t hash = 0;
+};
+
+// Lowering entry (wg_lower.cpp).
+int32_t wg_lower_tree(const wg_op_node *nodes, int32_t n_nodes, const int32_t *children,
+                      int32_t n_children, const uint32_t *sets, int32_t n_sets,
+                      const uint8_t *data, int32_t n_data, int32_t root, wg_grammar *out);

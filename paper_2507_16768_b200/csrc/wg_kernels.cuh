@@ -1,0 +1,513 @@
+// Device code of the mask path: build, cache, gather, apply (+ argmax), advance.
+// sm_100a; plain integer and load/store work -- nothing here is a dense contraction, so no
+// tensor-core instruction appears.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cstdint>
+
+#include "wg_internal.h"
+
+// ---------------------------------------------------------------------------------------
+// device-side views
+// ---------------------------------------------------------------------------------------
+struct GrammarDev {
+    const void *table;          // [n_states][n_classes] of uint16_t (wide == 0) or uint32_t
+    const uint8_t *byte_class;  // [256]
+    int32_t n_states, n_classes, start, done, eos_class, wide;
+};
+
+struct VocabDev {
+    const uint4 *rec;         // [V] first 16 bytes of every token, zero padded
+    const uint8_t *len;       // [V] min(length, 255)
+    const uint32_t *offsets;  // [V + 1] CSR, for tokens longer than the record
+    const uint8_t *bytes;
+    int32_t V, W, eos_id;
+};
+
+enum StatSlot {
+    ST_HITS = 0, ST_MISSES, ST_BUILT, ST_UNCACHED, ST_REJECTED, ST_EMPTY, ST_BAD_STATE, ST_COUNT
+};
+
+struct CtxDev {
+    const GrammarDev *grammars;
+    int32_t n_grammars;
+    // mask cache
+    unsigned long long *keys;  // [hash_size], 0 = empty, else ((gid + 1) << 32) | sid
+    int32_t *vals;             // [hash_size] pool row, or -1 for a key that found the pool full
+    uint32_t *pool;            // [capacity][pool_stride]
+    int32_t hash_size;         // power of two (0 when capacity == 0)
+    int32_t capacity;
+    int64_t pool_stride;       // words
+    int32_t *n_slots;          // pool rows handed out so far
+    // per-call scratch
+    int32_t *ent;              // [max_batch] hash entry of each row
+    int32_t *slot;             // [max_batch] resolved pool row of each row, or -1
+    int32_t *bl_gid, *bl_sid;  // [max_batch] build list
+    uint32_t **bl_dst;         // [max_batch] where each listed mask goes
+    int32_t *bl_count;
+    unsigned long long *argkey;  // [max_batch] packed (value key, ~id) maxima
+    unsigned long long *stats;   // [ST_COUNT]
+};
+
+constexpr uint32_t NEG_INF_F32 = 0xFF800000u;
+constexpr uint32_t NEG_INF_BF16X2 = 0xFF80FF80u;
+
+// ---------------------------------------------------------------------------------------
+// table walk
+// ---------------------------------------------------------------------------------------
+template <typename T>
+__device__ __forceinline__ uint32_t walk_record(const T *__restrict__ tab, int C,
+                                                const uint8_t *cls, uint32_t s, uint4 rec, int n) {
+    const uint32_t w[4] = {rec.x, rec.y, rec.z, rec.w};
+#pragma unroll
+    for (int j = 0; j < WG_REC_BYTES; ++j) {
+        if (j >= n || s == 0) break;
+        const uint32_t b = (w[j >> 2] >> (8 * (j & 3))) & 0xFFu;
+        s = tab[(size_t)s * C + cls[b]];
+    }
+    return s;
+}
+
+// State after token t from state s (0 = DEAD).  cls: the grammar's byte classes (shared or
+// global memory).  Tokens longer than the record continue from the CSR bytes.
+template <typename T>
+__device__ __forceinline__ uint32_t walk_token(const VocabDev &v, const T *__restrict__ tab,
+                                               int C, int eos_class, const uint8_t *cls,
+                                               uint32_t s, int t) {
+    if (t == v.eos_id) return tab[(size_t)s * C + eos_class];
+    const int n = v.len[t];
+    if (n == 0) return 0;
+    s = walk_record(tab, C, cls, s, __ldg(&v.rec[t]), n);
+    if (n > WG_REC_BYTES && s != 0) {
+        const uint32_t b = v.offsets[t] + WG_REC_BYTES, e = v.offsets[t + 1];
+        for (uint32_t i = b; i < e && s != 0; ++i) s = tab[(size_t)s * C + cls[v.bytes[i]]];
+    }
+    return s;
+}
+
+// ---------------------------------------------------------------------------------------
+// K1: mask build.  One thread per token, 32 consecutive tokens per warp, one ballot per word.
+// Work item = (mask m, chunk of BUILD_CHUNK tokens); a fixed-size grid strides over the items
+// so that a launch with nothing to build costs a few empty blocks.
+// ---------------------------------------------------------------------------------------
+constexpr int BUILD_THREADS = 256;
+constexpr int BUILD_CHUNK = 2048;
+
+struct BuildWork {
+    const int32_t *gid, *sid;   // per entry
+    uint32_t *const *dst_list;  // per entry destination, or NULL: use dst_base + m * dst_stride
+    uint32_t *dst_base;
+    int64_t dst_stride;
+    const int32_t *count_ptr;   // number of entries on the device, or NULL: use count
+    int32_t count;
+};
+
+template <typename T>
+__device__ __forceinline__ void build_chunk(const VocabDev &v, const GrammarDev &g,
+                                            const uint8_t *cls, uint32_t s0, int t_begin,
+                                            uint32_t *__restrict__ dst) {
+    const T *tab = static_cast<const T *>(g.table);
+    const int C = g.n_classes;
+    const int t_end = min(t_begin + BUILD_CHUNK, v.W * 32);
+    for (int t = t_begin + (int)threadIdx.x; t < t_end; t += BUILD_THREADS) {
+        bool alive = false;
+        if (t < v.V && s0 != 0) alive = walk_token<T>(v, tab, C, g.eos_class, cls, s0, t) != 0;
+        const uint32_t word = __ballot_sync(0xFFFFFFFFu, alive);
+        if ((threadIdx.x & 31) == 0) dst[t >> 5] = word;
+    }
+}
+
+__global__ void __launch_bounds__(BUILD_THREADS)
+build_masks_kernel(VocabDev v, CtxDev ctx, BuildWork work) {
+    __shared__ uint8_t cls[256];
+    __shared__ int cls_gid;
+    if (threadIdx.x == 0) cls_gid = -1;
+    __syncthreads();
+    const int n_entries = work.count_ptr ? *work.count_ptr : work.count;
+    const int n_chunks = (v.W * 32 + BUILD_CHUNK - 1) / BUILD_CHUNK;
+    const long long n_items = (long long)n_entries * n_chunks;
+    for (long long item = blockIdx.x; item < n_items; item += gridDim.x) {
+        const int m = (int)(item / n_chunks);
+        const int chunk = (int)(item % n_chunks);
+        const int gid = work.gid[m];
+        uint32_t s0 = (uint32_t)work.sid[m];
+        uint32_t *dst = work.dst_list ? work.dst_list[m] : work.dst_base + (int64_t)m * work.dst_stride;
+        const bool known = gid >= 0 && gid < ctx.n_grammars;
+        GrammarDev g = {};
+        if (known) g = ctx.grammars[gid];
+        if (!known || s0 >= (uint32_t)g.n_states) s0 = 0;  // unknown state: an all-zero row
+        if (known && cls_gid != gid) {
+            __syncthreads();
+            cls[threadIdx.x] = g.byte_class[threadIdx.x];
+            if (threadIdx.x == 0) cls_gid = gid;
+            __syncthreads();
+        }
+        if (chunk == 0 && threadIdx.x == 0) {
+            atomicAdd(&ctx.stats[ST_BUILT], 1ull);
+            if (s0 == 0 && work.sid[m] != 0) atomicAdd(&ctx.stats[ST_BAD_STATE], 1ull);
+        }
+        if (g.wide) build_chunk<uint32_t>(v, g, cls, s0, chunk * BUILD_CHUNK, dst);
+        else build_chunk<uint16_t>(v, g, cls, s0, chunk * BUILD_CHUNK, dst);
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// K2: mask cache.  Open addressing with linear probing over 64-bit keys.
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ unsigned long long cache_key(int gid, int sid) {
+    return ((unsigned long long)(uint32_t)(gid + 1) << 32) | (uint32_t)sid;
+}
+
+__device__ __forceinline__ uint32_t cache_hash(unsigned long long k) {
+    k ^= k >> 33; k *= 0xFF51AFD7ED558CCDull; k ^= k >> 33; k *= 0xC4CEB9FE1A85EC53ull; k ^= k >> 33;
+    return (uint32_t)k;
+}
+
+constexpr int32_t ENT_NEW = 0x40000000;  // marks the row that inserted its key in this call
+
+// Read-only probe: slot[r] = pool row or -1.
+__global__ void cache_lookup_kernel(CtxDev ctx, const int32_t *gid, const int32_t *sid, int B,
+                                    int32_t *slot) {
+    const int r = blockIdx.x * blockDim.x + threadIdx.x;
+    if (r >= B) return;
+    int32_t found = -1;
+    if (ctx.hash_size > 0) {
+        const unsigned long long key = cache_key(gid[r], sid[r]);
+        const uint32_t mask = (uint32_t)ctx.hash_size - 1;
+        uint32_t h = cache_hash(key) & mask;
+        for (int probe = 0; probe < ctx.hash_size; ++probe, h = (h + 1) & mask) {
+            const unsigned long long k = ctx.keys[h];
+            if (k == key) { found = ctx.vals[h]; break; }
+            if (k == 0) break;
+        }
+    }
+    slot[r] = found;
+}
+
+// Lookup-or-insert for one batch, run by ONE block so that a block barrier separates "every
+// key of the batch is in the table and owns a pool row" from "read the rows back".  Rows whose
+// state is new append one build-list entry per distinct state; when the pool or the table is
+// full the row is listed for an uncached build straight into its bitmask row.
+// bitmask may be NULL (prewarm): uncached rows are then dropped.
+__global__ void __launch_bounds__(1024)
+cache_lookup_insert_kernel(CtxDev ctx, const int32_t *gid, const int32_t *sid, int B,
+                           uint32_t *bitmask, int64_t mask_stride) {
+    if (threadIdx.x == 0) *ctx.bl_count = 0;
+    __syncthreads();
+    const uint32_t mask = (uint32_t)ctx.hash_size - 1;
+    for (int r = threadIdx.x; r < B; r += blockDim.x) {
+        ctx.argkey[r] = 0ull;
+        const int g = gid[r], s = sid[r];
+        int32_t entry = -1;
+        bool inserted = false;
+        if (ctx.hash_size > 0 && g >= 0 && g < ctx.n_grammars) {
+            const unsigned long long key = cache_key(g, s);
+            uint32_t h = cache_hash(key) & mask;
+            for (int probe = 0; probe < ctx.hash_size; ++probe, h = (h + 1) & mask) {
+                unsigned long long k = ctx.keys[h];
+                if (k == 0) {
+                    k = atomicCAS(&ctx.keys[h], 0ull, key);
+                    if (k == 0) {  // this thread owns the new entry
+                        const int32_t row = atomicAdd(ctx.n_slots, 1);
+                        if (row < ctx.capacity) {
+                            ctx.vals[h] = row;
+                            const int i = atomicAdd(ctx.bl_count, 1);
+                            ctx.bl_gid[i] = g;
+                            ctx.bl_sid[i] = s;
+                            ctx.bl_dst[i] = ctx.pool + (int64_t)row * ctx.pool_stride;
+                        } else {
+                            atomicSub(ctx.n_slots, 1);
+                            ctx.vals[h] = -1;
+                        }
+                        entry = (int32_t)h;
+                        inserted = true;
+                        break;
+                    }
+                }
+                if (k == key) { entry = (int32_t)h; break; }
+            }
+        }
+        ctx.ent[r] = (entry >= 0 && inserted) ? (entry | ENT_NEW) : entry;
+    }
+    __syncthreads();
+    for (int r = threadIdx.x; r < B; r += blockDim.x) {
+        const int32_t e = ctx.ent[r];
+        const int32_t row = e >= 0 ? ctx.vals[e & ~ENT_NEW] : -1;
+        ctx.slot[r] = row;
+        // a hit is a row served from a pool row that some earlier row or call already owned
+        atomicAdd(&ctx.stats[(row >= 0 && !(e & ENT_NEW)) ? ST_HITS : ST_MISSES], 1ull);
+        if (row < 0) {
+            atomicAdd(&ctx.stats[ST_UNCACHED], 1ull);
+            if (bitmask) {
+                const int i = atomicAdd(ctx.bl_count, 1);
+                ctx.bl_gid[i] = gid[r];
+                ctx.bl_sid[i] = sid[r];
+                ctx.bl_dst[i] = bitmask + (int64_t)r * mask_stride;
+            }
+        }
+    }
+}
+
+// Rows of a WG_NO_CACHE step: no pool row, and the packed maxima start at zero.
+__global__ void reset_rows_kernel(CtxDev ctx, int B) {
+    const int r = blockIdx.x * blockDim.x + threadIdx.x;
+    if (r < B) { ctx.slot[r] = -1; ctx.argkey[r] = 0ull; }
+}
+
+__global__ void cache_clear_kernel(CtxDev ctx) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < ctx.hash_size) { ctx.keys[i] = 0ull; ctx.vals[i] = -1; }
+    if (i == 0) *ctx.n_slots = 0;
+}
+
+__global__ void iota_states_kernel(int32_t *gid, int32_t *sid, int g, int first, int n) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) { gid[i] = g; sid[i] = first + i; }
+}
+
+// K3: copy cached rows out.  grid = (chunks, B).
+__global__ void cache_gather_kernel(CtxDev ctx, int W, uint32_t *bitmask, int64_t mask_stride) {
+    const int r = blockIdx.y;
+    const int32_t row = ctx.slot[r];
+    if (row < 0) return;  // built straight into the bitmask
+    const uint32_t *src = ctx.pool + (int64_t)row * ctx.pool_stride;
+    uint32_t *dst = bitmask + (int64_t)r * mask_stride;
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < W; i += gridDim.x * blockDim.x)
+        dst[i] = src[i];
+}
+
+// ---------------------------------------------------------------------------------------
+// K4 / K5: apply (+ greedy argmax).
+//
+// Fast kernel: a warp covers 2 KB of one logits row per pass with four 512-byte fully
+// coalesced 16-byte-per-lane accesses; lane l first loads mask word l of the span (one
+// coalesced 128-byte load), and each lane then fetches "its" word for every access by
+// shuffle.  Per 16-byte chunk: all bits clear -> store -inf without loading; all bits set ->
+// touch nothing (load only for the argmax); mixed -> load, patch, store.
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t order_key(uint32_t f32_bits) {
+    if (f32_bits == 0x80000000u) f32_bits = 0;  // -0.0 ties with +0.0
+    return (f32_bits & 0x80000000u) ? ~f32_bits : (f32_bits | 0x80000000u);
+}
+
+__device__ __forceinline__ unsigned long long pack_best(uint32_t key, int idx) {
+    return ((unsigned long long)key << 32) | (uint32_t)(0xFFFFFFFFu - (uint32_t)idx);
+}
+
+__device__ __forceinline__ int unpack_best(unsigned long long k) {
+    return k == 0ull ? -1 : (int)(0xFFFFFFFFu - (uint32_t)(k & 0xFFFFFFFFull));
+}
+
+template <typename E> struct ElemTraits;
+template <> struct ElemTraits<uint16_t> {  // bf16
+    static constexpr int PER_CHUNK = 8;    // elements per 16-byte chunk
+    static __device__ __forceinline__ uint32_t f32_bits(uint16_t e) { return (uint32_t)e << 16; }
+    static constexpr uint32_t NEG_INF = 0xFF80u;
+};
+template <> struct ElemTraits<uint32_t> {  // fp32
+    static constexpr int PER_CHUNK = 4;
+    static __device__ __forceinline__ uint32_t f32_bits(uint32_t e) { return e; }
+    static constexpr uint32_t NEG_INF = 0xFF800000u;
+};
+
+constexpr int APPLY_THREADS = 256;
+constexpr int APPLY_WARPS = APPLY_THREADS / 32;
+
+struct ApplyArgs {
+    void *logits;
+    int64_t row_stride;       // elements
+    const uint32_t *bitmask;  // row source when the row has no pool slot
+    uint32_t *bitmask_out;    // GATHER: where pool rows are copied to (same array as bitmask)
+    int64_t mask_stride;      // words
+    int32_t B, V, W;
+    int32_t spans_per_block;  // spans (32 mask words) each block handles
+};
+
+// element-wise masking of [begin, end) of one row; any alignment
+template <typename E, bool ARGMAX>
+__device__ __forceinline__ void apply_scalar(E *row, const uint32_t *mrow, int begin, int end,
+                                             unsigned long long &best) {
+    for (int t = begin + (int)threadIdx.x; t < end; t += APPLY_THREADS) {
+        const bool keep = (mrow[t >> 5] >> (t & 31)) & 1u;
+        if (!keep) {
+            row[t] = (E)ElemTraits<E>::NEG_INF;
+        } else if (ARGMAX) {
+            const unsigned long long k = pack_best(order_key(ElemTraits<E>::f32_bits(row[t])), t);
+            best = k > best ? k : best;
+        }
+    }
+}
+
+template <bool ARGMAX>
+__device__ __forceinline__ void block_argmax_commit(unsigned long long best,
+                                                    unsigned long long *dst) {
+    if constexpr (ARGMAX) {
+        __shared__ unsigned long long warp_best[APPLY_WARPS];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const unsigned long long other = __shfl_xor_sync(0xFFFFFFFFu, best, o);
+            best = other > best ? other : best;
+        }
+        if ((threadIdx.x & 31) == 0) warp_best[threadIdx.x >> 5] = best;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            for (int w = 1; w < APPLY_WARPS; ++w) best = warp_best[w] > best ? warp_best[w] : best;
+            if (best != 0ull) atomicMax(dst, best);
+        }
+    }
+}
+
+// grid = (blocks per row, B).  Requires 16-byte aligned rows (pointer and stride).
+template <typename E, bool ARGMAX, bool GATHER>
+__global__ void __launch_bounds__(APPLY_THREADS)
+apply_mask_kernel(ApplyArgs a, CtxDev ctx, unsigned long long *argkey) {
+    constexpr int EPC = ElemTraits<E>::PER_CHUNK;  // elements per chunk: bits per lane
+    constexpr int CHUNKS_PER_WORD = 32 / EPC;      // 4 (bf16) or 8 (fp32)
+    constexpr int PASSES = 32 * CHUNKS_PER_WORD / 32;  // 16-byte accesses per lane and span
+    constexpr uint32_t FULL = (1u << EPC) - 1;
+    const int r = blockIdx.y;
+    E *row = static_cast<E *>(a.logits) + (int64_t)r * a.row_stride;
+    const uint32_t *mrow = a.bitmask + (int64_t)r * a.mask_stride;
+    if (GATHER) {
+        const int32_t slot = ctx.slot[r];
+        if (slot >= 0) mrow = ctx.pool + (int64_t)slot * ctx.pool_stride;
+    }
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int n_spans = (a.W + 31) / 32;
+    const int span_begin = blockIdx.x * a.spans_per_block;
+    const int span_end = min(span_begin + a.spans_per_block, n_spans);
+    const int full_chunks = a.V / EPC;  // chunks that lie wholly inside the row
+    unsigned long long best = 0ull;
+
+    for (int span = span_begin + warp; span < span_end; span += APPLY_WARPS) {
+        const int word0 = span * 32;
+        uint32_t my_word = 0;
+        if (word0 + lane < a.W) {
+            my_word = mrow[word0 + lane];
+            if (GATHER && mrow != a.bitmask + (int64_t)r * a.mask_stride)
+                a.bitmask_out[(int64_t)r * a.mask_stride + word0 + lane] = my_word;
+        }
+#pragma unroll
+        for (int p = 0; p < PASSES; ++p) {
+            const int c_in_span = p * 32 + lane;  // chunk index inside the span
+            const uint32_t word = __shfl_sync(0xFFFFFFFFu, my_word, c_in_span / CHUNKS_PER_WORD);
+            const uint32_t bits = (word >> (EPC * (c_in_span % CHUNKS_PER_WORD))) & FULL;
+            const int chunk = word0 * CHUNKS_PER_WORD + c_in_span;
+            if (chunk >= full_chunks) continue;
+            uint4 *ptr = reinterpret_cast<uint4 *>(row) + chunk;
+            if (bits == 0) {
+                const uint32_t ninf = sizeof(E) == 2 ? NEG_INF_BF16X2 : NEG_INF_F32;
+                *ptr = make_uint4(ninf, ninf, ninf, ninf);
+            } else if (ARGMAX || bits != FULL) {
+                uint4 v = *ptr;
+                uint32_t w[4] = {v.x, v.y, v.z, v.w};
+                const int t0 = chunk * EPC;
+                if (sizeof(E) == 2) {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const uint32_t e = (w[i >> 1] >> (16 * (i & 1))) & 0xFFFFu;
+                        if ((bits >> i) & 1u) {
+                            if (ARGMAX) {
+                                const unsigned long long k = pack_best(order_key(e << 16), t0 + i);
+                                best = k > best ? k : best;
+                            }
+                        } else {
+                            w[i >> 1] = (i & 1) ? ((w[i >> 1] & 0x0000FFFFu) | 0xFF800000u)
+                                                : ((w[i >> 1] & 0xFFFF0000u) | 0x0000FF80u);
+                        }
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        if ((bits >> i) & 1u) {
+                            if (ARGMAX) {
+                                const unsigned long long k = pack_best(order_key(w[i]), t0 + i);
+                                best = k > best ? k : best;
+                            }
+                        } else {
+                            w[i] = NEG_INF_F32;
+                        }
+                    }
+                }
+                if (bits != FULL) *ptr = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+        }
+    }
+    // elements after the last whole chunk (V not a multiple of the chunk size)
+    if (blockIdx.x == gridDim.x - 1 && full_chunks * EPC < a.V)
+        apply_scalar<E, ARGMAX>(row, mrow, full_chunks * EPC, a.V, best);
+    block_argmax_commit<ARGMAX>(best, argkey + r);
+}
+
+// Any alignment: one block column per row, element-wise.
+template <typename E, bool ARGMAX, bool GATHER>
+__global__ void __launch_bounds__(APPLY_THREADS)
+apply_mask_unaligned_kernel(ApplyArgs a, CtxDev ctx, unsigned long long *argkey) {
+    const int r = blockIdx.y;
+    E *row = static_cast<E *>(a.logits) + (int64_t)r * a.row_stride;
+    const uint32_t *own = a.bitmask + (int64_t)r * a.mask_stride;
+    const uint32_t *mrow = own;
+    if (GATHER) {
+        const int32_t slot = ctx.slot[r];
+        if (slot >= 0) mrow = ctx.pool + (int64_t)slot * ctx.pool_stride;
+    }
+    const int per_block = ((a.V + gridDim.x - 1) / gridDim.x + 31) & ~31;
+    const int begin = blockIdx.x * per_block, end = min(begin + per_block, a.V);
+    if (GATHER && mrow != own)
+        for (int i = (begin >> 5) + (int)threadIdx.x; i < (end + 31) >> 5; i += APPLY_THREADS)
+            a.bitmask_out[(int64_t)r * a.mask_stride + i] = mrow[i];
+    unsigned long long best = 0ull;
+    if (begin < end) apply_scalar<E, ARGMAX>(row, mrow, begin, end, best);
+    block_argmax_commit<ARGMAX>(best, argkey + r);
+}
+
+__global__ void argmax_finish_kernel(const unsigned long long *argkey, int B, int32_t *out) {
+    const int r = blockIdx.x * blockDim.x + threadIdx.x;
+    if (r < B) out[r] = unpack_best(argkey[r]);
+}
+
+// ---------------------------------------------------------------------------------------
+// K6: advance.  One thread per row; at most a handful of dependent lookups.
+// from_keys: the token comes from the packed maxima of the fused step and is written out.
+// ---------------------------------------------------------------------------------------
+__global__ void advance_kernel(VocabDev v, CtxDev ctx, const int32_t *gid, int32_t *sid,
+                               const int32_t *token_in, int32_t *token_out, int B,
+                               int32_t *status, uint32_t flags, int from_keys) {
+    const int r = blockIdx.x * blockDim.x + threadIdx.x;
+    if (r >= B) return;
+    int t;
+    if (from_keys) {
+        t = unpack_best(ctx.argkey[r]);
+        token_out[r] = t;
+    } else {
+        t = token_in[r];
+    }
+    const int g = gid[r];
+    const uint32_t s = (uint32_t)sid[r];
+    int32_t st = WG_OK;
+    if (g < 0 || g >= ctx.n_grammars || s >= (uint32_t)ctx.grammars[g].n_states) {
+        st = WG_ERR_STATE;
+        atomicAdd(&ctx.stats[ST_BAD_STATE], 1ull);
+    } else if (from_keys && t < 0) {
+        st = WG_ERR_EMPTY_MASK;
+        atomicAdd(&ctx.stats[ST_EMPTY], 1ull);
+    } else {
+        const GrammarDev gr = ctx.grammars[g];
+        uint32_t next = 0;
+        if (t >= 0 && t < v.V && s != 0) {
+            next = gr.wide ? walk_token<uint32_t>(v, static_cast<const uint32_t *>(gr.table),
+                                                  gr.n_classes, gr.eos_class, gr.byte_class, s, t)
+                           : walk_token<uint16_t>(v, static_cast<const uint16_t *>(gr.table),
+                                                  gr.n_classes, gr.eos_class, gr.byte_class, s, t);
+        }
+        if (next == 0) {
+            st = WG_ERR_TOKEN_REJECTED;
+            atomicAdd(&ctx.stats[ST_REJECTED], 1ull);
+        } else {
+            if ((flags & WG_RESTART_ON_DONE) && next == (uint32_t)gr.done) next = (uint32_t)gr.start;
+            sid[r] = (int32_t)next;
+        }
+    }
+    if (status) status[r] = st;
+}

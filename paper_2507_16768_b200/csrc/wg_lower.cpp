@@ -1,0 +1,282 @@
+// Host-side lowering of an operator tree (paper Section 3.2: Sequence / Wait / Write /
+// IfElse / DoWhile) to a byte-level deterministic transition table.
+//
+// Construction: every operator is lowered against a CONTINUATION state k (where control
+// goes once the operator's language has been matched) and returns its ENTRY state.  A
+// Sequence folds its parts from the right; a Write is a chain of one-symbol states ending in
+// k; a Wait or Switch is one state whose deciding symbols lead to the entry of the chosen
+// body lowered against k and whose stay symbols loop; a DoWhile first allocates its
+// condition state c, lowers the body against c, and wires c's true symbols back to the
+// body's entry and its false symbols to k.  An absent body contributes nothing (its entry
+// is its continuation).  Because the deciding sets of one primitive are disjoint the result
+// is deterministic without a subset construction.  States are then renumbered breadth-first
+// from the start state and the 257 symbols are merged into classes with equal columns.
+#include <algorithm>
+#include <cstring>
+#include <queue>
+#include <unordered_map>
+
+#include "wg_internal.h"
+
+namespace {
+
+struct SymSet {
+    uint32_t w[WG_SET_WORDS];
+    bool has(int s) const { return (w[s >> 5] >> (s & 31)) & 1u; }
+    bool empty() const {
+        for (uint32_t x : w) if (x) return false;
+        return true;
+    }
+    bool meets(const SymSet &o) const {
+        for (int i = 0; i < WG_SET_WORDS; ++i) if (w[i] & o.w[i]) return true;
+        return false;
+    }
+};
+
+struct Edge {
+    SymSet on;
+    int32_t to;
+};
+
+struct Lowerer {
+    const wg_op_node *nodes;
+    int32_t n_nodes;
+    const int32_t *children;
+    const SymSet *sets;
+    const uint8_t *data;
+    std::vector<std::vector<Edge>> states;  // outgoing edges; symbols on no edge go to DEAD
+
+    int32_t new_state() {
+        states.emplace_back();
+        return (int32_t)states.size() - 1;
+    }
+
+    static SymSet single(int sym) {
+        SymSet s{};
+        s.w[sym >> 5] = 1u << (sym & 31);
+        return s;
+    }
+
+    // stay = (allow \ deny) \ (union of the deciding sets)
+    SymSet stay_set(const wg_op_node &n) const {
+        SymSet s = sets[n.set_off];
+        const SymSet &deny = sets[n.set_off + 1];
+        for (int i = 0; i < WG_SET_WORDS; ++i) s.w[i] &= ~deny.w[i];
+        for (int d = 2; d < n.n_set; ++d)
+            for (int i = 0; i < WG_SET_WORDS; ++i) s.w[i] &= ~sets[n.set_off + d].w[i];
+        return s;
+    }
+
+    int32_t lower(int32_t node, int32_t k) {
+        if (node < 0) return k;
+        const wg_op_node &n = nodes[node];
+        switch (n.kind) {
+        case WG_OP_SEQUENCE: {
+            int32_t next = k;
+            for (int j = n.n_child - 1; j >= 0; --j) next = lower(children[n.child_off + j], next);
+            return next;
+        }
+        case WG_OP_WRITE: {
+            int32_t next = k;
+            for (int j = n.data_len - 1; j >= 0; --j) {
+                int32_t s = new_state();
+                states[s].push_back({single(data[n.data_off + j]), next});
+                next = s;
+            }
+            return next;
+        }
+        case WG_OP_WAIT:
+        case WG_OP_SWITCH: {
+            int32_t s = new_state();
+            for (int c = 0; c < n.n_child; ++c) {
+                int32_t target = lower(children[n.child_off + c], k);
+                states[s].push_back({sets[n.set_off + 2 + c], target});
+            }
+            SymSet stay = stay_set(n);
+            if (!stay.empty()) states[s].push_back({stay, s});
+            return s;
+        }
+        default: {  // WG_OP_DOWHILE
+            int32_t c = new_state();
+            int32_t entry = lower(children[n.child_off], c);
+            states[c].push_back({sets[n.set_off + 2], entry});
+            states[c].push_back({sets[n.set_off + 3], k});
+            SymSet stay = stay_set(n);
+            if (!stay.empty()) states[c].push_back({stay, c});
+            return entry;
+        }
+        }
+    }
+};
+
+int32_t validate(const wg_op_node *nodes, int32_t n_nodes, const int32_t *children,
+                 int32_t n_children, const SymSet *sets, int32_t n_sets, int32_t n_data,
+                 int32_t root) {
+    std::vector<uint8_t> used(n_nodes, 0);
+    used[root] = 1;
+    for (int32_t i = 0; i < n_nodes; ++i) {
+        const wg_op_node &n = nodes[i];
+        if (n.n_child < 0 || n.child_off < 0 || (int64_t)n.child_off + n.n_child > n_children)
+            return WG_ERR_ARG;
+        if (n.n_set < 0 || n.set_off < 0 || (int64_t)n.set_off + n.n_set > n_sets) return WG_ERR_ARG;
+        if (n.data_len < 0 || n.data_off < 0 || (int64_t)n.data_off + n.data_len > n_data)
+            return WG_ERR_ARG;
+        bool shape_ok = false;
+        switch (n.kind) {
+        case WG_OP_SEQUENCE: shape_ok = n.n_set == 0; break;
+        case WG_OP_WRITE: shape_ok = n.n_child == 0 && n.n_set == 0; break;
+        case WG_OP_WAIT: shape_ok = n.n_child == 1 && n.n_set == 3; break;
+        case WG_OP_SWITCH: shape_ok = n.n_set >= 3 && n.n_child == n.n_set - 2; break;
+        case WG_OP_DOWHILE: shape_ok = n.n_child == 1 && n.n_set == 4; break;
+        default: break;
+        }
+        if (!shape_ok) return WG_ERR_ARG;
+        for (int j = 0; j < n.n_child; ++j) {
+            int32_t c = children[n.child_off + j];
+            if (c == -1) {
+                if (n.kind == WG_OP_SEQUENCE) return WG_ERR_ARG;
+                continue;
+            }
+            if (c < 0 || c >= n_nodes) return WG_ERR_ARG;
+            if (used[c]) return WG_ERR_GRAMMAR;  // a node reached twice: not a tree
+            used[c] = 1;
+        }
+        if (n.kind == WG_OP_WAIT || n.kind == WG_OP_SWITCH || n.kind == WG_OP_DOWHILE) {
+            const SymSet &deny = sets[n.set_off + 1];
+            for (int a = 2; a < n.n_set; ++a) {
+                const SymSet &sa = sets[n.set_off + a];
+                if (sa.empty() || sa.meets(deny)) return WG_ERR_GRAMMAR;
+                for (int b = a + 1; b < n.n_set; ++b)
+                    if (sa.meets(sets[n.set_off + b])) return WG_ERR_GRAMMAR;
+            }
+        }
+    }
+    for (int32_t i = 0; i < n_nodes; ++i)
+        if (!used[i]) return WG_ERR_GRAMMAR;  // a node that hangs nowhere
+    return WG_OK;
+}
+
+uint64_t fnv1a(uint64_t h, const void *p, size_t n) {
+    const uint8_t *b = (const uint8_t *)p;
+    for (size_t i = 0; i < n; ++i) h = (h ^ b[i]) * 0x100000001B3ull;
+    return h;
+}
+
+}  // namespace
+
+int32_t wg_lower_tree(const wg_op_node *nodes, int32_t n_nodes, const int32_t *children,
+                      int32_t n_children, const uint32_t *sets_raw, int32_t n_sets,
+                      const uint8_t *data, int32_t n_data, int32_t root, wg_grammar *out) {
+    if (!nodes || n_nodes <= 0 || root < 0 || root >= n_nodes || n_children < 0 || n_sets < 0 ||
+        n_data < 0 || (n_children > 0 && !children) || (n_sets > 0 && !sets_raw) ||
+        (n_data > 0 && !data))
+        return WG_ERR_ARG;
+    const SymSet *sets = reinterpret_cast<const SymSet *>(sets_raw);
+    int32_t rc = validate(nodes, n_nodes, children, n_children, sets, n_sets, n_data, root);
+    if (rc != WG_OK) return rc;
+
+    bool mentions_eos = false;
+    for (int32_t s = 0; s < n_sets; ++s) mentions_eos |= sets[s].has(WG_SYM_EOS);
+
+    Lowerer lw{nodes, n_nodes, children, sets, data, {}};
+    const int32_t dead = lw.new_state();  // 0: no edges
+    (void)dead;
+    const int32_t done = lw.new_state();
+    lw.states[done].push_back({Lowerer::single(WG_SYM_EOS), done});
+    int32_t k = done;
+    if (!mentions_eos) {  // the implicit trailing EOS
+        k = lw.new_state();
+        lw.states[k].push_back({Lowerer::single(WG_SYM_EOS), done});
+    }
+    const int32_t start = lw.lower(root, k);
+
+    // breadth-first renumbering from the start state; DEAD stays 0
+    const int32_t n_raw = (int32_t)lw.states.size();
+    std::vector<int32_t> new_id(n_raw, -1);
+    std::vector<int32_t> order;
+    order.reserve(n_raw);
+    new_id[0] = 0;
+    order.push_back(0);
+    std::queue<int32_t> q;
+    new_id[start] = 1;
+    order.push_back(start);
+    q.push(start);
+    while (!q.empty()) {
+        int32_t s = q.front();
+        q.pop();
+        for (const Edge &e : lw.states[s]) {
+            if (new_id[e.to] < 0) {
+                new_id[e.to] = (int32_t)order.size();
+                order.push_back(e.to);
+                q.push(e.to);
+            }
+        }
+    }
+    if (new_id[done] < 0) {  // cannot happen for a valid tree, but keep DONE addressable
+        new_id[done] = (int32_t)order.size();
+        order.push_back(done);
+    }
+    const int32_t S = (int32_t)order.size();
+
+    // symbol classes by partition refinement over the states' columns
+    std::vector<int32_t> cls(WG_N_SYMBOLS, 0);
+    int32_t n_cls = 1;
+    std::vector<int32_t> target(WG_N_SYMBOLS);
+    for (int32_t i = 0; i < S; ++i) {
+        const std::vector<Edge> &edges = lw.states[order[i]];
+        if (edges.empty()) continue;
+        for (int sym = 0; sym < WG_N_SYMBOLS; ++sym) {
+            int32_t t = 0;
+            for (const Edge &e : edges)
+                if (e.on.has(sym)) { t = new_id[e.to]; break; }
+            target[sym] = t;
+        }
+        std::unordered_map<uint64_t, int32_t> split;
+        std::vector<int32_t> next(WG_N_SYMBOLS);
+        int32_t n_next = 0;
+        for (int sym = 0; sym < WG_N_SYMBOLS; ++sym) {
+            uint64_t key = ((uint64_t)(uint32_t)cls[sym] << 32) | (uint32_t)target[sym];
+            auto it = split.find(key);
+            if (it == split.end()) it = split.emplace(key, n_next++).first;
+            next[sym] = it->second;
+        }
+        if (n_next != n_cls) { cls.swap(next); n_cls = n_next; }
+    }
+    // class ids in order of first appearance over the byte values, EOS last
+    {
+        std::vector<int32_t> remap(n_cls, -1);
+        int32_t n = 0;
+        for (int sym = 0; sym < WG_N_SYMBOLS; ++sym)
+            if (remap[cls[sym]] < 0) remap[cls[sym]] = n++;
+        for (int sym = 0; sym < WG_N_SYMBOLS; ++sym) cls[sym] = remap[cls[sym]];
+    }
+
+    out->n_states = S;
+    out->n_classes = n_cls;
+    out->start = 1;
+    out->done = new_id[done];
+    out->eos_class = cls[WG_SYM_EOS];
+    for (int b = 0; b < 256; ++b) out->byte_class[b] = (uint8_t)cls[b];
+    out->table.assign((size_t)S * n_cls, 0);
+    std::vector<int32_t> rep(n_cls, -1);  // one representative symbol per class
+    for (int sym = 0; sym < WG_N_SYMBOLS; ++sym)
+        if (rep[cls[sym]] < 0) rep[cls[sym]] = sym;
+    for (int32_t i = 0; i < S; ++i) {
+        const std::vector<Edge> &edges = lw.states[order[i]];
+        for (int32_t c = 0; c < n_cls; ++c) {
+            int32_t t = 0;
+            for (const Edge &e : edges)
+                if (e.on.has(rep[c])) { t = new_id[e.to]; break; }
+            out->table[(size_t)i * n_cls + c] = t;
+        }
+    }
+    uint64_t h = 0xCBF29CE484222325ull;
+    h = fnv1a(h, &out->n_states, 4);
+    h = fnv1a(h, &out->n_classes, 4);
+    h = fnv1a(h, &out->done, 4);
+    h = fnv1a(h, &out->eos_class, 4);
+    h = fnv1a(h, out->byte_class, 256);
+    h = fnv1a(h, out->table.data(), out->table.size() * sizeof(int32_t));
+    out->hash = h;
+    return WG_OK;
+}

@@ -1,0 +1,120 @@
+"""Host-side checks that need no GPU: the library loads and exports what wg.h declares, and
+the operator-to-table lowering agrees with the CPU checker transition by transition."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+import oracle
+from cosim import co_reachable, mentioned_symbols
+from wg_workloads import (ALL_BYTES, EOS, Cond, DoWhile, IfElse, Sequence, SymSet, Wait, Write,
+                          flatten, grammars)
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def wg():
+    from paper_2507_16768_b200 import build
+    build.build()
+    import paper_2507_16768_b200 as wg
+    return wg
+
+
+def test_library_exports_every_declared_symbol(wg):
+    header = open(os.path.join(ROOT, "include", "wg.h")).read()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    declared = set(re.findall(r"\b(wg_[a-z0-9_]+)\s*\(", header))
+    assert {"wg_load_vocab", "wg_compile_grammar", "wg_build_masks", "wg_mask_cache_lookup",
+            "wg_apply_mask", "wg_advance"} <= declared
+    lib = ctypes.CDLL(wg.binding.LIB_PATH)
+    for name in sorted(declared):
+        assert hasattr(lib, name), f"{name} is declared in wg.h but not exported"
+    assert declared == set(wg.binding.EXPORTED)
+
+
+def test_strerror_and_launch_counter(wg):
+    lib = ctypes.CDLL(wg.binding.LIB_PATH)
+    lib.wg_strerror.restype = ctypes.c_char_p
+    assert lib.wg_strerror(0) == b"ok"
+    assert b"grammar" in lib.wg_strerror(-2)
+    assert wg.kernel_launch_count() >= 0
+
+
+GRAMMARS = {
+    "listing": grammars.paper_listing_example,
+    "html": grammars.html_template,
+    "json_generic": lambda: grammars.json_reference_lookup(doc_nodes=0),
+    "json_doc": lambda: grammars.json_reference_lookup(doc_nodes=120),
+    "template1": lambda: grammars.random_template(1),
+    "template6": lambda: grammars.random_template(6),
+    "snippets": lambda: grammars.dynamic_snippet_template(2, n_args=3, enum_size=12),
+    "empty_bodies": lambda: Sequence(
+        Write(b""), DoWhile(None, Cond(ALL_BYTES, SymSet(b","), SymSet(b";"))),
+        Wait(SymSet(b"ab"), SymSet(b"!"), body=Sequence()), IfElse(
+            Cond(SymSet(b"xyz"), SymSet(b"y"), SymSet(b"z")), None, Sequence(Write(b""))),
+        Write(b"end")),
+}
+
+
+@pytest.mark.parametrize("name", sorted(GRAMMARS))
+def test_lowered_table_matches_checker_on_every_reachable_transition(wg, name):
+    op = GRAMMARS[name]()
+    flat = flatten(op)
+    tree = oracle.Tree(flat)
+    g = wg.Grammar(flat)
+    symbols = range(257) if flat.n_nodes < 60 else mentioned_symbols(flat)
+    cursor_of = co_reachable(tree, g, symbols)
+    # every table state is reachable and was paired (state 0 is DEAD)
+    assert sorted(cursor_of) == list(range(1, g.n_states))
+    assert g.start_state == 1
+    assert cursor_of[g.done_state] == oracle.DONE
+    assert g.step(g.done_state, EOS) == g.done_state
+    assert all(g.step(0, s) == 0 for s in (0, 65, EOS))
+    assert g.step(g.n_states, 65) == 0 and g.step(1, 257) == 0 and g.step(-1, 0) == 0
+
+
+def test_identical_trees_hash_equal_and_different_trees_do_not(wg):
+    a = wg.Grammar(flatten(grammars.random_template(3)))
+    b = wg.Grammar(flatten(grammars.random_template(3)))
+    c = wg.Grammar(flatten(grammars.random_template(4)))
+    assert a.content_hash == b.content_hash != c.content_hash
+
+
+@pytest.mark.parametrize("bad", [
+    Wait(allow=SymSet(b"a"), wait=SymSet()),
+    Wait(allow=SymSet(b"ab"), wait=SymSet(b"b"), deny=SymSet(b"b")),
+    IfElse(Cond(SymSet(b"ab"), SymSet(b"ab"), SymSet(b"b")), None, None),
+    DoWhile(Write(b"x"), Cond(SymSet(b"a"), SymSet(b"a"), SymSet())),
+])
+def test_compile_rejects_what_the_checker_rejects(wg, bad):
+    flat = flatten(bad)
+    with pytest.raises(oracle.OracleError) as oe:
+        oracle.Tree(flat)
+    with pytest.raises(wg.WgError) as we:
+        wg.Grammar(flat)
+    assert oe.value.code == oracle.ERR_GRAMMAR and we.value.status == wg.binding.WG_ERR_GRAMMAR
+
+
+def test_compile_rejects_malformed_arrays(wg):
+    flat = flatten(Sequence(Write(b"a"), Write(b"b")))
+    flat.children[1] = flat.children[0]
+    with pytest.raises(wg.WgError) as e:
+        wg.Grammar(flat)
+    assert e.value.status == wg.binding.WG_ERR_GRAMMAR
+    flat = flatten(Sequence(Write(b"a"), Write(b"b")))
+    flat.nodes[1, 6] = 99          # literal runs past the data array
+    with pytest.raises(wg.WgError) as e:
+        wg.Grammar(flat)
+    assert e.value.status == wg.binding.WG_ERR_ARG
+    flat = flatten(Write(b"a"))
+    flat.root = 5
+    with pytest.raises(wg.WgError):
+        wg.Grammar(flat)
+
+
+def test_large_enum_grammar_needs_wide_state_ids(wg):
+    g = wg.Grammar(flatten(grammars.dynamic_snippet_template(0, n_args=8, enum_size=1000)))
+    assert g.n_states > 40000

@@ -92,14 +92,41 @@ def id_path_string() -> Op:
     )
 
 
-def json_reference_lookup() -> Op:
-    """Configs 2 and 4: an array of {"topic": <0..63>, "paths": [<id path>, ...]}."""
+def document_node_paths(seed: int, n_nodes: int) -> List[bytes]:
+    """Node-id paths ("3", "3/1", "3/1/12", ...) of a seeded random document tree."""
+    rng = np.random.Generator(np.random.Philox(key=[seed, 0x646F63]))
+    paths: List[bytes] = []
+    frontier: List[tuple] = [(b"", 0)]
+    while frontier and len(paths) < n_nodes:
+        prefix, depth = frontier.pop(int(rng.integers(0, len(frontier))))
+        fan = int(rng.integers(2, 16)) if depth < 4 else 0
+        for k in range(1, fan + 1):
+            if len(paths) >= n_nodes:
+                break
+            path = (prefix + b"/" if prefix else b"") + str(k).encode()
+            paths.append(path)
+            frontier.append((path, depth + 1))
+    return paths
+
+
+def json_reference_lookup(doc_seed: int = 0, doc_nodes: int = 1350) -> Op:
+    """Configs 2 and 4: an array of {"topic": <0..63>, "paths": [<id path>, ...]}.
+
+    With ``doc_nodes`` > 0 every path string must be the id path of a node of the request's
+    document (Section 1: values are restricted to section ids), an enum over a seeded random
+    document tree; with ``doc_nodes`` = 0 it is any /-separated run of decimal ids.
+    """
     more_or_close = Cond(allow=SymSet(b",]"), true_waits=SymSet(b","), false_waits=SymSet(b"]"))
+    if doc_nodes > 0:
+        names = [p + b'"' for p in document_node_paths(doc_seed, doc_nodes)]
+        path = Sequence(Write(b'"'), enum_trie(names))
+    else:
+        path = id_path_string()
     obj = Sequence(
         Write(b'{"topic": '),
         int_0_63(b","),
         Write(b' "paths": ['),
-        DoWhile(body=id_path_string(), condition=more_or_close),
+        DoWhile(body=path, condition=more_or_close),
         Write(b"}"),
     )
     return Sequence(Write(b"["), DoWhile(body=obj, condition=more_or_close))
@@ -134,12 +161,12 @@ def random_template(seed: int, min_segments: int = 10, max_segments: int = 30) -
             parts.append(IfElse(
                 condition=Cond(allow=SymSet([a, b]), true_waits=SymSet([a]),
                                false_waits=SymSet([b])),
-                if_body=Write(_literal(rng, 6, 24)),
-                else_body=(Write(_literal(rng, 6, 24)) if rng.random() < 0.7 else None)))
+                if_body=Write(_literal(rng, 12, 48)),
+                else_body=(Write(_literal(rng, 12, 48)) if rng.random() < 0.7 else None)))
         else:
             sep, end = (int(x) for x in rng.choice(np.frombuffer(b",;|]})", dtype=np.uint8),
                                                   size=2, replace=False))
-            item = Sequence(Write(_literal(rng, 3, 16)), Wait(allow=DIGITS, wait=DIGITS))
+            item = Sequence(Write(_literal(rng, 8, 32)), Wait(allow=DIGITS, wait=DIGITS))
             parts.append(DoWhile(
                 body=item,
                 condition=Cond(allow=DIGITS | [sep, end], true_waits=SymSet([sep]),
