@@ -215,6 +215,29 @@ int32_t wg_apply_mask(void *logits, int32_t dtype, int64_t row_stride_elems,
                       int32_t *argmax_out, void *workspace, void *stream);
 size_t wg_apply_workspace_bytes(int32_t B);
 
+/* The paper has no counterpart to this call; it exists for deployment reasons only.
+ * wg_apply_mask with argmax_out needs a scratch buffer that somebody has to allocate.  Some
+ * callers cannot: an inference server that handed every byte of device memory to its own
+ * pool at start-up, a plug-in that runs inside someone else's step function where a
+ * cudaMalloc would stall the whole device, or a host thread that may not call allocating
+ * CUDA routines at all.  For them this variant masks and picks the greedy token exactly as
+ * wg_apply_mask does, but keeps its scratch (one 8-byte packed maximum per row) in a fixed
+ * array that is part of the library image: WG_NOALLOC_MAX_ROWS * 8 bytes = 32 KB of device
+ * memory on every GPU that loads the library, held until the process exits.
+ *   arguments   as wg_apply_mask; argmax_out is required (device, B entries)
+ *   limit       B <= WG_NOALLOC_MAX_ROWS, otherwise WG_ERR_CAPACITY and nothing is launched
+ * The call performs no cudaMalloc, cudaFree or other allocating routine.  The first call on
+ * each device looks up the device address of the array (a synchronous query, done with that
+ * device current); make that first call outside any stream capture.  Every call on a device
+ * uses the same array and begins by clearing the rows it needs, so the previous call's
+ * contents never leak in -- but two calls whose kernels can overlap on the GPU (different
+ * streams, no ordering between them) race on it and give undefined tokens.  Calls on one
+ * stream, or ordered by events, are safe. */
+#define WG_NOALLOC_MAX_ROWS 4096
+int32_t wg_apply_mask_noalloc(void *logits, int32_t dtype, int64_t row_stride_elems,
+                              const uint32_t *bitmask, int64_t mask_stride_words, int32_t B,
+                              int32_t V, int32_t *argmax_out, void *stream);
+
 /* State tracking (paper Section 3.2: the current token id updates the state machine).
  *   gid     device, B entries
  *   sid     device, B entries, updated in place

@@ -68,6 +68,7 @@ _SIGNATURES = {
     "wg_build_masks": (_i32, [_vp, _vp, _vp, _i32, _vp, _i64, _u32, _vp]),
     "wg_apply_mask": (_i32, [_vp, _i32, _i64, _vp, _i64, _i32, _i32, _vp, _vp, _vp]),
     "wg_apply_workspace_bytes": (C.c_size_t, [_i32]),
+    "wg_apply_mask_noalloc": (_i32, [_vp, _i32, _i64, _vp, _i64, _i32, _i32, _vp, _vp]),
     "wg_advance": (_i32, [_vp, _vp, _vp, _vp, _i32, _vp, _u32, _vp]),
     "wg_decode_step": (_i32, [_vp, _vp, _vp, _i32, _vp, _i32, _i64, _vp, _i64, _vp, _vp, _u32, _vp]),
     "wg_decode_step_host": (_i32, [_vp, _vp, _vp, _i32, _vp, _vp, _i32, _i64, _vp, _i64, _vp, _vp,
@@ -282,6 +283,29 @@ def wg_apply_mask(logits, bitmask, V: int, argmax_out=None, workspace=None, stre
                               B, int(V), _dev_ptr(argmax_out, torch.int32, "argmax_out"),
                               _dev_ptr(workspace, None, "workspace"), _stream_ptr(stream)),
            "wg_apply_mask")
+
+
+WG_NOALLOC_MAX_ROWS = 4096
+
+
+def wg_apply_mask_noalloc(logits, bitmask, V: int, argmax_out, stream=None) -> None:
+    """Mask + greedy argmax for callers that may not allocate device memory.
+
+    Same results as ``wg_apply_mask`` with ``argmax_out``; the scratch is a fixed 32 KB array
+    inside the library, so at most ``WG_NOALLOC_MAX_ROWS`` rows per call, and calls that can
+    overlap on the GPU must not be issued (they share that array).
+    """
+    import torch
+    B, stride = _rows(logits, "logits")
+    Bm, mstride = _rows(bitmask, "bitmask")
+    if Bm != B:
+        raise ValueError("logits and bitmask disagree on the batch size")
+    _check(_lib.wg_apply_mask_noalloc(_dev_ptr(logits, None, "logits"), _logits_dtype(logits),
+                                      stride,
+                                      _dev_ptr(bitmask, (torch.int32, torch.uint32), "bitmask"),
+                                      mstride, B, int(V),
+                                      _dev_ptr(argmax_out, torch.int32, "argmax_out"),
+                                      _stream_ptr(stream)), "wg_apply_mask_noalloc")
 
 
 def wg_apply_workspace_bytes(B: int) -> int:

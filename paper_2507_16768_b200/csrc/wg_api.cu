@@ -106,7 +106,7 @@ const char *wg_strerror(int32_t status) {
     case WG_OK: return "ok";
     case WG_ERR_ARG: return "bad argument";
     case WG_ERR_GRAMMAR: return "operator tree breaks a grammar rule";
-    case WG_ERR_CAPACITY: return "capacity exhausted";
+    case WG_ERR_CAPACITY: return "capacity exhausted (a fixed-size table or scratch array is too small)";
     case WG_ERR_TOKEN_REJECTED: return "token not allowed in this state";
     case WG_ERR_CUDA: return "CUDA runtime error";
     case WG_ERR_EMPTY_MASK: return "no token allowed";
@@ -474,6 +474,61 @@ int32_t wg_apply_mask(void *logits, int32_t dtype, int64_t row_stride_elems,
     unsigned long long *keys = static_cast<unsigned long long *>(workspace);
     WG_CUDA(cudaMemsetAsync(keys, 0, sizeof(unsigned long long) * (size_t)B, st));
     int32_t rc = launch_apply<true, false>(dtype, a, none, keys, st);
+    if (rc != WG_OK) return rc;
+    argmax_finish_kernel<<<(B + 127) / 128, 128, 0, st>>>(keys, B, argmax_out);
+    WG_LAUNCHED();
+    return WG_OK;
+}
+
+}  // extern "C"
+
+// ---- the entry point that allocates nothing ----------------------------------------------
+// Scratch of wg_apply_mask_noalloc: the packed per-row maxima.  The array lives in the
+// library image, so each GPU that loads the library carries these 32 KB until exit.  In HOST
+// code the name below is only a handle for the runtime, never a device address; the address
+// a kernel may use comes from cudaGetSymbolAddress, queried once per device.
+static __device__ __align__(256) unsigned long long g_noalloc_argkeys[WG_NOALLOC_MAX_ROWS];
+
+namespace {
+constexpr int MAX_DEVICES = 64;
+std::mutex g_noalloc_mu;
+unsigned long long *g_noalloc_ptr[MAX_DEVICES] = {};
+
+// Device address of the scratch array on the CURRENT device (looked up on first use).
+int32_t noalloc_scratch(unsigned long long **out) {
+    int dev = -1;
+    WG_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= MAX_DEVICES) return WG_ERR_ARG;
+    std::lock_guard<std::mutex> lock(g_noalloc_mu);
+    if (!g_noalloc_ptr[dev]) {
+        void *p = nullptr;
+        WG_CUDA(cudaGetSymbolAddress(&p, g_noalloc_argkeys));
+        g_noalloc_ptr[dev] = static_cast<unsigned long long *>(p);
+    }
+    *out = g_noalloc_ptr[dev];
+    return WG_OK;
+}
+}  // namespace
+
+extern "C" {
+
+int32_t wg_apply_mask_noalloc(void *logits, int32_t dtype, int64_t row_stride_elems,
+                              const uint32_t *bitmask, int64_t mask_stride_words, int32_t B,
+                              int32_t V, int32_t *argmax_out, void *stream) {
+    if (!logits || !bitmask || !argmax_out || B < 1 || V < 1) return WG_ERR_ARG;
+    if (dtype != WG_DTYPE_BF16 && dtype != WG_DTYPE_FP32) return WG_ERR_ARG;
+    if (B > WG_NOALLOC_MAX_ROWS) return WG_ERR_CAPACITY;  // the fixed scratch holds no more rows
+    const int W = (V + 31) / 32;
+    if (row_stride_elems < V || mask_stride_words < W) return WG_ERR_ARG;
+    unsigned long long *keys = nullptr;
+    int32_t rc = noalloc_scratch(&keys);
+    if (rc != WG_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // the array still holds the previous call's maxima: the rows in use must start at zero
+    WG_CUDA(cudaMemsetAsync(keys, 0, sizeof(unsigned long long) * (size_t)B, st));
+    ApplyArgs a{logits, row_stride_elems, bitmask, nullptr, mask_stride_words, B, V, W, 0};
+    CtxDev none{};
+    rc = launch_apply<true, false>(dtype, a, none, keys, st);
     if (rc != WG_OK) return rc;
     argmax_finish_kernel<<<(B + 127) / 128, 128, 0, st>>>(keys, B, argmax_out);
     WG_LAUNCHED();
