@@ -231,7 +231,8 @@ def run_ours(args, w, steer: float) -> None:
     grammar_ids = sorted({w.grammar_of_row(r) for r in range(B)})
     compiled = {g: wg.Grammar(flatten(w.grammar(g))) for g in grammar_ids}
     n_states = sum(c.n_states for c in compiled.values())
-    capacity = n_states + 64 if w.use_cache else 0
+    # every state of every grammar, but never more rows than a run can visit
+    capacity = min(n_states + 64, 1 << 16) if w.use_cache else 0
     ctx = wg.Context(dv, capacity, B)
     gid_of = {g: ctx.add_grammar(c) for g, c in compiled.items()}
     if w.prewarm:
@@ -288,18 +289,22 @@ def run_ours(args, w, steer: float) -> None:
 
     run_steps(args.warmup, False)
     ctx.reset_stats()
-    ctx.set_timing(True)
     sampler = ClockSampler(local) if rank == 0 else None
     launches0 = wg.kernel_launch_count()
     t_wall0 = time.perf_counter()
     ms = run_steps(args.steps, True)
     wall = time.perf_counter() - t_wall0
     launches = wg.kernel_launch_count() - launches0
-    clocks = sampler.stop() if sampler else {}
-    kt = ctx.get_timing()
-    ctx.set_timing(False)
     stats = ctx.stats()
     bad = int((d_status != 0).sum().item())
+    # per-kernel durations: the same steps once more, now with the library recording CUDA
+    # events around its kernels on the launching stream (the events sit between the kernels,
+    # so this pass is kept out of the headline time)
+    ctx.set_timing(True)
+    kernel_pass_ms = run_steps(min(args.steps, 4096), True)
+    kt = ctx.get_timing()
+    ctx.set_timing(False)
+    clocks = sampler.stop() if sampler else {}
 
     if world > 1:
         t = torch.tensor([ms], dtype=torch.float64, device="cuda")
@@ -344,12 +349,15 @@ def run_ours(args, w, steer: float) -> None:
     apply_ms = kt["apply_ms"] / max(1, kt["steps"])
     build_ms = kt["build_ms"] / max(1, kt["steps"])
     built = stats["masks_built"]
+    del kernel_pass_ms
     if w.use_cache or build_ms < apply_ms:
         achieved = algo_bytes / (apply_ms * 1e-3) / 1e9 if apply_ms > 0 else 0.0
         roofline = {"kernel": "apply_mask_kernel (gather + apply + argmax)", "bound": "hbm",
                     "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                     "peak_kind": f"of {peak_kind}", "traffic": None,
-                    "algorithmic_bytes_per_launch": algo_bytes, "avg_launch_ms": apply_ms}
+                    "algorithmic_bytes_per_launch": algo_bytes, "avg_launch_ms": apply_ms,
+                    "timed_by": "CUDA events recorded by the library around the kernel, in a "
+                                "second pass over the same steps"}
     else:
         tok_per_s = built * V / (kt["build_ms"] * 1e-3) if kt["build_ms"] > 0 else 0.0
         roofline = {"kernel": "build_masks_kernel", "bound": "alu", "achieved": tok_per_s / 1e9,
@@ -368,7 +376,7 @@ def run_ours(args, w, steer: float) -> None:
                    "timing": "CUDA events per chunk of <= ring steps; logits restored between "
                              "chunks outside the timed region"},
         "roofline": roofline,
-        "kernel_ms": {"build": build_ms, "apply": apply_ms},
+        "kernel_ms": {"lookup_and_build": build_ms, "apply": apply_ms},
         "tokens_checked_per_s": (built * V) / (ms * 1e-3) if built else 0.0,
         "cache": {k: stats[k] for k in ("cache_hits", "cache_misses", "masks_built",
                                          "rows_uncached", "cache_entries")},

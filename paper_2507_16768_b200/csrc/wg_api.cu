@@ -42,6 +42,24 @@ int sm_count() {
     return g_sm_count;
 }
 
+// Launch with programmatic stream serialization: the kernel may be scheduled while the
+// kernel before it in the stream is still running; it orders itself with griddepcontrol.wait.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, cudaStream_t st,
+                       Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 template <typename T>
 int32_t dev_alloc(T **p, size_t n) {
     *p = nullptr;
@@ -376,14 +394,19 @@ int32_t wg_reset_stats(wg_ctx *c, void *stream) {
 // ---- launch helpers -------------------------------------------------------------------
 namespace {
 
-int32_t launch_build(wg_ctx *c, const BuildWork &work, int max_entries, cudaStream_t st) {
+int32_t launch_build(wg_ctx *c, const BuildWork &work, int max_entries, cudaStream_t st,
+                     bool pdl = false) {
     const VocabDev &v = c->vocab->dev;
     const long long n_chunks = ((long long)v.W * 32 + BUILD_CHUNK - 1) / BUILD_CHUNK;
     long long items = (long long)max_entries * n_chunks;
     long long grid = (long long)sm_count() * 8;  // 8 resident blocks of 256 threads per SM
     if (items < grid) grid = items;
     if (grid < 1) grid = 1;
-    build_masks_kernel<<<(unsigned)grid, BUILD_THREADS, 0, st>>>(v, c->dev, work);
+    if (pdl)
+        WG_CUDA(launch_pdl(build_masks_kernel, dim3((unsigned)grid), dim3(BUILD_THREADS), st, v,
+                           c->dev, work));
+    else
+        build_masks_kernel<<<(unsigned)grid, BUILD_THREADS, 0, st>>>(v, c->dev, work);
     WG_LAUNCHED();
     return WG_OK;
 }
@@ -392,31 +415,46 @@ bool rows_aligned(const void *p, int64_t stride_elems, size_t elem) {
     return ((uintptr_t)p % 16 == 0) && ((stride_elems * (int64_t)elem) % 16 == 0);
 }
 
-template <typename E, bool ARGMAX, bool GATHER>
-int32_t launch_apply_t(const ApplyArgs &a_in, const CtxDev &ctx, unsigned long long *argkey,
-                       cudaStream_t st) {
-    ApplyArgs a = a_in;
+// Grid of the apply kernels, (blocks per row, B), and the spans each block handles: enough
+// blocks to fill the machine a few times over, at least 8 spans (16 KB of bf16) per block.
+dim3 apply_grid(ApplyArgs &a) {
     const int n_spans = (a.W + 31) / 32;
-    // enough blocks to fill the machine a few times over, at least 8 spans (16 KB bf16) each
     int blocks_per_row = (sm_count() * 16 + a.B - 1) / a.B;
     if (blocks_per_row > (n_spans + 7) / 8) blocks_per_row = (n_spans + 7) / 8;
     if (blocks_per_row < 1) blocks_per_row = 1;
     a.spans_per_block = (n_spans + blocks_per_row - 1) / blocks_per_row;
     blocks_per_row = (n_spans + a.spans_per_block - 1) / a.spans_per_block;
-    dim3 grid((unsigned)blocks_per_row, (unsigned)a.B);
-    if (rows_aligned(a.logits, a.row_stride, sizeof(E)))
+    return dim3((unsigned)blocks_per_row, (unsigned)a.B);
+}
+
+template <typename E, bool ARGMAX, bool GATHER>
+int32_t launch_apply_t(const ApplyArgs &a_in, const CtxDev &ctx, unsigned long long *argkey,
+                       cudaStream_t st, bool pdl) {
+    ApplyArgs a = a_in;
+    dim3 grid = apply_grid(a);
+    const bool aligned = rows_aligned(a.logits, a.row_stride, sizeof(E));
+    if (pdl) {
+        if (aligned)
+            WG_CUDA(launch_pdl(apply_mask_kernel<E, ARGMAX, GATHER>, grid, dim3(APPLY_THREADS), st,
+                               a, ctx, argkey));
+        else
+            WG_CUDA(launch_pdl(apply_mask_unaligned_kernel<E, ARGMAX, GATHER>, grid,
+                               dim3(APPLY_THREADS), st, a, ctx, argkey));
+    } else if (aligned) {
         apply_mask_kernel<E, ARGMAX, GATHER><<<grid, APPLY_THREADS, 0, st>>>(a, ctx, argkey);
-    else
+    } else {
         apply_mask_unaligned_kernel<E, ARGMAX, GATHER><<<grid, APPLY_THREADS, 0, st>>>(a, ctx, argkey);
+    }
     WG_LAUNCHED();
     return WG_OK;
 }
 
 template <bool ARGMAX, bool GATHER>
 int32_t launch_apply(int32_t dtype, const ApplyArgs &a, const CtxDev &ctx,
-                     unsigned long long *argkey, cudaStream_t st) {
-    if (dtype == WG_DTYPE_BF16) return launch_apply_t<uint16_t, ARGMAX, GATHER>(a, ctx, argkey, st);
-    return launch_apply_t<uint32_t, ARGMAX, GATHER>(a, ctx, argkey, st);
+                     unsigned long long *argkey, cudaStream_t st, bool pdl = false) {
+    if (dtype == WG_DTYPE_BF16)
+        return launch_apply_t<uint16_t, ARGMAX, GATHER>(a, ctx, argkey, st, pdl);
+    return launch_apply_t<uint32_t, ARGMAX, GATHER>(a, ctx, argkey, st, pdl);
 }
 
 bool batch_ok(const wg_ctx *c, int32_t B) { return c && B >= 1 && B <= c->max_batch; }
@@ -556,32 +594,35 @@ int32_t wg_decode_step(wg_ctx *c, const int32_t *gid, int32_t *sid, int32_t B, v
     if (row_stride_elems < v.V || mask_stride_words < v.W) return WG_ERR_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     ApplyArgs a{logits, row_stride_elems, bitmask, bitmask, mask_stride_words, B, v.V, v.W, 0};
+    const bool no_cache = (flags & WG_NO_CACHE) != 0;
+    // Every kernel of the step is launched with programmatic stream serialization and starts
+    // with griddepcontrol.wait, so launch latency and block scheduling of a kernel overlap the
+    // tail of the one before it (also across consecutive steps on one stream).
     int32_t rc;
-    if (flags & WG_NO_CACHE) {
-        reset_rows_kernel<<<(B + 255) / 256, 256, 0, st>>>(c->dev, B);
+    if ((rc = timing_mark(c, 0, st)) != WG_OK) return rc;
+    if (no_cache) {
+        // rows have no pool row; the packed maxima were left at zero by the last advance
+        WG_CUDA(launch_pdl(reset_rows_kernel, dim3((B + 255) / 256), dim3(256), st, c->dev, B));
         WG_LAUNCHED();
         BuildWork work{gid, sid, nullptr, bitmask, mask_stride_words, nullptr, B};
-        if ((rc = timing_mark(c, 0, st)) != WG_OK) return rc;
-        rc = launch_build(c, work, B, st);
-        if (rc != WG_OK) return rc;
-        if ((rc = timing_mark(c, 1, st)) != WG_OK) return rc;
-        if ((rc = timing_mark(c, 2, st)) != WG_OK) return rc;
-        rc = launch_apply<true, false>(dtype, a, c->dev, c->dev.argkey, st);
+        rc = launch_build(c, work, B, st, true);
     } else {
-        cache_lookup_insert_kernel<<<1, 1024, 0, st>>>(c->dev, gid, sid, B, bitmask, mask_stride_words);
+        WG_CUDA(launch_pdl(cache_lookup_insert_kernel, dim3(1), dim3(1024), st, c->dev, gid, sid, B,
+                           bitmask, mask_stride_words));
         WG_LAUNCHED();
         BuildWork work{c->dev.bl_gid, c->dev.bl_sid, c->dev.bl_dst, nullptr, 0, c->dev.bl_count, 0};
-        if ((rc = timing_mark(c, 0, st)) != WG_OK) return rc;
-        rc = launch_build(c, work, B, st);
-        if (rc != WG_OK) return rc;
-        if ((rc = timing_mark(c, 1, st)) != WG_OK) return rc;
-        if ((rc = timing_mark(c, 2, st)) != WG_OK) return rc;
-        rc = launch_apply<true, true>(dtype, a, c->dev, c->dev.argkey, st);
+        rc = launch_build(c, work, B, st, true);
     }
     if (rc != WG_OK) return rc;
+    if ((rc = timing_mark(c, 1, st)) != WG_OK) return rc;
+    if ((rc = timing_mark(c, 2, st)) != WG_OK) return rc;
+    rc = no_cache ? launch_apply<true, false>(dtype, a, c->dev, c->dev.argkey, st, true)
+                  : launch_apply<true, true>(dtype, a, c->dev, c->dev.argkey, st, true);
+    if (rc != WG_OK) return rc;
     if ((rc = timing_mark(c, 3, st)) != WG_OK) return rc;
-    advance_kernel<<<(B + 127) / 128, 128, 0, st>>>(v, c->dev, gid, sid, nullptr, token_out, B,
-                                                    status, flags & WG_RESTART_ON_DONE, 1);
+    WG_CUDA(launch_pdl(advance_kernel, dim3((B + 127) / 128), dim3(128), st, v, c->dev, gid, sid,
+                       (const int32_t *)nullptr, token_out, B, status,
+                       (uint32_t)(flags & WG_RESTART_ON_DONE), 1));
     WG_LAUNCHED();
     return WG_OK;
 }

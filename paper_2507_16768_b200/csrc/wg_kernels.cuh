@@ -53,6 +53,8 @@ struct CtxDev {
 constexpr uint32_t NEG_INF_F32 = 0xFF800000u;
 constexpr uint32_t NEG_INF_BF16X2 = 0xFF80FF80u;
 
+__device__ __forceinline__ void pdl_enter();
+
 // ---------------------------------------------------------------------------------------
 // table walk
 // ---------------------------------------------------------------------------------------
@@ -122,6 +124,7 @@ __global__ void __launch_bounds__(BUILD_THREADS)
 build_masks_kernel(VocabDev v, CtxDev ctx, BuildWork work) {
     __shared__ uint8_t cls[256];
     __shared__ int cls_gid;
+    pdl_enter();
     if (threadIdx.x == 0) cls_gid = -1;
     __syncthreads();
     const int n_entries = work.count_ptr ? *work.count_ptr : work.count;
@@ -193,6 +196,7 @@ __global__ void cache_lookup_kernel(CtxDev ctx, const int32_t *gid, const int32_
 __global__ void __launch_bounds__(1024)
 cache_lookup_insert_kernel(CtxDev ctx, const int32_t *gid, const int32_t *sid, int B,
                            uint32_t *bitmask, int64_t mask_stride) {
+    pdl_enter();
     if (threadIdx.x == 0) *ctx.bl_count = 0;
     __syncthreads();
     const uint32_t mask = (uint32_t)ctx.hash_size - 1;
@@ -231,14 +235,15 @@ cache_lookup_insert_kernel(CtxDev ctx, const int32_t *gid, const int32_t *sid, i
         ctx.ent[r] = (entry >= 0 && inserted) ? (entry | ENT_NEW) : entry;
     }
     __syncthreads();
+    int hits = 0, misses = 0, uncached = 0;
     for (int r = threadIdx.x; r < B; r += blockDim.x) {
         const int32_t e = ctx.ent[r];
         const int32_t row = e >= 0 ? ctx.vals[e & ~ENT_NEW] : -1;
         ctx.slot[r] = row;
         // a hit is a row served from a pool row that some earlier row or call already owned
-        atomicAdd(&ctx.stats[(row >= 0 && !(e & ENT_NEW)) ? ST_HITS : ST_MISSES], 1ull);
+        if (row >= 0 && !(e & ENT_NEW)) ++hits; else ++misses;
         if (row < 0) {
-            atomicAdd(&ctx.stats[ST_UNCACHED], 1ull);
+            ++uncached;
             if (bitmask) {
                 const int i = atomicAdd(ctx.bl_count, 1);
                 ctx.bl_gid[i] = gid[r];
@@ -247,10 +252,23 @@ cache_lookup_insert_kernel(CtxDev ctx, const int32_t *gid, const int32_t *sid, i
             }
         }
     }
+    // one atomic per warp and counter instead of one per row
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        hits += __shfl_xor_sync(0xFFFFFFFFu, hits, o);
+        misses += __shfl_xor_sync(0xFFFFFFFFu, misses, o);
+        uncached += __shfl_xor_sync(0xFFFFFFFFu, uncached, o);
+    }
+    if ((threadIdx.x & 31) == 0) {
+        if (hits) atomicAdd(&ctx.stats[ST_HITS], (unsigned long long)hits);
+        if (misses) atomicAdd(&ctx.stats[ST_MISSES], (unsigned long long)misses);
+        if (uncached) atomicAdd(&ctx.stats[ST_UNCACHED], (unsigned long long)uncached);
+    }
 }
 
 // Rows of a WG_NO_CACHE step: no pool row, and the packed maxima start at zero.
 __global__ void reset_rows_kernel(CtxDev ctx, int B) {
+    pdl_enter();
     const int r = blockIdx.x * blockDim.x + threadIdx.x;
     if (r < B) { ctx.slot[r] = -1; ctx.argkey[r] = 0ull; }
 }
@@ -358,60 +376,98 @@ __device__ __forceinline__ void block_argmax_commit(unsigned long long best,
     }
 }
 
+// Per-lane running maximum as (float value, id): a strict float compare keeps the first of
+// equal values and treats -0.0 and +0.0 as equal; !(v <= best) also takes the very first
+// allowed element, whatever its value (best starts as NaN).
+struct LaneBest {
+    float v;
+    int idx;
+    __device__ __forceinline__ void offer(uint32_t f32_bits, int t) {
+        const float x = __uint_as_float(f32_bits);
+        if (!(x <= v)) { v = x; idx = t; }
+    }
+    __device__ __forceinline__ unsigned long long packed() const {
+        return idx < 0 ? 0ull : pack_best(order_key(__float_as_uint(v)), idx);
+    }
+};
+
+// Programmatic dependent launch: let the next kernel of the stream be scheduled early, then
+// wait until the kernels before this one have finished and their writes are visible.  Both
+// are no-ops for a kernel launched without the attribute.
+__device__ __forceinline__ void pdl_enter() {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 // grid = (blocks per row, B).  Requires 16-byte aligned rows (pointer and stride).
 template <typename E, bool ARGMAX, bool GATHER>
 __global__ void __launch_bounds__(APPLY_THREADS)
 apply_mask_kernel(ApplyArgs a, CtxDev ctx, unsigned long long *argkey) {
     constexpr int EPC = ElemTraits<E>::PER_CHUNK;  // elements per chunk: bits per lane
     constexpr int CHUNKS_PER_WORD = 32 / EPC;      // 4 (bf16) or 8 (fp32)
-    constexpr int PASSES = 32 * CHUNKS_PER_WORD / 32;  // 16-byte accesses per lane and span
+    constexpr int PASSES = CHUNKS_PER_WORD;        // 16-byte accesses per lane and span
+    constexpr int GROUP = 4;                       // accesses issued together
     constexpr uint32_t FULL = (1u << EPC) - 1;
+    constexpr uint32_t SKIP = 0xFFFFFFFFu;
+    pdl_enter();
     const int r = blockIdx.y;
     E *row = static_cast<E *>(a.logits) + (int64_t)r * a.row_stride;
-    const uint32_t *mrow = a.bitmask + (int64_t)r * a.mask_stride;
+    const uint32_t *own = a.bitmask + (int64_t)r * a.mask_stride;
+    const uint32_t *mrow = own;
     if (GATHER) {
         const int32_t slot = ctx.slot[r];
         if (slot >= 0) mrow = ctx.pool + (int64_t)slot * ctx.pool_stride;
     }
+    const bool copy_out = GATHER && mrow != own;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int n_spans = (a.W + 31) / 32;
     const int span_begin = blockIdx.x * a.spans_per_block;
     const int span_end = min(span_begin + a.spans_per_block, n_spans);
     const int full_chunks = a.V / EPC;  // chunks that lie wholly inside the row
-    unsigned long long best = 0ull;
+    LaneBest best{__uint_as_float(0x7FC00000u), -1};
 
     for (int span = span_begin + warp; span < span_end; span += APPLY_WARPS) {
         const int word0 = span * 32;
         uint32_t my_word = 0;
         if (word0 + lane < a.W) {
             my_word = mrow[word0 + lane];
-            if (GATHER && mrow != a.bitmask + (int64_t)r * a.mask_stride)
-                a.bitmask_out[(int64_t)r * a.mask_stride + word0 + lane] = my_word;
+            if (copy_out) a.bitmask_out[(int64_t)r * a.mask_stride + word0 + lane] = my_word;
         }
+        const int chunk0 = word0 * CHUNKS_PER_WORD;
 #pragma unroll
-        for (int p = 0; p < PASSES; ++p) {
-            const int c_in_span = p * 32 + lane;  // chunk index inside the span
-            const uint32_t word = __shfl_sync(0xFFFFFFFFu, my_word, c_in_span / CHUNKS_PER_WORD);
-            const uint32_t bits = (word >> (EPC * (c_in_span % CHUNKS_PER_WORD))) & FULL;
-            const int chunk = word0 * CHUNKS_PER_WORD + c_in_span;
-            if (chunk >= full_chunks) continue;
-            uint4 *ptr = reinterpret_cast<uint4 *>(row) + chunk;
-            if (bits == 0) {
-                const uint32_t ninf = sizeof(E) == 2 ? NEG_INF_BF16X2 : NEG_INF_F32;
-                *ptr = make_uint4(ninf, ninf, ninf, ninf);
-            } else if (ARGMAX || bits != FULL) {
-                uint4 v = *ptr;
-                uint32_t w[4] = {v.x, v.y, v.z, v.w};
+        for (int p0 = 0; p0 < PASSES; p0 += GROUP) {
+            // the independent loads of the group first, then patch / compare / store
+            uint4 val[GROUP];
+            uint32_t bits[GROUP];
+#pragma unroll
+            for (int q = 0; q < GROUP; ++q) {
+                const int c = (p0 + q) * 32 + lane;  // chunk index inside the span
+                const uint32_t word = __shfl_sync(0xFFFFFFFFu, my_word, c / CHUNKS_PER_WORD);
+                bits[q] = (word >> (EPC * (c % CHUNKS_PER_WORD))) & FULL;
+                if (chunk0 + c >= full_chunks) bits[q] = SKIP;
+                else if (bits[q] != 0 && (ARGMAX || bits[q] != FULL))
+                    val[q] = __ldcs(reinterpret_cast<const uint4 *>(row) + chunk0 + c);
+            }
+#pragma unroll
+            for (int q = 0; q < GROUP; ++q) {
+                if (bits[q] == SKIP) continue;
+                const int chunk = chunk0 + (p0 + q) * 32 + lane;
+                uint4 *ptr = reinterpret_cast<uint4 *>(row) + chunk;
+                if (bits[q] == 0) {
+                    const uint32_t ninf = sizeof(E) == 2 ? NEG_INF_BF16X2 : NEG_INF_F32;
+                    __stcs(ptr, make_uint4(ninf, ninf, ninf, ninf));
+                    continue;
+                }
+                if (!ARGMAX && bits[q] == FULL) continue;
+                uint32_t w[4] = {val[q].x, val[q].y, val[q].z, val[q].w};
                 const int t0 = chunk * EPC;
                 if (sizeof(E) == 2) {
 #pragma unroll
                     for (int i = 0; i < 8; ++i) {
-                        const uint32_t e = (w[i >> 1] >> (16 * (i & 1))) & 0xFFFFu;
-                        if ((bits >> i) & 1u) {
-                            if (ARGMAX) {
-                                const unsigned long long k = pack_best(order_key(e << 16), t0 + i);
-                                best = k > best ? k : best;
-                            }
+                        if ((bits[q] >> i) & 1u) {
+                            if (ARGMAX)
+                                best.offer((i & 1) ? (w[i >> 1] & 0xFFFF0000u) : (w[i >> 1] << 16),
+                                           t0 + i);
                         } else {
                             w[i >> 1] = (i & 1) ? ((w[i >> 1] & 0x0000FFFFu) | 0xFF800000u)
                                                 : ((w[i >> 1] & 0xFFFF0000u) | 0x0000FF80u);
@@ -420,30 +476,29 @@ apply_mask_kernel(ApplyArgs a, CtxDev ctx, unsigned long long *argkey) {
                 } else {
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
-                        if ((bits >> i) & 1u) {
-                            if (ARGMAX) {
-                                const unsigned long long k = pack_best(order_key(w[i]), t0 + i);
-                                best = k > best ? k : best;
-                            }
+                        if ((bits[q] >> i) & 1u) {
+                            if (ARGMAX) best.offer(w[i], t0 + i);
                         } else {
                             w[i] = NEG_INF_F32;
                         }
                     }
                 }
-                if (bits != FULL) *ptr = make_uint4(w[0], w[1], w[2], w[3]);
+                if (bits[q] != FULL) __stcs(ptr, make_uint4(w[0], w[1], w[2], w[3]));
             }
         }
     }
+    unsigned long long packed = best.packed();
     // elements after the last whole chunk (V not a multiple of the chunk size)
     if (blockIdx.x == gridDim.x - 1 && full_chunks * EPC < a.V)
-        apply_scalar<E, ARGMAX>(row, mrow, full_chunks * EPC, a.V, best);
-    block_argmax_commit<ARGMAX>(best, argkey + r);
+        apply_scalar<E, ARGMAX>(row, mrow, full_chunks * EPC, a.V, packed);
+    block_argmax_commit<ARGMAX>(packed, argkey + r);
 }
 
 // Any alignment: one block column per row, element-wise.
 template <typename E, bool ARGMAX, bool GATHER>
 __global__ void __launch_bounds__(APPLY_THREADS)
 apply_mask_unaligned_kernel(ApplyArgs a, CtxDev ctx, unsigned long long *argkey) {
+    pdl_enter();
     const int r = blockIdx.y;
     E *row = static_cast<E *>(a.logits) + (int64_t)r * a.row_stride;
     const uint32_t *own = a.bitmask + (int64_t)r * a.mask_stride;
@@ -474,11 +529,13 @@ __global__ void argmax_finish_kernel(const unsigned long long *argkey, int B, in
 __global__ void advance_kernel(VocabDev v, CtxDev ctx, const int32_t *gid, int32_t *sid,
                                const int32_t *token_in, int32_t *token_out, int B,
                                int32_t *status, uint32_t flags, int from_keys) {
+    pdl_enter();
     const int r = blockIdx.x * blockDim.x + threadIdx.x;
     if (r >= B) return;
     int t;
     if (from_keys) {
         t = unpack_best(ctx.argkey[r]);
+        ctx.argkey[r] = 0ull;  // ready for the next step
         token_out[r] = t;
     } else {
         t = token_in[r];
