@@ -207,6 +207,7 @@ def run_ours(args, w, steer: float) -> None:
     import torch.distributed as dist
 
     import paper_2507_16768_b200 as wg
+    from paper_2507_16768_b200.sharding import max_over_ranks
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -240,9 +241,10 @@ def run_ours(args, w, steer: float) -> None:
             ctx.cache_prewarm(gid_of[g])
     d_gid = torch.tensor([gid_of[w.grammar_of_row(r)] for r in range(B)], dtype=torch.int32,
                          device="cuda")
-    start = torch.tensor([compiled[w.grammar_of_row(r)].start_state for r in range(B)],
+    # a row that starts one step late sits in DONE first: it emits EOS and then restarts
+    d_sid = torch.tensor([compiled[w.grammar_of_row(r)].done_state if w.row_delay(r) else
+                          compiled[w.grammar_of_row(r)].start_state for r in range(B)],
                          dtype=torch.int32, device="cuda")
-    d_sid = start.clone()
     d_mask = torch.zeros((B, W), dtype=torch.int32, device="cuda")
     d_tok = torch.zeros(B, dtype=torch.int32, device="cuda")
     d_status = torch.zeros(B, dtype=torch.int32, device="cuda")
@@ -261,14 +263,22 @@ def run_ours(args, w, steer: float) -> None:
             x += bonus
         pristine.append(x.to(tdtype))
         del x
+    late = [r for r in range(B) if w.row_delay(r)]
+    if late:
+        # a late row sees, one step later, the logits of the row before it (its leader)
+        late_idx = torch.tensor(late, device="cuda")
+        for i in range(ring):
+            pristine[i][late_idx] = pristine[i - 1][late_idx - 1]
     work = [torch.empty_like(p) for p in pristine]
 
     def restore():
         for dst, src in zip(work, pristine):
             dst.copy_(src)
 
+    plan = wg.StepPlan(ctx, d_gid, d_sid, d_mask, d_tok, d_status, flags)
+
     def step(i):
-        wg.wg_decode_step(ctx, d_gid, d_sid, work[i % ring], d_mask, d_tok, d_status, flags)
+        plan(work[i % ring])
 
     def run_steps(n, timed):
         """n steps in chunks of at most `ring`; returns the summed device time in ms."""
@@ -306,10 +316,7 @@ def run_ours(args, w, steer: float) -> None:
     ctx.set_timing(False)
     clocks = sampler.stop() if sampler else {}
 
-    if world > 1:
-        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(ms, device="cuda")
     rows_total = B * args.steps * world
     value = rows_total / (ms * 1e-3)
 
@@ -332,10 +339,7 @@ def run_ours(args, w, steer: float) -> None:
                                    tok_host, d_status, flags)
         barrier()
         dt = time.perf_counter() - t0
-        if world > 1:
-            t = torch.tensor([dt], dtype=torch.float64, device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            dt = float(t.item())
+        dt = max_over_ranks(dt, device="cuda")
         e2e = {"value": B * n_e2e * world / dt, "unit": UNIT, "h2d_bytes_per_step": B * row_bytes,
                "d2h_bytes_per_step": 4 * B, "steps": n_e2e}
 

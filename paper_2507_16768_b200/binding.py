@@ -335,6 +335,43 @@ def wg_decode_step(ctx: Context, gid, sid, logits, bitmask, token_out, status=No
                                _stream_ptr(stream)), "wg_decode_step")
 
 
+class StepPlan:
+    """A wg_decode_step call with everything but the logits marshalled once.
+
+    The per-call work of the binding (pointer extraction, dtype and shape checks) costs more
+    than a small decode step takes on the GPU; a plan does it once for buffers that stay put
+    (ids, states, bitmask, tokens, status) and only takes the logits tensor per call.
+    """
+
+    def __init__(self, ctx: Context, gid, sid, bitmask, token_out, status=None,
+                 flags: int = WG_USE_CACHE, stream=None):
+        import torch
+        self._keep = (ctx, gid, sid, bitmask, token_out, status)
+        self.B, self._mstride = _rows(bitmask, "bitmask")
+        if gid.shape[0] != self.B or sid.shape[0] != self.B or token_out.shape[0] != self.B:
+            raise ValueError("gid, sid, token_out and bitmask disagree on the batch size")
+        self._ctx = ctx.handle
+        self._gid = _dev_ptr(gid, torch.int32, "gid")
+        self._sid = _dev_ptr(sid, torch.int32, "sid")
+        self._mask = _dev_ptr(bitmask, (torch.int32, torch.uint32), "bitmask")
+        self._tok = _dev_ptr(token_out, torch.int32, "token_out")
+        self._status = _dev_ptr(status, torch.int32, "status")
+        self._flags = int(flags)
+        self._stream = _stream_ptr(stream)
+        self._dtypes = {torch.bfloat16: WG_DTYPE_BF16, torch.float32: WG_DTYPE_FP32}
+        self._fn = _lib.wg_decode_step
+
+    def __call__(self, logits) -> None:
+        if logits.dim() != 2 or logits.shape[0] != self.B or logits.stride(1) != 1 \
+                or not logits.is_cuda:
+            raise ValueError("logits must be a CUDA tensor [B, V] with unit inner stride")
+        rc = self._fn(self._ctx, self._gid, self._sid, self.B, logits.data_ptr(),
+                      self._dtypes[logits.dtype], logits.stride(0), self._mask, self._mstride,
+                      self._tok, self._status, self._flags, self._stream)
+        if rc != WG_OK:
+            raise WgError(rc, "wg_decode_step")
+
+
 def wg_decode_step_host(ctx: Context, gid, sid, logits_host, logits_dev, bitmask, token_dev,
                         token_host, status=None, flags: int = WG_USE_CACHE, stream=None) -> None:
     """logits_host / token_host are CPU tensors (pinned for asynchronous copies)."""

@@ -2,6 +2,7 @@
 #include <atomic>
 #include <cstdio>
 #include <cstring>
+#include <cstdlib>
 #include <mutex>
 #include <new>
 #include <vector>
@@ -72,6 +73,7 @@ int32_t dev_alloc(T **p, size_t n) {
 struct wg_vocab {
     VocabDev dev{};
     void *d_rec = nullptr, *d_len = nullptr, *d_offsets = nullptr, *d_bytes = nullptr;
+    void *d_meta = nullptr, *d_sig = nullptr;
     int device = 0;
 };
 
@@ -79,7 +81,7 @@ struct GrammarSlot {
     uint64_t hash;
     std::vector<int32_t> table;  // host copy, for exact comparison on hash equality
     int32_t n_states, n_classes;
-    void *d_table, *d_cls;
+    void *d_table, *d_cls, *d_first_ok, *d_leaves;
 };
 
 struct wg_ctx {
@@ -149,10 +151,16 @@ int32_t wg_load_vocab(const uint32_t *offsets, const uint8_t *bytes, int32_t V, 
     if (total > 0 && !bytes) return WG_ERR_ARG;
 
     std::vector<uint8_t> rec((size_t)V * WG_REC_BYTES, 0), len(V, 0);
+    std::vector<uint32_t> meta(V, 0);
+    std::vector<unsigned long long> sig(V, 0ull);
     for (int32_t t = 0; t < V; ++t) {
         const uint32_t n = (t == eos_id) ? 0u : offsets[t + 1] - offsets[t];
         len[t] = (uint8_t)(n > 255u ? 255u : n);
         if (n) memcpy(&rec[(size_t)t * WG_REC_BYTES], bytes + offsets[t], n < WG_REC_BYTES ? n : WG_REC_BYTES);
+        unsigned long long folded = 0ull;  // which byte values (mod 64) occur anywhere in the token
+        for (uint32_t i = 0; i < n; ++i) folded |= 1ull << (bytes[offsets[t] + i] & 63);
+        sig[t] = folded;
+        meta[t] = (uint32_t)len[t] | (n ? (uint32_t)bytes[offsets[t]] << 8 : 0u);
     }
     wg_vocab *v = new (std::nothrow) wg_vocab();
     if (!v) return WG_ERR_ARG;
@@ -160,17 +168,25 @@ int32_t wg_load_vocab(const uint32_t *offsets, const uint8_t *bytes, int32_t V, 
     if (cudaGetDevice(&v->device) != cudaSuccess) return fail(WG_ERR_CUDA);
     if (cudaMalloc(&v->d_rec, rec.size()) != cudaSuccess ||
         cudaMalloc(&v->d_len, len.size()) != cudaSuccess ||
+        cudaMalloc(&v->d_meta, meta.size() * sizeof(uint32_t)) != cudaSuccess ||
+        cudaMalloc(&v->d_sig, sig.size() * sizeof(unsigned long long)) != cudaSuccess ||
         cudaMalloc(&v->d_offsets, sizeof(uint32_t) * ((size_t)V + 1)) != cudaSuccess ||
         cudaMalloc(&v->d_bytes, total ? total : 1) != cudaSuccess)
         return fail(WG_ERR_CUDA);
     if (cudaMemcpy(v->d_rec, rec.data(), rec.size(), cudaMemcpyHostToDevice) != cudaSuccess ||
         cudaMemcpy(v->d_len, len.data(), len.size(), cudaMemcpyHostToDevice) != cudaSuccess ||
+        cudaMemcpy(v->d_meta, meta.data(), meta.size() * sizeof(uint32_t),
+                   cudaMemcpyHostToDevice) != cudaSuccess ||
+        cudaMemcpy(v->d_sig, sig.data(), sig.size() * sizeof(unsigned long long),
+                   cudaMemcpyHostToDevice) != cudaSuccess ||
         cudaMemcpy(v->d_offsets, offsets, sizeof(uint32_t) * ((size_t)V + 1),
                    cudaMemcpyHostToDevice) != cudaSuccess ||
         (total && cudaMemcpy(v->d_bytes, bytes, total, cudaMemcpyHostToDevice) != cudaSuccess))
         return fail(WG_ERR_CUDA);
     v->dev.rec = static_cast<const uint4 *>(v->d_rec);
     v->dev.len = static_cast<const uint8_t *>(v->d_len);
+    v->dev.meta = static_cast<const uint32_t *>(v->d_meta);
+    v->dev.sig = static_cast<const unsigned long long *>(v->d_sig);
     v->dev.offsets = static_cast<const uint32_t *>(v->d_offsets);
     v->dev.bytes = static_cast<const uint8_t *>(v->d_bytes);
     v->dev.V = V;
@@ -184,6 +200,8 @@ void wg_vocab_free(wg_vocab *v) {
     if (!v) return;
     cudaFree(v->d_rec);
     cudaFree(v->d_len);
+    cudaFree(v->d_meta);
+    cudaFree(v->d_sig);
     cudaFree(v->d_offsets);
     cudaFree(v->d_bytes);
     delete v;
@@ -301,6 +319,8 @@ void wg_ctx_free(wg_ctx *c) {
     for (GrammarSlot &s : c->slots) {
         cudaFree(s.d_table);
         cudaFree(s.d_cls);
+        cudaFree(s.d_first_ok);
+        cudaFree(s.d_leaves);
     }
     delete c;
 }
@@ -318,7 +338,7 @@ int32_t wg_ctx_add_grammar(wg_ctx *c, const wg_grammar *g, int32_t *grammar_id) 
     }
     if (c->slots.size() >= 65535) return WG_ERR_CAPACITY;
     const bool wide = g->n_states > 65535;
-    GrammarSlot slot{g->hash, g->table, g->n_states, g->n_classes, nullptr, nullptr};
+    GrammarSlot slot{g->hash, g->table, g->n_states, g->n_classes, nullptr, nullptr, nullptr, nullptr};
     const size_t n = g->table.size();
     if (wide) {
         WG_CUDA(cudaMalloc(&slot.d_table, n * sizeof(uint32_t)));
@@ -331,7 +351,29 @@ int32_t wg_ctx_add_grammar(wg_ctx *c, const wg_grammar *g, int32_t *grammar_id) 
     }
     WG_CUDA(cudaMalloc(&slot.d_cls, 256));
     WG_CUDA(cudaMemcpy(slot.d_cls, g->byte_class, 256, cudaMemcpyHostToDevice));
-    GrammarDev gd{slot.d_table, static_cast<const uint8_t *>(slot.d_cls), g->n_states,
+    // per state: the bytes that keep it alive, and (folded mod 64) the bytes that leave it
+    {
+        const int32_t S = g->n_states, C = g->n_classes;
+        std::vector<uint32_t> first_ok((size_t)S * 8, 0u);
+        std::vector<unsigned long long> leaves(S, 0ull);
+        for (int32_t st = 1; st < S; ++st) {
+            const int32_t *row = &g->table[(size_t)st * C];
+            for (int b = 0; b < 256; ++b) {
+                const int32_t to = row[g->byte_class[b]];
+                if (to != 0) first_ok[(size_t)st * 8 + (b >> 5)] |= 1u << (b & 31);
+                if (to != st) leaves[st] |= 1ull << (b & 63);
+            }
+        }
+        WG_CUDA(cudaMalloc(&slot.d_first_ok, first_ok.size() * sizeof(uint32_t)));
+        WG_CUDA(cudaMemcpy(slot.d_first_ok, first_ok.data(), first_ok.size() * sizeof(uint32_t),
+                           cudaMemcpyHostToDevice));
+        WG_CUDA(cudaMalloc(&slot.d_leaves, leaves.size() * sizeof(unsigned long long)));
+        WG_CUDA(cudaMemcpy(slot.d_leaves, leaves.data(), leaves.size() * sizeof(unsigned long long),
+                           cudaMemcpyHostToDevice));
+    }
+    GrammarDev gd{slot.d_table, static_cast<const uint8_t *>(slot.d_cls),
+                  static_cast<const uint32_t *>(slot.d_first_ok),
+                  static_cast<const unsigned long long *>(slot.d_leaves), g->n_states,
                   g->n_classes, g->start, g->done, g->eos_class, wide ? 1 : 0};
     const int32_t id = (int32_t)c->slots.size();
     if (id >= c->grammar_cap) {  // grow the registry; queued kernels still read the old one
@@ -397,16 +439,19 @@ namespace {
 int32_t launch_build(wg_ctx *c, const BuildWork &work, int max_entries, cudaStream_t st,
                      bool pdl = false) {
     const VocabDev &v = c->vocab->dev;
-    const long long n_chunks = ((long long)v.W * 32 + BUILD_CHUNK - 1) / BUILD_CHUNK;
+    // few masks: small chunks so that one mask still spreads over many blocks
+    BuildWork w = work;
+    w.chunk = max_entries <= 32 ? 2048 : BUILD_CHUNK_MAX;
+    const long long n_chunks = ((long long)v.W * 32 + w.chunk - 1) / w.chunk;
     long long items = (long long)max_entries * n_chunks;
     long long grid = (long long)sm_count() * 8;  // 8 resident blocks of 256 threads per SM
     if (items < grid) grid = items;
     if (grid < 1) grid = 1;
     if (pdl)
         WG_CUDA(launch_pdl(build_masks_kernel, dim3((unsigned)grid), dim3(BUILD_THREADS), st, v,
-                           c->dev, work));
+                           c->dev, w));
     else
-        build_masks_kernel<<<(unsigned)grid, BUILD_THREADS, 0, st>>>(v, c->dev, work);
+        build_masks_kernel<<<(unsigned)grid, BUILD_THREADS, 0, st>>>(v, c->dev, w);
     WG_LAUNCHED();
     return WG_OK;
 }
@@ -415,15 +460,19 @@ bool rows_aligned(const void *p, int64_t stride_elems, size_t elem) {
     return ((uintptr_t)p % 16 == 0) && ((stride_elems * (int64_t)elem) % 16 == 0);
 }
 
-// Grid of the apply kernels, (blocks per row, B), and the spans each block handles: enough
-// blocks to fill the machine a few times over, at least 8 spans (16 KB of bf16) per block.
+// Grid of the apply kernels, (blocks per row, B), and the spans each block handles: every
+// warp of a block takes 1, 2 or 4 spans of 1024 tokens; the smaller counts are used while the
+// grid would otherwise not cover the machine about twice.
 dim3 apply_grid(ApplyArgs &a) {
     const int n_spans = (a.W + 31) / 32;
-    int blocks_per_row = (sm_count() * 16 + a.B - 1) / a.B;
-    if (blocks_per_row > (n_spans + 7) / 8) blocks_per_row = (n_spans + 7) / 8;
-    if (blocks_per_row < 1) blocks_per_row = 1;
-    a.spans_per_block = (n_spans + blocks_per_row - 1) / blocks_per_row;
-    blocks_per_row = (n_spans + a.spans_per_block - 1) / a.spans_per_block;
+    int per_warp = APPLY_SPANS_PER_WARP;
+    while (per_warp > 1 &&
+           (long long)a.B * ((n_spans + APPLY_WARPS * per_warp - 1) / (APPLY_WARPS * per_warp)) <
+               2LL * sm_count())
+        per_warp >>= 1;
+    a.spans_per_block = APPLY_WARPS * per_warp;
+    if (const char *e = getenv("WG_TUNE_SPANS")) { int v = atoi(e); if (v > 0 && v <= APPLY_WARPS * APPLY_SPANS_PER_WARP) a.spans_per_block = v; }
+    const int blocks_per_row = (n_spans + a.spans_per_block - 1) / a.spans_per_block;
     return dim3((unsigned)blocks_per_row, (unsigned)a.B);
 }
 
@@ -481,12 +530,12 @@ int32_t wg_build_masks(wg_ctx *c, const int32_t *gid, const int32_t *sid, int32_
     if (row_stride_words < W || (flags & ~(uint32_t)WG_NO_CACHE)) return WG_ERR_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (flags & WG_NO_CACHE) {
-        BuildWork work{gid, sid, nullptr, bitmask, row_stride_words, nullptr, B};
+        BuildWork work{gid, sid, nullptr, bitmask, row_stride_words, nullptr, B, 0};
         return launch_build(c, work, B, st);
     }
     cache_lookup_insert_kernel<<<1, 1024, 0, st>>>(c->dev, gid, sid, B, bitmask, row_stride_words);
     WG_LAUNCHED();
-    BuildWork work{c->dev.bl_gid, c->dev.bl_sid, c->dev.bl_dst, nullptr, 0, c->dev.bl_count, 0};
+    BuildWork work{c->dev.bl_gid, c->dev.bl_sid, c->dev.bl_dst, nullptr, 0, c->dev.bl_count, 0, 0};
     int32_t rc = launch_build(c, work, B, st);
     if (rc != WG_OK) return rc;
     dim3 grid((unsigned)((W + 1023) / 1024), (unsigned)B);
@@ -604,13 +653,13 @@ int32_t wg_decode_step(wg_ctx *c, const int32_t *gid, int32_t *sid, int32_t B, v
         // rows have no pool row; the packed maxima were left at zero by the last advance
         WG_CUDA(launch_pdl(reset_rows_kernel, dim3((B + 255) / 256), dim3(256), st, c->dev, B));
         WG_LAUNCHED();
-        BuildWork work{gid, sid, nullptr, bitmask, mask_stride_words, nullptr, B};
+        BuildWork work{gid, sid, nullptr, bitmask, mask_stride_words, nullptr, B, 0};
         rc = launch_build(c, work, B, st, true);
     } else {
         WG_CUDA(launch_pdl(cache_lookup_insert_kernel, dim3(1), dim3(1024), st, c->dev, gid, sid, B,
                            bitmask, mask_stride_words));
         WG_LAUNCHED();
-        BuildWork work{c->dev.bl_gid, c->dev.bl_sid, c->dev.bl_dst, nullptr, 0, c->dev.bl_count, 0};
+        BuildWork work{c->dev.bl_gid, c->dev.bl_sid, c->dev.bl_dst, nullptr, 0, c->dev.bl_count, 0, 0};
         rc = launch_build(c, work, B, st, true);
     }
     if (rc != WG_OK) return rc;
@@ -689,7 +738,7 @@ int32_t wg_cache_prewarm(wg_ctx *c, int32_t grammar_id, void *stream) {
         cache_lookup_insert_kernel<<<1, 1024, 0, st>>>(c->dev, c->d_stage_gid, c->d_stage_sid, n,
                                                        nullptr, 0);
         WG_LAUNCHED();
-        BuildWork work{c->dev.bl_gid, c->dev.bl_sid, c->dev.bl_dst, nullptr, 0, c->dev.bl_count, 0};
+        BuildWork work{c->dev.bl_gid, c->dev.bl_sid, c->dev.bl_dst, nullptr, 0, c->dev.bl_count, 0, 0};
         rc = launch_build(c, work, n, st);
         if (rc != WG_OK) return rc;
     }

@@ -14,12 +14,17 @@
 struct GrammarDev {
     const void *table;          // [n_states][n_classes] of uint16_t (wide == 0) or uint32_t
     const uint8_t *byte_class;  // [256]
+    const uint32_t *first_ok;   // [n_states][8] bit b: byte b does not lead to DEAD
+    const unsigned long long *leaves;  // [n_states] OR of 1 << (b & 63) over bytes b that
+                                       // lead anywhere but back to the state itself
     int32_t n_states, n_classes, start, done, eos_class, wide;
 };
 
 struct VocabDev {
     const uint4 *rec;         // [V] first 16 bytes of every token, zero padded
     const uint8_t *len;       // [V] min(length, 255)
+    const uint32_t *meta;     // [V] min(length, 255) | first byte << 8
+    const unsigned long long *sig;  // [V] OR of 1 << (b & 63) over ALL bytes b of the token
     const uint32_t *offsets;  // [V + 1] CSR, for tokens longer than the record
     const uint8_t *bytes;
     int32_t V, W, eos_id;
@@ -89,12 +94,21 @@ __device__ __forceinline__ uint32_t walk_token(const VocabDev &v, const T *__res
 }
 
 // ---------------------------------------------------------------------------------------
-// K1: mask build.  One thread per token, 32 consecutive tokens per warp, one ballot per word.
-// Work item = (mask m, chunk of BUILD_CHUNK tokens); a fixed-size grid strides over the items
-// so that a launch with nothing to build costs a few empty blocks.
+// K1: mask build.  Work item = (mask m, chunk of tokens); a fixed-size grid strides over the
+// items, so a launch with nothing to build costs a few empty blocks.
+//
+// Most tokens are decided without walking the table.  Per token the vocabulary holds its
+// first byte and a 64-bit signature (which byte values, folded mod 64, occur in it); per
+// state the grammar holds the set of bytes that do not kill it and the folded set of bytes
+// that LEAVE it.  Then, in id order, one thread per token:
+//   first byte kills the state            -> not allowed          (literal states: ~all tokens)
+//   no byte of the token can leave state  -> allowed              (free-text states: ~all tokens)
+//   otherwise                             -> queued in shared memory
+// and the queue is walked densely afterwards (no lane idles next to a walking lane).  The
+// bits of a chunk are assembled in shared memory and stored as whole words.
 // ---------------------------------------------------------------------------------------
 constexpr int BUILD_THREADS = 256;
-constexpr int BUILD_CHUNK = 2048;
+constexpr int BUILD_CHUNK_MAX = 8192;  // tokens per work item (the launch picks 2048 or 8192)
 
 struct BuildWork {
     const int32_t *gid, *sid;   // per entry
@@ -103,36 +117,29 @@ struct BuildWork {
     int64_t dst_stride;
     const int32_t *count_ptr;   // number of entries on the device, or NULL: use count
     int32_t count;
+    int32_t chunk;              // tokens per work item: a multiple of 32, <= BUILD_CHUNK_MAX
 };
-
-template <typename T>
-__device__ __forceinline__ void build_chunk(const VocabDev &v, const GrammarDev &g,
-                                            const uint8_t *cls, uint32_t s0, int t_begin,
-                                            uint32_t *__restrict__ dst) {
-    const T *tab = static_cast<const T *>(g.table);
-    const int C = g.n_classes;
-    const int t_end = min(t_begin + BUILD_CHUNK, v.W * 32);
-    for (int t = t_begin + (int)threadIdx.x; t < t_end; t += BUILD_THREADS) {
-        bool alive = false;
-        if (t < v.V && s0 != 0) alive = walk_token<T>(v, tab, C, g.eos_class, cls, s0, t) != 0;
-        const uint32_t word = __ballot_sync(0xFFFFFFFFu, alive);
-        if ((threadIdx.x & 31) == 0) dst[t >> 5] = word;
-    }
-}
 
 __global__ void __launch_bounds__(BUILD_THREADS)
 build_masks_kernel(VocabDev v, CtxDev ctx, BuildWork work) {
     __shared__ uint8_t cls[256];
     __shared__ int cls_gid;
+    __shared__ uint32_t first_ok[8];
+    __shared__ uint32_t words[BUILD_CHUNK_MAX / 32];
+    __shared__ uint16_t todo[BUILD_CHUNK_MAX];
+    __shared__ int n_todo;
     pdl_enter();
     if (threadIdx.x == 0) cls_gid = -1;
     __syncthreads();
+    const int lane = threadIdx.x & 31;
     const int n_entries = work.count_ptr ? *work.count_ptr : work.count;
-    const int n_chunks = (v.W * 32 + BUILD_CHUNK - 1) / BUILD_CHUNK;
+    const int n_tok = v.W * 32;
+    const int n_chunks = (n_tok + work.chunk - 1) / work.chunk;
     const long long n_items = (long long)n_entries * n_chunks;
     for (long long item = blockIdx.x; item < n_items; item += gridDim.x) {
         const int m = (int)(item / n_chunks);
-        const int chunk = (int)(item % n_chunks);
+        const int t_begin = (int)(item % n_chunks) * work.chunk;
+        const int t_end = min(t_begin + work.chunk, n_tok);
         const int gid = work.gid[m];
         uint32_t s0 = (uint32_t)work.sid[m];
         uint32_t *dst = work.dst_list ? work.dst_list[m] : work.dst_base + (int64_t)m * work.dst_stride;
@@ -140,18 +147,61 @@ build_masks_kernel(VocabDev v, CtxDev ctx, BuildWork work) {
         GrammarDev g = {};
         if (known) g = ctx.grammars[gid];
         if (!known || s0 >= (uint32_t)g.n_states) s0 = 0;  // unknown state: an all-zero row
-        if (known && cls_gid != gid) {
-            __syncthreads();
-            cls[threadIdx.x] = g.byte_class[threadIdx.x];
-            if (threadIdx.x == 0) cls_gid = gid;
-            __syncthreads();
-        }
-        if (chunk == 0 && threadIdx.x == 0) {
+        if (t_begin == 0 && threadIdx.x == 0) {
             atomicAdd(&ctx.stats[ST_BUILT], 1ull);
             if (s0 == 0 && work.sid[m] != 0) atomicAdd(&ctx.stats[ST_BAD_STATE], 1ull);
         }
-        if (g.wide) build_chunk<uint32_t>(v, g, cls, s0, chunk * BUILD_CHUNK, dst);
-        else build_chunk<uint16_t>(v, g, cls, s0, chunk * BUILD_CHUNK, dst);
+        __syncthreads();  // the previous item is done with the shared arrays
+        if (known && cls_gid != gid) cls[threadIdx.x] = g.byte_class[threadIdx.x];
+        if (threadIdx.x < 8) first_ok[threadIdx.x] = s0 ? g.first_ok[(size_t)s0 * 8 + threadIdx.x] : 0u;
+        if (threadIdx.x == 0) n_todo = 0;
+        const unsigned long long leaves = s0 ? g.leaves[s0] : 0ull;
+        uint32_t eos_next = 0;
+        if (s0) eos_next = g.wide ? static_cast<const uint32_t *>(g.table)[(size_t)s0 * g.n_classes + g.eos_class]
+                                  : static_cast<const uint16_t *>(g.table)[(size_t)s0 * g.n_classes + g.eos_class];
+        __syncthreads();
+        if (threadIdx.x == 0 && known) cls_gid = gid;  // read again only after the next barrier
+        // phase 1: decide or queue, 32 consecutive tokens per warp and round
+        for (int t = t_begin + (int)threadIdx.x; t < t_end; t += BUILD_THREADS) {
+            bool alive = false, walk = false;
+            if (t < v.V && s0 != 0) {
+                if (t == v.eos_id) {
+                    alive = eos_next != 0;
+                } else {
+                    const uint32_t mt = __ldg(&v.meta[t]);
+                    const uint32_t fb = (mt >> 8) & 0xFFu;
+                    if ((mt & 0xFFu) != 0 && ((first_ok[fb >> 5] >> (fb & 31)) & 1u)) {
+                        if ((__ldg(&v.sig[t]) & leaves) == 0ull) alive = true;
+                        else walk = true;
+                    }
+                }
+            }
+            const uint32_t word = __ballot_sync(0xFFFFFFFFu, alive);
+            const uint32_t queue = __ballot_sync(0xFFFFFFFFu, walk);
+            if (lane == 0) words[(t - t_begin) >> 5] = word;
+            if (queue) {
+                int base = 0;
+                if (lane == 0) base = atomicAdd(&n_todo, __popc(queue));
+                base = __shfl_sync(0xFFFFFFFFu, base, 0);
+                if (walk) todo[base + __popc(queue & ((1u << lane) - 1))] = (uint16_t)(t - t_begin);
+            }
+        }
+        __syncthreads();
+        // phase 2: walk the queued tokens, one per thread
+        const int n = n_todo;
+        for (int i = threadIdx.x; i < n; i += BUILD_THREADS) {
+            const int rel = todo[i];
+            const uint32_t end = g.wide
+                ? walk_token<uint32_t>(v, static_cast<const uint32_t *>(g.table), g.n_classes,
+                                       g.eos_class, cls, s0, t_begin + rel)
+                : walk_token<uint16_t>(v, static_cast<const uint16_t *>(g.table), g.n_classes,
+                                       g.eos_class, cls, s0, t_begin + rel);
+            if (end != 0) atomicOr(&words[rel >> 5], 1u << (rel & 31));
+        }
+        __syncthreads();
+        // phase 3: whole words out
+        for (int w = threadIdx.x; w < (t_end - t_begin) >> 5; w += BUILD_THREADS)
+            dst[(t_begin >> 5) + w] = words[w];
     }
 }
 
@@ -331,6 +381,7 @@ template <> struct ElemTraits<uint32_t> {  // fp32
 
 constexpr int APPLY_THREADS = 256;
 constexpr int APPLY_WARPS = APPLY_THREADS / 32;
+constexpr int APPLY_SPANS_PER_WARP = 4;  // a block covers at most 8 * 4 spans = 32768 tokens
 
 struct ApplyArgs {
     void *logits;
@@ -426,13 +477,24 @@ apply_mask_kernel(ApplyArgs a, CtxDev ctx, unsigned long long *argkey) {
     const int full_chunks = a.V / EPC;  // chunks that lie wholly inside the row
     LaneBest best{__uint_as_float(0x7FC00000u), -1};
 
-    for (int span = span_begin + warp; span < span_end; span += APPLY_WARPS) {
-        const int word0 = span * 32;
-        uint32_t my_word = 0;
-        if (word0 + lane < a.W) {
-            my_word = mrow[word0 + lane];
-            if (copy_out) a.bitmask_out[(int64_t)r * a.mask_stride + word0 + lane] = my_word;
+    // The mask words of every span this warp will handle are fetched first, so their L2
+    // latency is paid once and not once per span (the spans themselves are store streams).
+    uint32_t words[APPLY_SPANS_PER_WARP];
+#pragma unroll
+    for (int k = 0; k < APPLY_SPANS_PER_WARP; ++k) {
+        const int w = (span_begin + warp + k * APPLY_WARPS) * 32 + lane;
+        words[k] = 0;
+        if (span_begin + warp + k * APPLY_WARPS < span_end && w < a.W) {
+            words[k] = mrow[w];
+            if (copy_out) a.bitmask_out[(int64_t)r * a.mask_stride + w] = words[k];
         }
+    }
+#pragma unroll
+    for (int k = 0; k < APPLY_SPANS_PER_WARP; ++k) {
+        const int span = span_begin + warp + k * APPLY_WARPS;
+        if (span >= span_end) break;
+        const int word0 = span * 32;
+        const uint32_t my_word = words[k];
         const int chunk0 = word0 * CHUNKS_PER_WORD;
 #pragma unroll
         for (int p0 = 0; p0 < PASSES; p0 += GROUP) {

@@ -172,12 +172,16 @@ class Sim:
         self.seed, self.steer = seed, steer
         self.bonus = has_structural_byte(vocab)
         self.delays = delays or [0] * self.B
+        # a row that starts one step late sits in DONE first: it emits EOS and restarts
+        late = [d > 0 for d in self.delays]
         # checker side
-        self.cursors = [self.trees[g].start() for g in self.row_grammar]
+        self.cursors = [oracle.DONE if late[r] else self.trees[g].start()
+                        for r, g in enumerate(self.row_grammar)]
         # library side
         self.d_gid = to_dev(torch, np.array([self.gids[g] for g in self.row_grammar], np.int32))
-        self.d_sid = to_dev(torch, np.array([self.grams[g].start_state for g in self.row_grammar],
-                                            np.int32))
+        self.d_sid = to_dev(torch, np.array(
+            [self.grams[g].done_state if late[r] else self.grams[g].start_state
+             for r, g in enumerate(self.row_grammar)], np.int32))
         self.h_sid = self.d_sid.cpu().numpy().copy()
         self.W = self.dv.W
         self.d_mask = torch.zeros((self.B, self.W), dtype=torch.int32, device="cuda")
@@ -187,14 +191,21 @@ class Sim:
         self.visited = set()
 
     def logits(self):
-        return make_logits(self.B, self.vocab.size, self.dtype, [self.seed, self.B], self.step_no,
-                           self.bonus, self.steer)
+        x = make_logits(self.B, self.vocab.size, self.dtype, [self.seed, self.B], self.step_no,
+                        self.bonus, self.steer)
+        if any(self.delays) and self.step_no > 0:
+            # a late row sees what the row before it saw one step earlier
+            prev = make_logits(self.B, self.vocab.size, self.dtype, [self.seed, self.B],
+                               self.step_no - 1, self.bonus, self.steer)
+            for r, d in enumerate(self.delays):
+                if d > 0:
+                    x[r] = prev[r - 1]
+        return x
 
     def step(self, check_rows=None, fused=True):
         wg, torch, vocab = self.wg, self.torch, self.vocab
         rows = range(self.B) if check_rows is None else check_rows
         host = self.logits()
-        active = [r for r in range(self.B) if self.delays[r] <= self.step_no]
         # ---- checker: mask -> apply -> argmax -> advance on the checked rows
         trees = [self.trees[self.row_grammar[r]] for r in rows]
         want_mask = oracle.masks(trees, vocab, [self.cursors[r] for r in rows], n_threads=8)
