@@ -73,7 +73,7 @@ int32_t dev_alloc(T **p, size_t n) {
 struct wg_vocab {
     VocabDev dev{};
     void *d_rec = nullptr, *d_len = nullptr, *d_offsets = nullptr, *d_bytes = nullptr;
-    void *d_meta = nullptr, *d_sig = nullptr;
+    void *d_first_mask = nullptr, *d_fold_mask = nullptr, *d_valid_mask = nullptr;
     int device = 0;
 };
 
@@ -151,16 +151,21 @@ int32_t wg_load_vocab(const uint32_t *offsets, const uint8_t *bytes, int32_t V, 
     if (total > 0 && !bytes) return WG_ERR_ARG;
 
     std::vector<uint8_t> rec((size_t)V * WG_REC_BYTES, 0), len(V, 0);
-    std::vector<uint32_t> meta(V, 0);
-    std::vector<unsigned long long> sig(V, 0ull);
+    // V-bit masks used by the build kernel: starts-with-byte (256), contains-a-byte-folding-to
+    // (64), has-any-byte (1); W words each
+    const size_t W = ((size_t)V + 31) / 32;
+    std::vector<uint32_t> first_mask(256 * W, 0u), fold_mask(64 * W, 0u), valid_mask(W, 0u);
     for (int32_t t = 0; t < V; ++t) {
         const uint32_t n = (t == eos_id) ? 0u : offsets[t + 1] - offsets[t];
         len[t] = (uint8_t)(n > 255u ? 255u : n);
-        if (n) memcpy(&rec[(size_t)t * WG_REC_BYTES], bytes + offsets[t], n < WG_REC_BYTES ? n : WG_REC_BYTES);
-        unsigned long long folded = 0ull;  // which byte values (mod 64) occur anywhere in the token
-        for (uint32_t i = 0; i < n; ++i) folded |= 1ull << (bytes[offsets[t] + i] & 63);
-        sig[t] = folded;
-        meta[t] = (uint32_t)len[t] | (n ? (uint32_t)bytes[offsets[t]] << 8 : 0u);
+        if (!n) continue;
+        const uint8_t *b = bytes + offsets[t];
+        memcpy(&rec[(size_t)t * WG_REC_BYTES], b, n < WG_REC_BYTES ? n : WG_REC_BYTES);
+        const uint32_t bit = 1u << (t & 31);
+        const size_t w = (size_t)t >> 5;
+        valid_mask[w] |= bit;
+        first_mask[(size_t)b[0] * W + w] |= bit;
+        for (uint32_t i = 0; i < n; ++i) fold_mask[(size_t)(b[i] & 63) * W + w] |= bit;
     }
     wg_vocab *v = new (std::nothrow) wg_vocab();
     if (!v) return WG_ERR_ARG;
@@ -168,16 +173,19 @@ int32_t wg_load_vocab(const uint32_t *offsets, const uint8_t *bytes, int32_t V, 
     if (cudaGetDevice(&v->device) != cudaSuccess) return fail(WG_ERR_CUDA);
     if (cudaMalloc(&v->d_rec, rec.size()) != cudaSuccess ||
         cudaMalloc(&v->d_len, len.size()) != cudaSuccess ||
-        cudaMalloc(&v->d_meta, meta.size() * sizeof(uint32_t)) != cudaSuccess ||
-        cudaMalloc(&v->d_sig, sig.size() * sizeof(unsigned long long)) != cudaSuccess ||
+        cudaMalloc(&v->d_first_mask, first_mask.size() * sizeof(uint32_t)) != cudaSuccess ||
+        cudaMalloc(&v->d_fold_mask, fold_mask.size() * sizeof(uint32_t)) != cudaSuccess ||
+        cudaMalloc(&v->d_valid_mask, valid_mask.size() * sizeof(uint32_t)) != cudaSuccess ||
         cudaMalloc(&v->d_offsets, sizeof(uint32_t) * ((size_t)V + 1)) != cudaSuccess ||
         cudaMalloc(&v->d_bytes, total ? total : 1) != cudaSuccess)
         return fail(WG_ERR_CUDA);
     if (cudaMemcpy(v->d_rec, rec.data(), rec.size(), cudaMemcpyHostToDevice) != cudaSuccess ||
         cudaMemcpy(v->d_len, len.data(), len.size(), cudaMemcpyHostToDevice) != cudaSuccess ||
-        cudaMemcpy(v->d_meta, meta.data(), meta.size() * sizeof(uint32_t),
+        cudaMemcpy(v->d_first_mask, first_mask.data(), first_mask.size() * sizeof(uint32_t),
                    cudaMemcpyHostToDevice) != cudaSuccess ||
-        cudaMemcpy(v->d_sig, sig.data(), sig.size() * sizeof(unsigned long long),
+        cudaMemcpy(v->d_fold_mask, fold_mask.data(), fold_mask.size() * sizeof(uint32_t),
+                   cudaMemcpyHostToDevice) != cudaSuccess ||
+        cudaMemcpy(v->d_valid_mask, valid_mask.data(), valid_mask.size() * sizeof(uint32_t),
                    cudaMemcpyHostToDevice) != cudaSuccess ||
         cudaMemcpy(v->d_offsets, offsets, sizeof(uint32_t) * ((size_t)V + 1),
                    cudaMemcpyHostToDevice) != cudaSuccess ||
@@ -185,8 +193,9 @@ int32_t wg_load_vocab(const uint32_t *offsets, const uint8_t *bytes, int32_t V, 
         return fail(WG_ERR_CUDA);
     v->dev.rec = static_cast<const uint4 *>(v->d_rec);
     v->dev.len = static_cast<const uint8_t *>(v->d_len);
-    v->dev.meta = static_cast<const uint32_t *>(v->d_meta);
-    v->dev.sig = static_cast<const unsigned long long *>(v->d_sig);
+    v->dev.first_mask = static_cast<const uint32_t *>(v->d_first_mask);
+    v->dev.fold_mask = static_cast<const uint32_t *>(v->d_fold_mask);
+    v->dev.valid_mask = static_cast<const uint32_t *>(v->d_valid_mask);
     v->dev.offsets = static_cast<const uint32_t *>(v->d_offsets);
     v->dev.bytes = static_cast<const uint8_t *>(v->d_bytes);
     v->dev.V = V;
@@ -200,8 +209,9 @@ void wg_vocab_free(wg_vocab *v) {
     if (!v) return;
     cudaFree(v->d_rec);
     cudaFree(v->d_len);
-    cudaFree(v->d_meta);
-    cudaFree(v->d_sig);
+    cudaFree(v->d_first_mask);
+    cudaFree(v->d_fold_mask);
+    cudaFree(v->d_valid_mask);
     cudaFree(v->d_offsets);
     cudaFree(v->d_bytes);
     delete v;

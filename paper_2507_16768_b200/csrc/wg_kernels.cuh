@@ -23,8 +23,9 @@ struct GrammarDev {
 struct VocabDev {
     const uint4 *rec;         // [V] first 16 bytes of every token, zero padded
     const uint8_t *len;       // [V] min(length, 255)
-    const uint32_t *meta;     // [V] min(length, 255) | first byte << 8
-    const unsigned long long *sig;  // [V] OR of 1 << (b & 63) over ALL bytes b of the token
+    const uint32_t *first_mask;  // [256][W] bit t: token t is non-empty and starts with byte b
+    const uint32_t *fold_mask;   // [64][W]  bit t: some byte b of token t has (b & 63) == c
+    const uint32_t *valid_mask;  // [W]      bit t: token t has at least one byte (EOS has none)
     const uint32_t *offsets;  // [V + 1] CSR, for tokens longer than the record
     const uint8_t *bytes;
     int32_t V, W, eos_id;
@@ -97,18 +98,20 @@ __device__ __forceinline__ uint32_t walk_token(const VocabDev &v, const T *__res
 // K1: mask build.  Work item = (mask m, chunk of tokens); a fixed-size grid strides over the
 // items, so a launch with nothing to build costs a few empty blocks.
 //
-// Most tokens are decided without walking the table.  Per token the vocabulary holds its
-// first byte and a 64-bit signature (which byte values, folded mod 64, occur in it); per
-// state the grammar holds the set of bytes that do not kill it and the folded set of bytes
-// that LEAVE it.  Then, in id order, one thread per token:
-//   first byte kills the state            -> not allowed          (literal states: ~all tokens)
-//   no byte of the token can leave state  -> allowed              (free-text states: ~all tokens)
-//   otherwise                             -> queued in shared memory
-// and the queue is walked densely afterwards (no lane idles next to a walking lane).  The
-// bits of a chunk are assembled in shared memory and stored as whole words.
+// Most tokens are decided 32 at a time, without walking the table.  The vocabulary holds
+// V-bit masks "token starts with byte b" (256 of them) and "token contains a byte that folds
+// to c = b & 63" (64 of them); a state holds the set of first bytes that do not kill it and
+// the folded set of bytes that LEAVE it.  For a word of 32 tokens:
+//   P = tokens whose first byte keeps the state alive   (OR of a few first-byte masks, or the
+//                                                         complement when most bytes are fine)
+//   Q = tokens that contain a byte which may leave       (OR of a few fold masks)
+//   P & ~Q  are allowed: every byte loops on the state   (free-text states: ~all tokens)
+//   ~P      are not allowed                              (literal states: ~all tokens)
+//   P & Q   are queued in shared memory and walked afterwards, densely, one per thread.
 // ---------------------------------------------------------------------------------------
 constexpr int BUILD_THREADS = 256;
 constexpr int BUILD_CHUNK_MAX = 8192;  // tokens per work item (the launch picks 2048 or 8192)
+constexpr int BUILD_MAX_FOLDS = 20;    // more leaving folds than this: queue every P token
 
 struct BuildWork {
     const int32_t *gid, *sid;   // per entry
@@ -120,11 +123,13 @@ struct BuildWork {
     int32_t chunk;              // tokens per work item: a multiple of 32, <= BUILD_CHUNK_MAX
 };
 
-__global__ void __launch_bounds__(BUILD_THREADS)
+__global__ void __launch_bounds__(BUILD_THREADS, 6)
 build_masks_kernel(VocabDev v, CtxDev ctx, BuildWork work) {
     __shared__ uint8_t cls[256];
     __shared__ int cls_gid;
-    __shared__ uint32_t first_ok[8];
+    __shared__ uint8_t first_list[128];  // first bytes to OR (or to exclude, when complemented)
+    __shared__ uint8_t fold_list[64];
+    __shared__ int n_first, n_fold;
     __shared__ uint32_t words[BUILD_CHUNK_MAX / 32];
     __shared__ uint16_t todo[BUILD_CHUNK_MAX];
     __shared__ int n_todo;
@@ -153,37 +158,61 @@ build_masks_kernel(VocabDev v, CtxDev ctx, BuildWork work) {
         }
         __syncthreads();  // the previous item is done with the shared arrays
         if (known && cls_gid != gid) cls[threadIdx.x] = g.byte_class[threadIdx.x];
-        if (threadIdx.x < 8) first_ok[threadIdx.x] = s0 ? g.first_ok[(size_t)s0 * 8 + threadIdx.x] : 0u;
-        if (threadIdx.x == 0) n_todo = 0;
+        if (threadIdx.x == 0) { n_todo = 0; n_first = 0; n_fold = 0; }
+        // the state's first-byte set; complemented when more than half of the bytes are fine
+        const uint32_t ok_word = s0 ? g.first_ok[(size_t)s0 * 8 + (threadIdx.x >> 5)] : 0u;
+        int n_ok = 0;
+        if (s0) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) n_ok += __popc(g.first_ok[(size_t)s0 * 8 + i]);
+        }
+        const bool complement = n_ok > 128;
         const unsigned long long leaves = s0 ? g.leaves[s0] : 0ull;
+        const bool queue_all = __popcll(leaves) > BUILD_MAX_FOLDS;
         uint32_t eos_next = 0;
         if (s0) eos_next = g.wide ? static_cast<const uint32_t *>(g.table)[(size_t)s0 * g.n_classes + g.eos_class]
                                   : static_cast<const uint16_t *>(g.table)[(size_t)s0 * g.n_classes + g.eos_class];
         __syncthreads();
         if (threadIdx.x == 0 && known) cls_gid = gid;  // read again only after the next barrier
-        // phase 1: decide or queue, 32 consecutive tokens per warp and round
-        for (int t = t_begin + (int)threadIdx.x; t < t_end; t += BUILD_THREADS) {
-            bool alive = false, walk = false;
-            if (t < v.V && s0 != 0) {
-                if (t == v.eos_id) {
-                    alive = eos_next != 0;
-                } else {
-                    const uint32_t mt = __ldg(&v.meta[t]);
-                    const uint32_t fb = (mt >> 8) & 0xFFu;
-                    if ((mt & 0xFFu) != 0 && ((first_ok[fb >> 5] >> (fb & 31)) & 1u)) {
-                        if ((__ldg(&v.sig[t]) & leaves) == 0ull) alive = true;
-                        else walk = true;
-                    }
-                }
+        {
+            const bool is_ok = (ok_word >> lane) & 1u;   // thread b looks at byte b
+            if (is_ok != complement) first_list[atomicAdd(&n_first, 1)] = (uint8_t)threadIdx.x;
+            if (threadIdx.x < 64 && !queue_all && ((leaves >> threadIdx.x) & 1ull))
+                fold_list[atomicAdd(&n_fold, 1)] = (uint8_t)threadIdx.x;
+        }
+        __syncthreads();
+        // phase 1: one word of 32 tokens per thread
+        const int n_words = (t_end - t_begin) >> 5;
+        const int nf = n_first, nq = n_fold;
+        for (int wl = threadIdx.x; wl < ((n_words + 31) & ~31); wl += BUILD_THREADS) {
+            uint32_t alive = 0, queue = 0;
+            const int w = (t_begin >> 5) + wl;
+            if (wl < n_words && s0 != 0) {
+                uint32_t p = 0;
+                for (int i = 0; i < nf; ++i) p |= __ldg(&v.first_mask[(size_t)first_list[i] * v.W + w]);
+                if (complement) p = __ldg(&v.valid_mask[w]) & ~p;
+                uint32_t q = queue_all ? 0xFFFFFFFFu : 0u;
+                for (int i = 0; i < nq; ++i) q |= __ldg(&v.fold_mask[(size_t)fold_list[i] * v.W + w]);
+                alive = p & ~q;
+                queue = p & q;
+                if ((v.eos_id >> 5) == w && eos_next != 0) alive |= 1u << (v.eos_id & 31);
             }
-            const uint32_t word = __ballot_sync(0xFFFFFFFFu, alive);
-            const uint32_t queue = __ballot_sync(0xFFFFFFFFu, walk);
-            if (lane == 0) words[(t - t_begin) >> 5] = word;
-            if (queue) {
-                int base = 0;
-                if (lane == 0) base = atomicAdd(&n_todo, __popc(queue));
-                base = __shfl_sync(0xFFFFFFFFu, base, 0);
-                if (walk) todo[base + __popc(queue & ((1u << lane) - 1))] = (uint16_t)(t - t_begin);
+            if (wl < n_words) words[wl] = alive;
+            // queue the undecided tokens: one shared-memory atomic per warp
+            const int mine = __popc(queue);
+            int before = mine;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int x = __shfl_up_sync(0xFFFFFFFFu, before, o);
+                if (lane >= o) before += x;
+            }
+            int base = 0;
+            if (lane == 31 && before > 0) base = atomicAdd(&n_todo, before);
+            base = __shfl_sync(0xFFFFFFFFu, base, 31) + before - mine;
+            while (queue) {
+                const int bit = __ffs(queue) - 1;
+                queue &= queue - 1;
+                todo[base++] = (uint16_t)(wl * 32 + bit);
             }
         }
         __syncthreads();
@@ -200,8 +229,8 @@ build_masks_kernel(VocabDev v, CtxDev ctx, BuildWork work) {
         }
         __syncthreads();
         // phase 3: whole words out
-        for (int w = threadIdx.x; w < (t_end - t_begin) >> 5; w += BUILD_THREADS)
-            dst[(t_begin >> 5) + w] = words[w];
+        for (int wl = threadIdx.x; wl < n_words; wl += BUILD_THREADS)
+            dst[(t_begin >> 5) + wl] = words[wl];
     }
 }
 
