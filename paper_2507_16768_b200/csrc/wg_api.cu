@@ -472,13 +472,13 @@ bool rows_aligned(const void *p, int64_t stride_elems, size_t elem) {
 
 // Grid of the apply kernels, (blocks per row, B), and the spans each block handles: every
 // warp of a block takes 1, 2 or 4 spans of 1024 tokens; the smaller counts are used while the
-// grid would otherwise not cover the machine about twice.
+// grid would otherwise hold fewer than about four waves of blocks (a short last wave costs).
 dim3 apply_grid(ApplyArgs &a) {
     const int n_spans = (a.W + 31) / 32;
     int per_warp = APPLY_SPANS_PER_WARP;
     while (per_warp > 1 &&
            (long long)a.B * ((n_spans + APPLY_WARPS * per_warp - 1) / (APPLY_WARPS * per_warp)) <
-               2LL * sm_count())
+               16LL * sm_count())
         per_warp >>= 1;
     a.spans_per_block = APPLY_WARPS * per_warp;
     if (const char *e = getenv("WG_TUNE_SPANS")) { int v = atoi(e); if (v > 0 && v <= APPLY_WARPS * APPLY_SPANS_PER_WARP) a.spans_per_block = v; }

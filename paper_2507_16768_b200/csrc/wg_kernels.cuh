@@ -518,38 +518,55 @@ apply_mask_kernel(ApplyArgs a, CtxDev ctx, unsigned long long *argkey) {
             if (copy_out) a.bitmask_out[(int64_t)r * a.mask_stride + w] = words[k];
         }
     }
+    // Sweep 1: every chunk whose bits are all clear is a pure store; chunks that will have to
+    // be read (mixed bits, or any allowed element when the argmax is wanted) are only
+    // prefetched into L2 here, so no warp waits on DRAM while its stores could be going out.
 #pragma unroll
     for (int k = 0; k < APPLY_SPANS_PER_WARP; ++k) {
         const int span = span_begin + warp + k * APPLY_WARPS;
         if (span >= span_end) break;
-        const int word0 = span * 32;
-        const uint32_t my_word = words[k];
-        const int chunk0 = word0 * CHUNKS_PER_WORD;
+        const int chunk0 = span * 32 * CHUNKS_PER_WORD;
+#pragma unroll
+        for (int p = 0; p < PASSES; ++p) {
+            const int c = p * 32 + lane;  // chunk index inside the span
+            const uint32_t word = __shfl_sync(0xFFFFFFFFu, words[k], c / CHUNKS_PER_WORD);
+            const uint32_t bits = (word >> (EPC * (c % CHUNKS_PER_WORD))) & FULL;
+            if (chunk0 + c >= full_chunks) continue;
+            uint4 *ptr = reinterpret_cast<uint4 *>(row) + chunk0 + c;
+            if (bits == 0) {
+                const uint32_t ninf = sizeof(E) == 2 ? NEG_INF_BF16X2 : NEG_INF_F32;
+                __stcs(ptr, make_uint4(ninf, ninf, ninf, ninf));
+            } else if (ARGMAX || bits != FULL) {
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr));
+            }
+        }
+    }
+    // Sweep 2: the chunks that need their old contents, a group of independent loads at a time.
+#pragma unroll
+    for (int k = 0; k < APPLY_SPANS_PER_WARP; ++k) {
+        const int span = span_begin + warp + k * APPLY_WARPS;
+        if (span >= span_end) break;
+        const int chunk0 = span * 32 * CHUNKS_PER_WORD;
+        // a span without a single allowed token has nothing left to do (uniform per warp)
+        if (__ballot_sync(0xFFFFFFFFu, words[k] != 0) == 0) continue;
 #pragma unroll
         for (int p0 = 0; p0 < PASSES; p0 += GROUP) {
-            // the independent loads of the group first, then patch / compare / store
             uint4 val[GROUP];
             uint32_t bits[GROUP];
 #pragma unroll
             for (int q = 0; q < GROUP; ++q) {
-                const int c = (p0 + q) * 32 + lane;  // chunk index inside the span
-                const uint32_t word = __shfl_sync(0xFFFFFFFFu, my_word, c / CHUNKS_PER_WORD);
+                const int c = (p0 + q) * 32 + lane;
+                const uint32_t word = __shfl_sync(0xFFFFFFFFu, words[k], c / CHUNKS_PER_WORD);
                 bits[q] = (word >> (EPC * (c % CHUNKS_PER_WORD))) & FULL;
-                if (chunk0 + c >= full_chunks) bits[q] = SKIP;
-                else if (bits[q] != 0 && (ARGMAX || bits[q] != FULL))
+                if (chunk0 + c >= full_chunks || bits[q] == 0 || (!ARGMAX && bits[q] == FULL))
+                    bits[q] = SKIP;
+                else
                     val[q] = __ldcs(reinterpret_cast<const uint4 *>(row) + chunk0 + c);
             }
 #pragma unroll
             for (int q = 0; q < GROUP; ++q) {
                 if (bits[q] == SKIP) continue;
                 const int chunk = chunk0 + (p0 + q) * 32 + lane;
-                uint4 *ptr = reinterpret_cast<uint4 *>(row) + chunk;
-                if (bits[q] == 0) {
-                    const uint32_t ninf = sizeof(E) == 2 ? NEG_INF_BF16X2 : NEG_INF_F32;
-                    __stcs(ptr, make_uint4(ninf, ninf, ninf, ninf));
-                    continue;
-                }
-                if (!ARGMAX && bits[q] == FULL) continue;
                 uint32_t w[4] = {val[q].x, val[q].y, val[q].z, val[q].w};
                 const int t0 = chunk * EPC;
                 if (sizeof(E) == 2) {
@@ -574,7 +591,8 @@ apply_mask_kernel(ApplyArgs a, CtxDev ctx, unsigned long long *argkey) {
                         }
                     }
                 }
-                if (bits[q] != FULL) __stcs(ptr, make_uint4(w[0], w[1], w[2], w[3]));
+                if (bits[q] != FULL)
+                    __stcs(reinterpret_cast<uint4 *>(row) + chunk, make_uint4(w[0], w[1], w[2], w[3]));
             }
         }
     }
