@@ -141,6 +141,33 @@ int32_t wg_compile_grammar(const wg_op_node *nodes, int32_t n_nodes, const int32
                            const uint8_t *data, int32_t n_data, int32_t root, wg_grammar **out);
 void wg_grammar_free(wg_grammar *grammar);
 
+/* Regular-expression front end (paper Section 3.2, "From Regular Expressions to Wait/Write
+ * Operator Composition"; the syntax-prior path of Section 4.1's "WGrammar (online)").
+ * Translates a pattern into an operator tree: classes and characters become Wait, literal runs
+ * Write, repetition and branching DoWhile / IfElse(Switch) / Sequence, followed by EOS.
+ * Dialect (bytes): literals, '.', escapes \d \w \s \D \W \S \n \t \r \f \v \0 \xHH
+ * and \<punctuation>, classes [a-z0-9_] and [^...], groups ( ) and (?: ), '|', and the
+ * quantifiers * + ? {m} {m,} {m,n} (n <= 64; a trailing lazy '?' is ignored).  '^' at the very
+ * start and '$' at the very end are accepted and mean nothing: the whole output must match.
+ * The operators decide on one symbol, so wherever the pattern chooses (stay in a repetition
+ * or leave it, which alternative) the candidate first symbols must not overlap, a repeated
+ * group must begin with a character, class or repeated class, and what follows a repetition
+ * must begin with one as well.  Anything else returns WG_ERR_GRAMMAR; wg_regex_error() then
+ * gives the reason (thread-local, valid until the next call on the thread).
+ *   pattern  host, `length` bytes, need not be NUL-terminated
+ * wg_compile_regex = wg_regex_to_optree + wg_compile_grammar.  The tree itself can be read
+ * back with wg_optree_sizes / wg_optree_copy (arrays as in wg_compile_grammar; any pointer of
+ * wg_optree_copy may be NULL to skip that array).  Free with wg_optree_free. */
+typedef struct wg_optree wg_optree;
+int32_t wg_regex_to_optree(const char *pattern, int32_t length, wg_optree **out);
+int32_t wg_optree_sizes(const wg_optree *tree, int32_t *n_nodes, int32_t *n_children,
+                        int32_t *n_sets, int32_t *n_data, int32_t *root);
+int32_t wg_optree_copy(const wg_optree *tree, wg_op_node *nodes, int32_t *children, uint32_t *sets,
+                       uint8_t *data);
+void wg_optree_free(wg_optree *tree);
+int32_t wg_compile_regex(const char *pattern, int32_t length, wg_grammar **out);
+const char *wg_regex_error(void);
+
 /* Host-side facts about a compiled grammar.  Any output pointer may be NULL.
  * content_hash identifies the table: two compilations with equal tables hash equally. */
 int32_t wg_grammar_info(const wg_grammar *grammar, int32_t *n_states, int32_t *start_state,

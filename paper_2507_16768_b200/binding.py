@@ -54,6 +54,13 @@ _SIGNATURES = {
     "wg_vocab_free": (None, [_vp]),
     "wg_compile_grammar": (_i32, [_vp, _i32, _vp, _i32, _vp, _i32, _vp, _i32, _i32, C.POINTER(_vp)]),
     "wg_grammar_free": (None, [_vp]),
+    "wg_regex_to_optree": (_i32, [C.c_char_p, _i32, C.POINTER(_vp)]),
+    "wg_optree_sizes": (_i32, [_vp, C.POINTER(_i32), C.POINTER(_i32), C.POINTER(_i32),
+                               C.POINTER(_i32), C.POINTER(_i32)]),
+    "wg_optree_copy": (_i32, [_vp, _vp, _vp, _vp, _vp]),
+    "wg_optree_free": (None, [_vp]),
+    "wg_compile_regex": (_i32, [C.c_char_p, _i32, C.POINTER(_vp)]),
+    "wg_regex_error": (C.c_char_p, []),
     "wg_grammar_info": (_i32, [_vp, C.POINTER(_i32), C.POINTER(_i32), C.POINTER(_i32),
                                C.POINTER(_i32), C.POINTER(C.c_uint64)]),
     "wg_grammar_step": (_i32, [_vp, _i32, _i32]),
@@ -151,25 +158,68 @@ class Vocab:
         self.close()
 
 
-class Grammar:
-    """wg_compile_grammar: lowers a flat operator tree to a byte-level table (host side)."""
+class RegexTree:
+    """The operator tree of a regular expression as flat arrays (wg_regex_to_optree)."""
 
-    def __init__(self, flat):
-        nodes = np.ascontiguousarray(flat.nodes, np.int32)
-        children = np.ascontiguousarray(flat.children, np.int32)
-        sets = np.ascontiguousarray(flat.sets, np.uint32)
-        data = np.ascontiguousarray(flat.data, np.uint8)
+    def __init__(self, pattern):
+        if isinstance(pattern, str):
+            pattern = pattern.encode("utf-8")
         h = _vp()
-        _check(_lib.wg_compile_grammar(_np_ptr(nodes), nodes.shape[0], _np_ptr(children),
-                                       children.shape[0], _np_ptr(sets), sets.shape[0],
-                                       _np_ptr(data), data.shape[0], int(flat.root), C.byref(h)),
-               "wg_compile_grammar")
+        rc = _lib.wg_regex_to_optree(pattern, len(pattern), C.byref(h))
+        if rc != WG_OK:
+            raise WgError(rc, "wg_regex_to_optree: " + _lib.wg_regex_error().decode())
+        try:
+            n = [_i32() for _ in range(5)]
+            _check(_lib.wg_optree_sizes(h, *[C.byref(x) for x in n]), "wg_optree_sizes")
+            self.nodes = np.zeros((n[0].value, 8), np.int32)
+            self.children = np.zeros(n[1].value, np.int32)
+            self.sets = np.zeros((n[2].value, 9), np.uint32)
+            self.data = np.zeros(n[3].value, np.uint8)
+            self.root = n[4].value
+            _check(_lib.wg_optree_copy(h, _np_ptr(self.nodes), _np_ptr(self.children),
+                                       _np_ptr(self.sets), _np_ptr(self.data)), "wg_optree_copy")
+        finally:
+            _lib.wg_optree_free(h)
+
+    @property
+    def n_nodes(self) -> int:
+        return int(self.nodes.shape[0])
+
+
+class Grammar:
+    """wg_compile_grammar: lowers a flat operator tree to a byte-level table (host side).
+
+    ``Grammar.from_regex(pattern)`` goes through wg_compile_regex instead.
+    """
+
+    def __init__(self, flat=None, _handle=None):
+        if _handle is None:
+            nodes = np.ascontiguousarray(flat.nodes, np.int32)
+            children = np.ascontiguousarray(flat.children, np.int32)
+            sets = np.ascontiguousarray(flat.sets, np.uint32)
+            data = np.ascontiguousarray(flat.data, np.uint8)
+            _handle = _vp()
+            _check(_lib.wg_compile_grammar(_np_ptr(nodes), nodes.shape[0], _np_ptr(children),
+                                           children.shape[0], _np_ptr(sets), sets.shape[0],
+                                           _np_ptr(data), data.shape[0], int(flat.root),
+                                           C.byref(_handle)), "wg_compile_grammar")
+        h = _handle
         self.handle = h
         n, s, d, c, hs = _i32(), _i32(), _i32(), _i32(), C.c_uint64()
         _check(_lib.wg_grammar_info(h, C.byref(n), C.byref(s), C.byref(d), C.byref(c), C.byref(hs)),
                "wg_grammar_info")
         self.n_states, self.start_state, self.done_state = n.value, s.value, d.value
         self.n_classes, self.content_hash = c.value, hs.value
+
+    @classmethod
+    def from_regex(cls, pattern) -> "Grammar":
+        if isinstance(pattern, str):
+            pattern = pattern.encode("utf-8")
+        h = _vp()
+        rc = _lib.wg_compile_regex(pattern, len(pattern), C.byref(h))
+        if rc != WG_OK:
+            raise WgError(rc, "wg_compile_regex: " + _lib.wg_regex_error().decode())
+        return cls(_handle=h)
 
     def step(self, state: int, symbol: int) -> int:
         return int(_lib.wg_grammar_step(self.handle, int(state), int(symbol)))

@@ -160,7 +160,7 @@ class Sim:
     def __init__(self, wg, torch, vocab, ops, row_grammar, dtype, cache_capacity, use_cache=True,
                  seed=0, steer=6.0, delays=None):
         self.wg, self.torch, self.vocab, self.dtype = wg, torch, vocab, dtype
-        self.flats = [flatten(op) for op in ops]
+        self.flats = [op if hasattr(op, "nodes") else flatten(op) for op in ops]
         self.trees = [oracle.Tree(f) for f in self.flats]
         self.grams = [wg.Grammar(f) for f in self.flats]
         self.dv = wg.Vocab(vocab.offsets, vocab.data, vocab.eos_id)
@@ -401,3 +401,20 @@ def test_host_argument_errors(wg, torch):
         wg.wg_build_masks(ctx, five[:4], five[:4], narrow)
     with pytest.raises(wg.WgError):
         ctx.cache_prewarm(3)                                       # unknown grammar id
+
+
+def test_trajectory_on_grammars_compiled_from_regular_expressions(wg, torch):
+    from wg_workloads.optree import FlatTree
+    patterns = [r"\[\d+(,\d+)*\]", r'\{"id": \d+, "tags": \[("[a-z]+"(, "[a-z]+")*)?\]\}',
+                r"(yes|no|maybe)( \w+)*\."]
+    flats = []
+    for pat in patterns:
+        t = wg.binding.RegexTree(pat)
+        flats.append(FlatTree(t.nodes, t.children, t.sets, t.data, t.root))
+    vocab = make_vocab(8192, seed=12)
+    rows = [0, 1, 2, 0, 1, 2, 1, 1]
+    sim = Sim(wg, torch, vocab, flats, rows, "fp32", cache_capacity=512, seed=8, steer=3.0)
+    for _ in range(40):
+        sim.step()
+    assert len(sim.visited) > 25
+    assert len({g for g, _ in sim.visited}) == 3
