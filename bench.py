@@ -29,6 +29,13 @@ import numpy as np  # noqa: E402
 
 from wg_workloads import BY_NAME, flatten, has_structural_byte, make_logits, make_vocab  # noqa: E402
 
+# dram__bytes_read.sum + dram__bytes_write.sum of ONE launch of the dominant kernel, from the ncu
+# capture summarised under profiles/ (same launch shape as the timed run).  Set an entry to None
+# when its kernel changes and the capture has not been redone.
+NCU_TRAFFIC_BYTES = {
+    "json_warm": 222.2e6,       # profiles/apply_mask_kernel_json_warm.md
+}
+
 METRIC = "masked logit rows/s (mask build+apply)"
 UNIT = "rows/s"
 FALLBACK_HBM_GBS = 6650.0
@@ -358,7 +365,8 @@ def run_ours(args, w, steer: float) -> None:
         achieved = algo_bytes / (apply_ms * 1e-3) / 1e9 if apply_ms > 0 else 0.0
         roofline = {"kernel": "apply_mask_kernel (gather + apply + argmax)", "bound": "hbm",
                     "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                    "peak_kind": f"of {peak_kind}", "traffic": None,
+                    "peak_kind": f"of {peak_kind}",
+                    "traffic": NCU_TRAFFIC_BYTES.get(w.name) if B == w.batch else None,
                     "algorithmic_bytes_per_launch": algo_bytes, "avg_launch_ms": apply_ms,
                     "timed_by": "CUDA events recorded by the library around the kernel, in a "
                                 "second pass over the same steps"}

@@ -2,7 +2,6 @@
 #include <atomic>
 #include <cstdio>
 #include <cstring>
-#include <cstdlib>
 #include <mutex>
 #include <new>
 #include <vector>
@@ -481,7 +480,6 @@ dim3 apply_grid(ApplyArgs &a) {
                16LL * sm_count())
         per_warp >>= 1;
     a.spans_per_block = APPLY_WARPS * per_warp;
-    if (const char *e = getenv("WG_TUNE_SPANS")) { int v = atoi(e); if (v > 0 && v <= APPLY_WARPS * APPLY_SPANS_PER_WARP) a.spans_per_block = v; }
     const int blocks_per_row = (n_spans + a.spans_per_block - 1) / a.spans_per_block;
     return dim3((unsigned)blocks_per_row, (unsigned)a.B);
 }

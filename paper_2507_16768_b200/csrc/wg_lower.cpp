@@ -218,29 +218,40 @@ int32_t wg_lower_tree(const wg_op_node *nodes, int32_t n_nodes, const int32_t *c
     }
     const int32_t S = (int32_t)order.size();
 
-    // symbol classes by partition refinement over the states' columns
+    // Symbol classes: two symbols share a class when they belong to exactly the same edge
+    // sets, which makes their columns equal in every state.  The refinement runs over the
+    // DISTINCT sets only (a few hundred even for tables with 10^5 states, where most states
+    // are one-byte steps of a literal).
     std::vector<int32_t> cls(WG_N_SYMBOLS, 0);
     int32_t n_cls = 1;
-    std::vector<int32_t> target(WG_N_SYMBOLS);
-    for (int32_t i = 0; i < S; ++i) {
-        const std::vector<Edge> &edges = lw.states[order[i]];
-        if (edges.empty()) continue;
-        for (int sym = 0; sym < WG_N_SYMBOLS; ++sym) {
-            int32_t t = 0;
-            for (const Edge &e : edges)
-                if (e.on.has(sym)) { t = new_id[e.to]; break; }
-            target[sym] = t;
+    {
+        struct SetHash {
+            size_t operator()(const SymSet &x) const {
+                uint64_t h = 0xCBF29CE484222325ull;
+                for (uint32_t w : x.w) h = (h ^ w) * 0x100000001B3ull;
+                return (size_t)h;
+            }
+        };
+        struct SetEq {
+            bool operator()(const SymSet &a, const SymSet &b) const {
+                return memcmp(a.w, b.w, sizeof(a.w)) == 0;
+            }
+        };
+        std::unordered_map<SymSet, int, SetHash, SetEq> seen;
+        std::vector<int32_t> renum;
+        for (int32_t i = 0; i < S; ++i) {
+            for (const Edge &e : lw.states[order[i]]) {
+                if (!seen.emplace(e.on, 0).second) continue;
+                renum.assign((size_t)n_cls * 2, -1);
+                int32_t n_next = 0;
+                for (int sym = 0; sym < WG_N_SYMBOLS; ++sym) {
+                    const int32_t key = cls[sym] * 2 + (e.on.has(sym) ? 1 : 0);
+                    if (renum[key] < 0) renum[key] = n_next++;
+                    cls[sym] = renum[key];
+                }
+                n_cls = n_next;
+            }
         }
-        std::unordered_map<uint64_t, int32_t> split;
-        std::vector<int32_t> next(WG_N_SYMBOLS);
-        int32_t n_next = 0;
-        for (int sym = 0; sym < WG_N_SYMBOLS; ++sym) {
-            uint64_t key = ((uint64_t)(uint32_t)cls[sym] << 32) | (uint32_t)target[sym];
-            auto it = split.find(key);
-            if (it == split.end()) it = split.emplace(key, n_next++).first;
-            next[sym] = it->second;
-        }
-        if (n_next != n_cls) { cls.swap(next); n_cls = n_next; }
     }
     // class ids in order of first appearance over the byte values, EOS last
     {

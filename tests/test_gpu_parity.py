@@ -418,3 +418,75 @@ def test_trajectory_on_grammars_compiled_from_regular_expressions(wg, torch):
         sim.step()
     assert len(sim.visited) > 25
     assert len({g for g, _ in sim.visited}) == 3
+
+
+def test_host_buffer_step_and_step_plan_equal_the_plain_step(wg, torch):
+    vocab = make_vocab(8192, seed=13)
+    flat = flatten(grammars.json_reference_lookup(doc_nodes=60))
+    g = wg.Grammar(flat)
+    dv = wg.Vocab(vocab.offsets, vocab.data, vocab.eos_id)
+    B, V = 6, vocab.size
+    results = []
+    for mode in ("plain", "plan", "host"):
+        ctx = wg.Context(dv, 256, B)
+        gid = torch.full((B,), ctx.add_grammar(g), dtype=torch.int32, device="cuda")
+        sid = torch.full((B,), g.start_state, dtype=torch.int32, device="cuda")
+        mask = torch.zeros((B, dv.W), dtype=torch.int32, device="cuda")
+        tok = torch.zeros(B, dtype=torch.int32, device="cuda")
+        status = torch.zeros(B, dtype=torch.int32, device="cuda")
+        plan = wg.StepPlan(ctx, gid, sid, mask, tok, status, wg.WG_RESTART_ON_DONE)
+        tok_host = torch.zeros(B, dtype=torch.int32).pin_memory()
+        trace = []
+        for step in range(25):
+            host = torch.from_numpy(make_logits(B, V, "fp32", [3, 1], step))
+            dl = host.cuda()
+            if mode == "plain":
+                wg.wg_decode_step(ctx, gid, sid, dl, mask, tok, status, wg.WG_RESTART_ON_DONE)
+            elif mode == "plan":
+                plan(dl)
+            else:
+                stage = torch.empty((B, V), dtype=torch.float32, device="cuda")
+                wg.wg_decode_step_host(ctx, gid, sid, host.pin_memory(), stage, mask, tok, tok_host,
+                                       status, wg.WG_RESTART_ON_DONE)
+                assert (tok_host == tok.cpu()).all()
+                dl = stage
+            trace.append((tok.cpu().numpy().copy(), sid.cpu().numpy().copy(),
+                          mask.cpu().numpy().copy(), dl.cpu().numpy().view(np.uint32).copy()))
+            assert (status == 0).all()
+        results.append(trace)
+    for a, b in zip(results[0], results[1]):
+        assert all((x == y).all() for x, y in zip(a, b))
+    for a, b in zip(results[0], results[2]):
+        assert all((x == y).all() for x, y in zip(a, b))
+
+
+def test_degenerate_vocabularies_and_full_batches(wg, torch):
+    # one-token vocabulary (the EOS token alone), very long tokens, a batch of exactly max_batch
+    lone = vocab_from_tokens([b""], eos_id=0)
+    g = wg.Grammar(flatten(Write(b"")))
+    dv = wg.Vocab(lone.offsets, lone.data, 0)
+    ctx = wg.Context(dv, 4, 3)
+    gid = torch.full((3,), ctx.add_grammar(g), dtype=torch.int32, device="cuda")
+    sid = torch.full((3,), g.start_state, dtype=torch.int32, device="cuda")
+    mask = torch.zeros((3, 1), dtype=torch.int32, device="cuda")
+    tok = torch.full((3,), 9, dtype=torch.int32, device="cuda")
+    logits = torch.zeros((3, 8), device="cuda")[:, :1]          # V = 1, rows 32 bytes apart
+    wg.wg_decode_step(ctx, gid, sid, logits, mask, tok)
+    assert mask.cpu().tolist() == [[1]] * 3 and tok.cpu().tolist() == [0] * 3
+    assert sid.cpu().tolist() == [g.done_state] * 3
+
+    long_tokens = [b"ab" * 200, b"ab" * 127 + b"a", b"ab" * 200 + b"c", b"", b"a" * 255, b"a" * 256,
+                   b"b" + b"a" * 300]
+    vocab = vocab_from_tokens(long_tokens, eos_id=3)
+    op = Sequence(Wait(SymSet(b"ab"), SymSet(b"c")), Write(b"!"))
+    tree = oracle.Tree(flatten(op))
+    g = wg.Grammar(flatten(op))
+    dv = wg.Vocab(vocab.offsets, vocab.data, vocab.eos_id)
+    ctx = wg.Context(dv, 0, 2)
+    out = torch.zeros((2, 1), dtype=torch.int32, device="cuda")
+    wg.wg_build_masks(ctx, torch.full((2,), ctx.add_grammar(g), dtype=torch.int32, device="cuda"),
+                      torch.tensor([g.start_state, g.step(g.start_state, ord("c"))],
+                                   dtype=torch.int32, device="cuda"), out, wg.WG_NO_CACHE)
+    want = oracle.masks([tree, tree], vocab, [tree.start(), tree.step(tree.start(), ord("c"))])
+    assert (out.cpu().numpy().view(np.uint32) == want).all()
+    assert want[0, 0] == 0b1110111 and want[1, 0] == 0
