@@ -75,7 +75,8 @@ enum {
     WG_OP_WRITE = 1,
     WG_OP_WAIT = 2,
     WG_OP_SWITCH = 3, /* IfElse and its k-way generalisation */
-    WG_OP_DOWHILE = 4
+    WG_OP_DOWHILE = 4,
+    WG_OP_WAIT_UNTIL = 5 /* a Wait whose wait "token" is a multi-byte string */
 };
 
 /* One node of a flattened operator tree.  Children, symbol sets and literal bytes live in
@@ -86,7 +87,11 @@ enum {
  *   WAIT      sets     = [allow, deny, wait],               children = [body or -1]
  *   SWITCH    sets     = [allow, deny, case_0 .. case_k-1], children = [body_0 .. body_k-1]
  *             (IfElse: case_0 = true_waits -> if_body, case_1 = false_waits -> else_body)
- *   DOWHILE   sets     = [allow, deny, true_waits, false_waits], children = [body or -1] */
+ *   DOWHILE   sets     = [allow, deny, true_waits, false_waits], children = [body or -1]
+ *   WAIT_UNTIL sets    = [allow, deny], data = the string waited for, children = [body or -1]
+ *             (paper Section 3.2: the waits of a Wait are tokens, e.g. a closing tag; at byte
+ *             level such a token is a string.  Accepts text over (allow \ deny) and the
+ *             string's own bytes up to and including the FIRST occurrence of the string.) */
 typedef struct wg_op_node {
     int32_t kind;
     int32_t n_child, child_off;
@@ -130,12 +135,13 @@ void wg_vocab_free(wg_vocab *vocab);
  * library walks token BYTES, so a literal may be produced by any tokens whose bytes spell it).
  * All pointers are host arrays in the layout described at wg_op_node.
  * Languages: Write = its literal; Wait = stay* w body (ends at the first wait symbol, paper
- * Section 6); Switch = stay* (s_i body_i); DoWhile = (body stay* t)* body stay* f; Sequence =
+ * Section 6); WaitUntil = text up to the first occurrence of its string, then body; Switch = stay* (s_i body_i); DoWhile = (body stay* t)* body stay* f; Sequence =
  * concatenation; stay = (allow \ deny) \ deciding symbols; an absent body is empty.  If no
  * set mentions EOS, the program is followed by one EOS.  After the program comes the DONE
  * state, which accepts EOS only and stays DONE.
  * Errors: WG_ERR_ARG for malformed arrays; WG_ERR_GRAMMAR for an empty deciding set,
- * deciding sets that overlap each other or the deny set, or a node used twice (not a tree). */
+ * deciding sets that overlap each other or the deny set, an empty or partly denied WaitUntil
+ * string, or a node used twice (not a tree). */
 int32_t wg_compile_grammar(const wg_op_node *nodes, int32_t n_nodes, const int32_t *children,
                            int32_t n_children, const uint32_t *sets, int32_t n_sets,
                            const uint8_t *data, int32_t n_data, int32_t root, wg_grammar **out);

@@ -22,6 +22,10 @@
  *   IfElse / Switch(cases Si)     stay* ( s_i L(body_i) )   (Section 3.2; absent body = empty)
  *   DoWhile(body, cond)           (L(body) stay* t)* L(body) stay* f   (Section 3.2 listing)
  *   Sequence(x1..xk)              concatenation
+ *   WaitUntil(A, D, u, body)      the paper's Wait whose wait "token" is a multi-byte string u
+ *                                 (Section 3.2: waits are tokens, e.g. a closing tag): any text
+ *                                 over (A \ D) and the bytes of u, up to and including the FIRST
+ *                                 occurrence of u, then L(body)
  * Readings where the paper is silent: a tree in which no set mentions EOS is followed by an
  * implicit Wait(allow={EOS}, wait={EOS}); once the program has completed the cursor is DONE,
  * which accepts EOS only and stays DONE.
@@ -39,7 +43,7 @@
 #include <omp.h>
 #endif
 
-enum { K_SEQUENCE = 0, K_WRITE = 1, K_WAIT = 2, K_SWITCH = 3, K_DOWHILE = 4 };
+enum { K_SEQUENCE = 0, K_WRITE = 1, K_WAIT = 2, K_SWITCH = 3, K_DOWHILE = 4, K_WAIT_UNTIL = 5 };
 enum { SYM_EOS = 256, SET_WORDS = 9 };
 enum { CUR_DONE = -1, CUR_DEAD = -2, CUR_FINAL_EOS = -3 };
 enum { ERR_ARG = -1, ERR_GRAMMAR = -2, ERR_REJECTED = -4 };
@@ -121,6 +125,7 @@ int wgo_tree_create(const int32_t *nodes, int32_t n_nodes, const int32_t *childr
         case K_WAIT: if (n->n_child != 1 || n->n_set != 3) rc = ERR_ARG; break;
         case K_SWITCH: if (n->n_set < 3 || n->n_child != n->n_set - 2) rc = ERR_ARG; break;
         case K_DOWHILE: if (n->n_child != 1 || n->n_set != 4) rc = ERR_ARG; break;
+        case K_WAIT_UNTIL: if (n->n_child != 1 || n->n_set != 2) rc = ERR_ARG; break;
         default: rc = ERR_ARG;
         }
         if (rc) break;
@@ -143,6 +148,11 @@ int wgo_tree_create(const int32_t *nodes, int32_t n_nodes, const int32_t *childr
                 if (sets_meet(t, a, n->set_off + 1)) rc = ERR_GRAMMAR;
                 for (int b = a + 1; b < last && !rc; b++) if (sets_meet(t, a, b)) rc = ERR_GRAMMAR;
             }
+        }
+        if (n->kind == K_WAIT_UNTIL) { /* a non-empty string, none of whose bytes is denied */
+            if (n->data_len < 1) rc = ERR_GRAMMAR;
+            for (int j = 0; j < n->data_len && !rc; j++)
+                if (in_set(t, n->set_off + 1, t->data[n->data_off + j])) rc = ERR_GRAMMAR;
         }
     }
     if (!rc) { /* every node must hang below the root exactly once */
@@ -170,6 +180,7 @@ static cursor_t enter(const wgo_tree *t, int32_t n, int32_t came_from) {
         return nd->data_len == 0 ? complete(t, n) : cur(n, 0);
     case K_WAIT:
     case K_SWITCH:
+    case K_WAIT_UNTIL:
         return cur(n, 0);
     case K_DOWHILE: {
         int32_t body = t->children[nd->child_off];
@@ -207,6 +218,27 @@ static cursor_t step(const wgo_tree *t, cursor_t c, int sym) {
         return c.off + 1 == nd->data_len ? complete(t, c.node) : cur(c.node, c.off + 1);
     }
     int32_t allow = nd->set_off, deny = nd->set_off + 1;
+    if (nd->kind == K_WAIT_UNTIL) {
+        /* c.off = how many bytes of u the text read so far ends with (the longest such
+         * prefix of u).  After one more symbol: the longest prefix of u that is a suffix of
+         * u[0..off) + symbol, found by trying every length from the top. */
+        const uint8_t *u = t->data + nd->data_off;
+        const int len = nd->data_len;
+        int is_u_byte = 0;
+        for (int j = 0; j < len; j++) if (sym < 256 && u[j] == (uint8_t)sym) is_u_byte = 1;
+        if (!is_u_byte && !(in_set(t, allow, sym) && !in_set(t, deny, sym))) return cur(CUR_DEAD, 0);
+        if (sym >= 256) return cur(c.node, 0); /* EOS is never part of u */
+        int best = 0;
+        for (int j = (c.off + 1 < len ? c.off + 1 : len); j >= 1 && !best; j--) {
+            /* does u[0..j) equal the last j symbols of u[0..off) + symbol? */
+            int same = u[j - 1] == (uint8_t)sym;
+            for (int i = 0; i < j - 1 && same; i++)
+                if (u[i] != u[c.off - (j - 1) + i]) same = 0;
+            if (same) best = j;
+        }
+        if (best == len) return enter(t, t->children[nd->child_off], c.node);
+        return cur(c.node, best);
+    }
     if (nd->kind == K_WAIT) {
         if (in_set(t, nd->set_off + 2, sym)) return enter(t, t->children[nd->child_off], c.node);
     } else if (nd->kind == K_SWITCH) {

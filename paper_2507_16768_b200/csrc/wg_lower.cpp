@@ -96,6 +96,40 @@ struct Lowerer {
             if (!stay.empty()) states[s].push_back({stay, s});
             return s;
         }
+        case WG_OP_WAIT_UNTIL: {
+            // One state per length of matched prefix of the string u (0 .. len-1), wired as
+            // the string-matching automaton of u: from "k bytes matched", byte b leads to the
+            // longest prefix of u that is a suffix of u[0..k) + b, found through the failure
+            // links.  Reaching the full length enters the body.
+            const uint8_t *u = data + n.data_off;
+            const int len = n.data_len;
+            std::vector<int> fail(len, 0);
+            for (int i = 1, m = 0; i < len; ++i) {
+                while (m > 0 && u[i] != u[m]) m = fail[m - 1];
+                if (u[i] == u[m]) ++m;
+                fail[i] = m;
+            }
+            std::vector<int32_t> st(len);
+            for (int i = 0; i < len; ++i) st[i] = new_state();
+            const int32_t done = lower(children[n.child_off], k);
+            SymSet ok = sets[n.set_off];
+            for (int i = 0; i < WG_SET_WORDS; ++i) ok.w[i] &= ~sets[n.set_off + 1].w[i];
+            for (int i = 0; i < len; ++i) ok.w[u[i] >> 5] |= 1u << (u[i] & 31);
+            for (int at = 0; at < len; ++at) {
+                std::vector<SymSet> to(len + 1, SymSet{});
+                for (int b = 0; b < 256; ++b) {
+                    if (!ok.has(b)) continue;
+                    int j = at;
+                    while (j > 0 && u[j] != (uint8_t)b) j = fail[j - 1];
+                    if (u[j] == (uint8_t)b) ++j;
+                    to[j].w[b >> 5] |= 1u << (b & 31);
+                }
+                if (ok.has(WG_SYM_EOS)) to[0].w[WG_SYM_EOS >> 5] |= 1u << (WG_SYM_EOS & 31);
+                for (int j = 0; j <= len; ++j)
+                    if (!to[j].empty()) states[st[at]].push_back({to[j], j == len ? done : st[j]});
+            }
+            return st[0];
+        }
         default: {  // WG_OP_DOWHILE
             int32_t c = new_state();
             int32_t entry = lower(children[n.child_off], c);
@@ -110,8 +144,8 @@ struct Lowerer {
 };
 
 int32_t validate(const wg_op_node *nodes, int32_t n_nodes, const int32_t *children,
-                 int32_t n_children, const SymSet *sets, int32_t n_sets, int32_t n_data,
-                 int32_t root) {
+                 int32_t n_children, const SymSet *sets, int32_t n_sets, const uint8_t *data,
+                 int32_t n_data, int32_t root) {
     std::vector<uint8_t> used(n_nodes, 0);
     used[root] = 1;
     for (int32_t i = 0; i < n_nodes; ++i) {
@@ -128,6 +162,7 @@ int32_t validate(const wg_op_node *nodes, int32_t n_nodes, const int32_t *childr
         case WG_OP_WAIT: shape_ok = n.n_child == 1 && n.n_set == 3; break;
         case WG_OP_SWITCH: shape_ok = n.n_set >= 3 && n.n_child == n.n_set - 2; break;
         case WG_OP_DOWHILE: shape_ok = n.n_child == 1 && n.n_set == 4; break;
+        case WG_OP_WAIT_UNTIL: shape_ok = n.n_child == 1 && n.n_set == 2; break;
         default: break;
         }
         if (!shape_ok) return WG_ERR_ARG;
@@ -140,6 +175,11 @@ int32_t validate(const wg_op_node *nodes, int32_t n_nodes, const int32_t *childr
             if (c < 0 || c >= n_nodes) return WG_ERR_ARG;
             if (used[c]) return WG_ERR_GRAMMAR;  // a node reached twice: not a tree
             used[c] = 1;
+        }
+        if (n.kind == WG_OP_WAIT_UNTIL) {
+            if (n.data_len < 1) return WG_ERR_GRAMMAR;
+            for (int j = 0; j < n.data_len; ++j)
+                if (sets[n.set_off + 1].has(data[n.data_off + j])) return WG_ERR_GRAMMAR;
         }
         if (n.kind == WG_OP_WAIT || n.kind == WG_OP_SWITCH || n.kind == WG_OP_DOWHILE) {
             const SymSet &deny = sets[n.set_off + 1];
@@ -172,7 +212,7 @@ int32_t wg_lower_tree(const wg_op_node *nodes, int32_t n_nodes, const int32_t *c
         (n_data > 0 && !data))
         return WG_ERR_ARG;
     const SymSet *sets = reinterpret_cast<const SymSet *>(sets_raw);
-    int32_t rc = validate(nodes, n_nodes, children, n_children, sets, n_sets, n_data, root);
+    int32_t rc = validate(nodes, n_nodes, children, n_children, sets, n_sets, data, n_data, root);
     if (rc != WG_OK) return rc;
 
     bool mentions_eos = false;

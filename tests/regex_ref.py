@@ -11,7 +11,7 @@ from __future__ import annotations
 
 import regex
 
-from wg_workloads.optree import EOS, DoWhile, Sequence, Switch, SymSet, Wait, Write
+from wg_workloads.optree import EOS, DoWhile, Sequence, Switch, SymSet, Wait, WaitUntil, Write
 
 EOS_BYTE = 0x02
 
@@ -51,6 +51,11 @@ def pattern(op) -> bytes:
     if isinstance(op, Wait):
         stay = (op.allow - op.deny) - op.wait
         return _star(stay) + _cls(op.wait) + pattern(op.body)
+    if isinstance(op, WaitUntil):
+        # any accepted symbol as long as the string does not START here, then the string
+        lit = b"".join(b"\\x%02x" % b for b in op.until)
+        ok = (op.allow - op.deny) | SymSet(op.until)
+        return b"(?:(?!" + lit + b")" + _cls(ok) + b")*" + lit + pattern(op.body)
     if isinstance(op, Switch):
         stay = (op.allow - op.deny) - _union(op.cases)
         alts = b"|".join(_cls(c) + pattern(b) for c, b in zip(op.cases, op.bodies))
@@ -71,6 +76,8 @@ def mentions_eos(op) -> bool:
         return False
     if isinstance(op, Wait):
         return any(EOS in s for s in (op.allow, op.deny, op.wait)) or mentions_eos(op.body)
+    if isinstance(op, WaitUntil):
+        return EOS in op.allow or EOS in op.deny or mentions_eos(op.body)
     if isinstance(op, Switch):
         return (any(EOS in s for s in [op.allow, op.deny] + op.cases)
                 or any(mentions_eos(b) for b in op.bodies))

@@ -9,8 +9,8 @@ import pytest
 
 import oracle
 from cosim import co_reachable, mentioned_symbols
-from wg_workloads import (ALL_BYTES, EOS, Cond, DoWhile, IfElse, Sequence, SymSet, Wait, Write,
-                          flatten, grammars)
+from wg_workloads import (ALL_BYTES, EOS, Cond, DoWhile, IfElse, Sequence, SymSet, Wait, WaitUntil,
+                          Write, flatten, grammars)
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
@@ -51,6 +51,9 @@ GRAMMARS = {
     "template1": lambda: grammars.random_template(1),
     "template6": lambda: grammars.random_template(6),
     "snippets": lambda: grammars.dynamic_snippet_template(2, n_args=3, enum_size=12),
+    "html_tags": lambda: grammars.html_template(wait_for_tag=True),
+    "overlapping_until": lambda: Sequence(WaitUntil(SymSet(b"abc"), b"abcab", body=Write(b"x")),
+                                          WaitUntil(ALL_BYTES, b"aa")),
     "empty_bodies": lambda: Sequence(
         Write(b""), DoWhile(None, Cond(ALL_BYTES, SymSet(b","), SymSet(b";"))),
         Wait(SymSet(b"ab"), SymSet(b"!"), body=Sequence()), IfElse(
@@ -88,6 +91,8 @@ def test_identical_trees_hash_equal_and_different_trees_do_not(wg):
     Wait(allow=SymSet(b"ab"), wait=SymSet(b"b"), deny=SymSet(b"b")),
     IfElse(Cond(SymSet(b"ab"), SymSet(b"ab"), SymSet(b"b")), None, None),
     DoWhile(Write(b"x"), Cond(SymSet(b"a"), SymSet(b"a"), SymSet())),
+    WaitUntil(ALL_BYTES, b""),
+    WaitUntil(ALL_BYTES, b"ab", deny=SymSet(b"a")),
 ])
 def test_compile_rejects_what_the_checker_rejects(wg, bad):
     flat = flatten(bad)

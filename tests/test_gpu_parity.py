@@ -62,6 +62,7 @@ SMALL = {
     "template2": lambda: grammars.random_template(2),
     "snippets": lambda: grammars.dynamic_snippet_template(4, n_args=3, enum_size=10),
     "listing": grammars.paper_listing_example,
+    "html_tags": lambda: grammars.html_template(wait_for_tag=True),
 }
 
 

@@ -19,7 +19,7 @@ import pytest
 import oracle
 import regex_ref
 from wg_workloads import (ALL_BYTES, DIGITS, EOS, Cond, DoWhile, IfElse, Sequence, Switch, SymSet,
-                          Wait, Write, bf16_bits_to_f32, enum_trie, flatten, grammars,
+                          Wait, WaitUntil, Write, bf16_bits_to_f32, enum_trie, flatten, grammars,
                           make_logits, make_vocab, vocab_from_tokens)
 
 
@@ -161,6 +161,7 @@ SMALL_GRAMMARS = {
     "template0": lambda: grammars.random_template(0, 4, 6),
     "template5": lambda: grammars.random_template(5, 4, 6),
     "snippets": lambda: grammars.dynamic_snippet_template(3, n_args=2, enum_size=7),
+    "html_tags": lambda: grammars.html_template(wait_for_tag=True),
 }
 
 
@@ -416,3 +417,59 @@ def test_enum_trie_accepts_exactly_its_strings():
         assert tree.accepts(list(b'"' + n + b";") + [EOS])
     for bad in [b'alp"', b'alphas"', b'bet"', b'gamma-3"', b'"']:
         assert not tree.accepts(list(b'"' + bad + b";") + [EOS])
+
+
+# ---------------------------------------------------------------------------------------
+# Wait on a multi-byte string (the paper's waits are tokens such as a closing tag)
+# ---------------------------------------------------------------------------------------
+def test_wait_until_ends_at_the_first_occurrence_of_its_string():
+    tree = tree_of(Sequence(Write(b"<p>"), WaitUntil(ALL_BYTES, b"</p>"), Write(b"!")))
+    for s, want in [(b"<p>hello</p>!", True), (b"<p></p>!", True), (b"<p>a<b</</p>!", True),
+                    (b"<p></p></p>!", False), (b"<p>a</p!", False), (b"<p>a</p>", False)]:
+        assert tree.accepts(list(s) + [EOS]) is want, s
+    # a string that overlaps itself: the match must restart from the longest border
+    tree = tree_of(WaitUntil(SymSet(b"ab"), b"aab"))
+    for s, want in [(b"aab", True), (b"aaab", True), (b"abaab", True), (b"bbaaaab", True),
+                    (b"aabaab", False), (b"abab", False), (b"acab", False), (b"aa", False)]:
+        assert tree.accepts(list(s) + [EOS]) is want, s
+    # bytes of the string are accepted even when allow does not list them; deny still rules
+    tree = tree_of(WaitUntil(SymSet(b"xy"), b"end", deny=SymSet(b"y")))
+    assert tree.accepts(list(b"xxenend") + [EOS]) and not tree.accepts(list(b"xyend") + [EOS])
+    for bad in (WaitUntil(ALL_BYTES, b""), WaitUntil(ALL_BYTES, b"ab", deny=SymSet(b"b"))):
+        with pytest.raises(oracle.OracleError) as e:
+            tree_of(bad)
+        assert e.value.code == oracle.ERR_GRAMMAR
+
+
+def test_wait_until_language_by_plain_string_search():
+    # membership by the definition itself: the string occurs, and first occurs at the very end
+    until = b"abab"
+    tree = tree_of(WaitUntil(SymSet(b"abc"), until))
+    for n in range(0, 9):
+        for tup in itertools.product(b"abcx", repeat=n):
+            s = bytes(tup)
+            want = s.endswith(until) and s.find(until) == len(s) - len(until) and b"x" not in s
+            assert tree.accepts(list(s) + [EOS]) is want, s
+
+
+def test_wait_until_mask_closed_form(vocab32k):
+    closing = b"</h1>\n"
+    op = Sequence(Write(b"<h1>"), WaitUntil(ALL_BYTES, closing), Write(b"<p>"))
+    tree = tree_of(op)
+    seen = b"so far: 1 <"                       # the text already ends with one byte of the tag
+    cursor = tree.walk(tree.start(), list(b"<h1>" + seen))
+    got = unpack(oracle.mask(tree, vocab32k, cursor), vocab32k.size)
+    n_cut = 0
+    for t, tok in enumerate(vocab32k.tokens()):
+        if t == 2 or not tok:
+            want = False
+        else:
+            text = seen + tok
+            at = text.find(closing)
+            if at < 0:
+                want = True                      # still inside the slot
+            else:                                # what follows the tag must start the next literal
+                want = b"<p>".startswith(text[at + len(closing):])
+                n_cut += 1
+        assert bool(got[t]) == want, tok
+    assert got.mean() > 0.95

@@ -12,7 +12,7 @@ from typing import List
 import numpy as np
 
 from .optree import (ALL_BYTES, DIGITS, Cond, DoWhile, IfElse, Op, Sequence, Switch, SymSet,
-                     Wait, Write, enum_trie)
+                     Wait, WaitUntil, Write, enum_trie)
 
 LT = ord("<")
 
@@ -50,12 +50,20 @@ HTML_TAGS = [
 ]
 
 
-def html_template() -> Op:
-    """Config 1: eight literal tags in a fixed order with four free-text slots."""
+def html_template(wait_for_tag: bool = False) -> Op:
+    """Config 1: eight literal tags in a fixed order with four free-text slots.
+
+    By default a slot is free of '<' and ends at the first '<' (single-symbol wait sets).
+    With ``wait_for_tag`` the slot is a Wait on the whole closing tag: any text, '<' included,
+    up to the first occurrence of the tag.
+    """
     parts: List[Op] = []
     for open_tag, close_tag in HTML_TAGS:
         parts.append(Write(open_tag))
-        parts.extend(text_slot(close_tag))
+        if wait_for_tag:
+            parts.append(WaitUntil(ALL_BYTES, close_tag))
+        else:
+            parts.extend(text_slot(close_tag))
     return Sequence(parts)
 
 

@@ -23,6 +23,7 @@ Per kind:
   WAIT      sets     = [allow, deny, wait];             children = [body]
   SWITCH    sets     = [allow, deny, case_0..case_k-1]; children = [body_0..body_k-1]
   DOWHILE   sets     = [allow, deny, true, false];      children = [body]
+  WAIT_UNTIL sets    = [allow, deny]; data = the string waited for; children = [body]
 
 IfElse is the two-case SWITCH: case_0 = true_waits -> if_body, case_1 =
 false_waits -> else_body.
@@ -43,6 +44,7 @@ KIND_WRITE = 1
 KIND_WAIT = 2
 KIND_SWITCH = 3
 KIND_DOWHILE = 4
+KIND_WAIT_UNTIL = 5
 
 SymbolsLike = Union[bytes, str, Iterable[int], "SymSet"]
 
@@ -142,6 +144,23 @@ class Wait(Op):
         self.allow = SymSet(self.allow)
         self.wait = SymSet(self.wait)
         self.deny = SymSet(self.deny)
+
+
+@dataclass
+class WaitUntil(Op):
+    """A Wait whose wait "token" is a multi-byte string: text over ``allow`` (minus ``deny``)
+    and the string's own bytes, up to and including the first occurrence of ``until``."""
+
+    allow: SymSet
+    until: bytes
+    deny: SymSet = field(default_factory=SymSet)
+    body: Optional[Op] = None
+
+    def __post_init__(self):
+        self.allow = SymSet(self.allow)
+        self.deny = SymSet(self.deny)
+        if isinstance(self.until, str):
+            self.until = self.until.encode("utf-8")
 
 
 @dataclass
@@ -253,6 +272,13 @@ def flatten(root: Op) -> FlatTree:
         elif isinstance(op, Wait):
             idx = new_node(KIND_WAIT)
             add_sets(idx, [op.allow, op.deny, op.wait])
+            kids = [op.body]
+        elif isinstance(op, WaitUntil):
+            idx = new_node(KIND_WAIT_UNTIL)
+            add_sets(idx, [op.allow, op.deny])
+            nodes[idx][5] = len(data)
+            nodes[idx][6] = len(op.until)
+            data.extend(op.until)
             kids = [op.body]
         elif isinstance(op, Switch):
             idx = new_node(KIND_SWITCH)
