@@ -76,7 +76,8 @@ enum {
     WG_OP_WAIT = 2,
     WG_OP_SWITCH = 3, /* IfElse and its k-way generalisation */
     WG_OP_DOWHILE = 4,
-    WG_OP_WAIT_UNTIL = 5 /* a Wait whose wait "token" is a multi-byte string */
+    WG_OP_WAIT_UNTIL = 5,  /* a Wait whose wait "token" is a multi-byte string */
+    WG_OP_WRITE_TOKENS = 6 /* the paper's token-level Write: forced token ids        */
 };
 
 /* One node of a flattened operator tree.  Children, symbol sets and literal bytes live in
@@ -91,7 +92,12 @@ enum {
  *   WAIT_UNTIL sets    = [allow, deny], data = the string waited for, children = [body or -1]
  *             (paper Section 3.2: the waits of a Wait are tokens, e.g. a closing tag; at byte
  *             level such a token is a string.  Accepts text over (allow \ deny) and the
- *             string's own bytes up to and including the FIRST occurrence of the string.) */
+ *             string's own bytes up to and including the FIRST occurrence of the string.)
+ *   WRITE_TOKENS data  = the forced token ids, 4 little-endian bytes each (ids >= 0)
+ *             (paper Section 3.2: Write "outputs predetermined token sequences"; Section 3.3:
+ *             a chain of Waits each expecting one token.  Exactly these ids, one per decode
+ *             step; entered and left at token boundaries only, so no token's bytes may run
+ *             into or out of it.  An id beyond the vocabulary yields an empty mask.) */
 typedef struct wg_op_node {
     int32_t kind;
     int32_t n_child, child_off;
@@ -182,6 +188,11 @@ int32_t wg_grammar_info(const wg_grammar *grammar, int32_t *n_states, int32_t *s
 /* Host-side single transition: the state after `symbol` (0..256) in `state`, 0 = DEAD.
  * Out-of-range arguments give 0.  For tests and tooling; not on the decode path. */
 int32_t wg_grammar_step(const wg_grammar *grammar, int32_t state, int32_t symbol);
+
+/* Host-side: is `state` a forced-token state of a WRITE_TOKENS operator?  Returns 1 and fills
+ * *token / *next_state (either may be NULL) if so, 0 otherwise (also for bad arguments). */
+int32_t wg_grammar_forced_token(const wg_grammar *grammar, int32_t state, int32_t *token,
+                                int32_t *next_state);
 
 /* Creates the device context on the current device: grammar table registry, the mask cache
  * (a hash table keyed by (grammar id, state id) plus a pool of `cache_capacity` mask rows,

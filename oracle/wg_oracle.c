@@ -26,6 +26,11 @@
  *                                 (Section 3.2: waits are tokens, e.g. a closing tag): any text
  *                                 over (A \ D) and the bytes of u, up to and including the FIRST
  *                                 occurrence of u, then L(body)
+ *   WriteTokens(t1..tn)           the paper's own Write (Section 3.2: "outputs predetermined token
+ *                                 sequences"; Section 3.3: a chain of Waits each expecting one
+ *                                 token): exactly these token ids, one per decode step.  It is
+ *                                 entered and left only at token boundaries: no token's bytes
+ *                                 may run into it or out of it.
  * Readings where the paper is silent: a tree in which no set mentions EOS is followed by an
  * implicit Wait(allow={EOS}, wait={EOS}); once the program has completed the cursor is DONE,
  * which accepts EOS only and stays DONE.
@@ -43,7 +48,7 @@
 #include <omp.h>
 #endif
 
-enum { K_SEQUENCE = 0, K_WRITE = 1, K_WAIT = 2, K_SWITCH = 3, K_DOWHILE = 4, K_WAIT_UNTIL = 5 };
+enum { K_SEQUENCE = 0, K_WRITE = 1, K_WAIT = 2, K_SWITCH = 3, K_DOWHILE = 4, K_WAIT_UNTIL = 5, K_WRITE_TOKENS = 6 };
 enum { SYM_EOS = 256, SET_WORDS = 9 };
 enum { CUR_DONE = -1, CUR_DEAD = -2, CUR_FINAL_EOS = -3 };
 enum { ERR_ARG = -1, ERR_GRAMMAR = -2, ERR_REJECTED = -4 };
@@ -126,6 +131,7 @@ int wgo_tree_create(const int32_t *nodes, int32_t n_nodes, const int32_t *childr
         case K_SWITCH: if (n->n_set < 3 || n->n_child != n->n_set - 2) rc = ERR_ARG; break;
         case K_DOWHILE: if (n->n_child != 1 || n->n_set != 4) rc = ERR_ARG; break;
         case K_WAIT_UNTIL: if (n->n_child != 1 || n->n_set != 2) rc = ERR_ARG; break;
+        case K_WRITE_TOKENS: if (n->n_child != 0 || n->n_set != 0 || n->data_len % 4) rc = ERR_ARG; break;
         default: rc = ERR_ARG;
         }
         if (rc) break;
@@ -177,6 +183,7 @@ static cursor_t enter(const wgo_tree *t, int32_t n, int32_t came_from) {
     const node_t *nd = &t->nodes[n];
     switch (nd->kind) {
     case K_WRITE:
+    case K_WRITE_TOKENS:
         return nd->data_len == 0 ? complete(t, n) : cur(n, 0);
     case K_WAIT:
     case K_SWITCH:
@@ -213,6 +220,7 @@ static cursor_t step(const wgo_tree *t, cursor_t c, int sym) {
     if (c.node == CUR_DONE || c.node == CUR_FINAL_EOS)
         return sym == SYM_EOS ? cur(CUR_DONE, 0) : cur(CUR_DEAD, 0);
     const node_t *nd = &t->nodes[c.node];
+    if (nd->kind == K_WRITE_TOKENS) return cur(CUR_DEAD, 0); /* only whole tokens pass here */
     if (nd->kind == K_WRITE) {
         if (sym >= 256 || t->data[nd->data_off + c.off] != (uint8_t)sym) return cur(CUR_DEAD, 0);
         return c.off + 1 == nd->data_len ? complete(t, c.node) : cur(c.node, c.off + 1);
@@ -270,6 +278,14 @@ void wgo_step(const wgo_tree *t, const int32_t *in, int32_t sym, int32_t *out) {
  * A zero-length token other than EOS is refused (it would leave the request where it is). */
 static cursor_t walk_token(const wgo_tree *t, cursor_t c, const uint32_t *offsets,
                            const uint8_t *bytes, int32_t eos_id, int32_t tok) {
+    if (c.node >= 0 && t->nodes[c.node].kind == K_WRITE_TOKENS) {
+        /* the next token of the forced sequence, as a whole token, and nothing else */
+        const node_t *nd = &t->nodes[c.node];
+        int32_t want;
+        memcpy(&want, t->data + nd->data_off + 4 * c.off, 4);
+        if (tok != want) return cur(CUR_DEAD, 0);
+        return 4 * (c.off + 1) == nd->data_len ? complete(t, c.node) : cur(c.node, c.off + 1);
+    }
     if (tok == eos_id) return step(t, c, SYM_EOS);
     uint32_t b = offsets[tok], e = offsets[tok + 1];
     if (b == e) return cur(CUR_DEAD, 0);

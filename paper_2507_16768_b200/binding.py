@@ -64,6 +64,7 @@ _SIGNATURES = {
     "wg_grammar_info": (_i32, [_vp, C.POINTER(_i32), C.POINTER(_i32), C.POINTER(_i32),
                                C.POINTER(_i32), C.POINTER(C.c_uint64)]),
     "wg_grammar_step": (_i32, [_vp, _i32, _i32]),
+    "wg_grammar_forced_token": (_i32, [_vp, _i32, C.POINTER(_i32), C.POINTER(_i32)]),
     "wg_ctx_create": (_i32, [_vp, _i32, _i32, C.POINTER(_vp)]),
     "wg_ctx_free": (None, [_vp]),
     "wg_ctx_add_grammar": (_i32, [_vp, _vp, C.POINTER(_i32)]),
@@ -223,6 +224,20 @@ class Grammar:
 
     def step(self, state: int, symbol: int) -> int:
         return int(_lib.wg_grammar_step(self.handle, int(state), int(symbol)))
+
+    def forced_token(self, state: int):
+        """(token id, next state) if ``state`` belongs to a token-level Write, else None."""
+        tok, nxt = _i32(), _i32()
+        if _lib.wg_grammar_forced_token(self.handle, int(state), C.byref(tok), C.byref(nxt)):
+            return tok.value, nxt.value
+        return None
+
+    def step_token(self, state: int, token: int, symbols) -> int:
+        """Host-side state after a whole token (``symbols`` = its bytes, or [256] for EOS)."""
+        forced = self.forced_token(state)
+        if forced is not None:
+            return forced[1] if token == forced[0] else 0
+        return self.walk(state, symbols)
 
     def walk(self, state: int, symbols) -> int:
         for s in symbols:

@@ -79,8 +79,9 @@ struct wg_vocab {
 struct GrammarSlot {
     uint64_t hash;
     std::vector<int32_t> table;  // host copy, for exact comparison on hash equality
+    std::vector<int32_t> forced_tok, forced_next;
     int32_t n_states, n_classes;
-    void *d_table, *d_cls, *d_first_ok, *d_leaves;
+    void *d_table, *d_cls, *d_first_ok, *d_leaves, *d_forced;
 };
 
 struct wg_ctx {
@@ -252,6 +253,15 @@ int32_t wg_grammar_info(const wg_grammar *g, int32_t *n_states, int32_t *start_s
     return WG_OK;
 }
 
+int32_t wg_grammar_forced_token(const wg_grammar *g, int32_t state, int32_t *token,
+                                int32_t *next_state) {
+    if (!g || state < 0 || state >= g->n_states || g->forced_tok.empty()) return 0;
+    if (g->forced_tok[state] < 0) return 0;
+    if (token) *token = g->forced_tok[state];
+    if (next_state) *next_state = g->forced_next[state];
+    return 1;
+}
+
 int32_t wg_grammar_step(const wg_grammar *g, int32_t state, int32_t symbol) {
     if (!g || state < 0 || state >= g->n_states || symbol < 0 || symbol >= WG_N_SYMBOLS) return 0;
     const int c = symbol == WG_SYM_EOS ? g->eos_class : g->byte_class[symbol];
@@ -330,6 +340,7 @@ void wg_ctx_free(wg_ctx *c) {
         cudaFree(s.d_cls);
         cudaFree(s.d_first_ok);
         cudaFree(s.d_leaves);
+        cudaFree(s.d_forced);
     }
     delete c;
 }
@@ -340,14 +351,22 @@ int32_t wg_ctx_add_grammar(wg_ctx *c, const wg_grammar *g, int32_t *grammar_id) 
     for (size_t i = 0; i < c->slots.size(); ++i) {
         const GrammarSlot &s = c->slots[i];
         if (s.hash == g->hash && s.n_states == g->n_states && s.n_classes == g->n_classes &&
-            s.table == g->table) {
+            s.table == g->table && s.forced_tok == g->forced_tok && s.forced_next == g->forced_next) {
             *grammar_id = (int32_t)i;
             return WG_OK;
         }
     }
     if (c->slots.size() >= 65535) return WG_ERR_CAPACITY;
     const bool wide = g->n_states > 65535;
-    GrammarSlot slot{g->hash, g->table, g->n_states, g->n_classes, nullptr, nullptr, nullptr, nullptr};
+    GrammarSlot slot{g->hash, g->table, g->forced_tok, g->forced_next, g->n_states, g->n_classes,
+                     nullptr, nullptr, nullptr, nullptr, nullptr};
+    if (!g->forced_tok.empty()) {
+        std::vector<int2> forced(g->n_states);
+        for (int32_t st = 0; st < g->n_states; ++st) forced[st] = make_int2(g->forced_tok[st], g->forced_next[st]);
+        WG_CUDA(cudaMalloc(&slot.d_forced, forced.size() * sizeof(int2)));
+        WG_CUDA(cudaMemcpy(slot.d_forced, forced.data(), forced.size() * sizeof(int2),
+                           cudaMemcpyHostToDevice));
+    }
     const size_t n = g->table.size();
     if (wide) {
         WG_CUDA(cudaMalloc(&slot.d_table, n * sizeof(uint32_t)));
@@ -382,7 +401,8 @@ int32_t wg_ctx_add_grammar(wg_ctx *c, const wg_grammar *g, int32_t *grammar_id) 
     }
     GrammarDev gd{slot.d_table, static_cast<const uint8_t *>(slot.d_cls),
                   static_cast<const uint32_t *>(slot.d_first_ok),
-                  static_cast<const unsigned long long *>(slot.d_leaves), g->n_states,
+                  static_cast<const unsigned long long *>(slot.d_leaves),
+                  static_cast<const int2 *>(slot.d_forced), g->n_states,
                   g->n_classes, g->start, g->done, g->eos_class, wide ? 1 : 0};
     const int32_t id = (int32_t)c->slots.size();
     if (id >= c->grammar_cap) {  // grow the registry; queued kernels still read the old one

@@ -23,6 +23,10 @@ struct wg_grammar {
     int32_t eos_class = 0;
     uint8_t byte_class[256] = {};
     std::vector<int32_t> table;
+    // Token-level Write: forced_tok[s] >= 0 marks a state that accepts exactly that token id
+    // (as a whole token) and continues in forced_next[s]; its table row is all DEAD.  Both
+    // vectors are empty when the grammar has no such state.
+    std::vector<int32_t> forced_tok, forced_next;
     uint64_t hash = 0;
 };
 

@@ -17,6 +17,8 @@ struct GrammarDev {
     const uint32_t *first_ok;   // [n_states][8] bit b: byte b does not lead to DEAD
     const unsigned long long *leaves;  // [n_states] OR of 1 << (b & 63) over bytes b that
                                        // lead anywhere but back to the state itself
+    const int2 *forced;         // [n_states] (token id or -1, next state), or NULL: states of a
+                                // token-level Write accept exactly one whole token
     int32_t n_states, n_classes, start, done, eos_class, wide;
 };
 
@@ -172,6 +174,7 @@ build_masks_kernel(VocabDev v, CtxDev ctx, BuildWork work) {
         uint32_t eos_next = 0;
         if (s0) eos_next = g.wide ? static_cast<const uint32_t *>(g.table)[(size_t)s0 * g.n_classes + g.eos_class]
                                   : static_cast<const uint16_t *>(g.table)[(size_t)s0 * g.n_classes + g.eos_class];
+        const int forced_tok = (s0 && g.forced) ? g.forced[s0].x : -1;  // token-level Write state
         __syncthreads();
         if (threadIdx.x == 0 && known) cls_gid = gid;  // read again only after the next barrier
         {
@@ -187,7 +190,9 @@ build_masks_kernel(VocabDev v, CtxDev ctx, BuildWork work) {
         for (int wl = threadIdx.x; wl < ((n_words + 31) & ~31); wl += BUILD_THREADS) {
             uint32_t alive = 0, queue = 0;
             const int w = (t_begin >> 5) + wl;
-            if (wl < n_words && s0 != 0) {
+            if (wl < n_words && forced_tok >= 0) {
+                if ((forced_tok >> 5) == w && forced_tok < v.V) alive = 1u << (forced_tok & 31);
+            } else if (wl < n_words && s0 != 0) {
                 uint32_t p = 0;
                 for (int i = 0; i < nf; ++i) p |= __ldg(&v.first_mask[(size_t)first_list[i] * v.W + w]);
                 if (complement) p = __ldg(&v.valid_mask[w]) & ~p;
@@ -661,7 +666,10 @@ __global__ void advance_kernel(VocabDev v, CtxDev ctx, const int32_t *gid, int32
     } else {
         const GrammarDev gr = ctx.grammars[g];
         uint32_t next = 0;
-        if (t >= 0 && t < v.V && s != 0) {
+        if (gr.forced && s != 0 && gr.forced[s].x >= 0) {  // token-level Write: that token only
+            const int2 f = gr.forced[s];
+            if (t == f.x && t < v.V) next = (uint32_t)f.y;
+        } else if (t >= 0 && t < v.V && s != 0) {
             next = gr.wide ? walk_token<uint32_t>(v, static_cast<const uint32_t *>(gr.table),
                                                   gr.n_classes, gr.eos_class, gr.byte_class, s, t)
                            : walk_token<uint16_t>(v, static_cast<const uint16_t *>(gr.table),

@@ -45,9 +45,12 @@ struct Lowerer {
     const SymSet *sets;
     const uint8_t *data;
     std::vector<std::vector<Edge>> states;  // outgoing edges; symbols on no edge go to DEAD
+    std::vector<int32_t> forced_tok, forced_next;  // per state; -1 = an ordinary state
 
     int32_t new_state() {
         states.emplace_back();
+        forced_tok.push_back(-1);
+        forced_next.push_back(0);
         return (int32_t)states.size() - 1;
     }
 
@@ -95,6 +98,19 @@ struct Lowerer {
             SymSet stay = stay_set(n);
             if (!stay.empty()) states[s].push_back({stay, s});
             return s;
+        }
+        case WG_OP_WRITE_TOKENS: {
+            // One state per forced token: no byte leaves it, only the token id itself.
+            int32_t next = k;
+            for (int j = n.data_len / 4 - 1; j >= 0; --j) {
+                int32_t tok;
+                memcpy(&tok, data + n.data_off + 4 * j, 4);
+                const int32_t s = new_state();
+                forced_tok[s] = tok;
+                forced_next[s] = next;
+                next = s;
+            }
+            return next;
         }
         case WG_OP_WAIT_UNTIL: {
             // One state per length of matched prefix of the string u (0 .. len-1), wired as
@@ -163,6 +179,7 @@ int32_t validate(const wg_op_node *nodes, int32_t n_nodes, const int32_t *childr
         case WG_OP_SWITCH: shape_ok = n.n_set >= 3 && n.n_child == n.n_set - 2; break;
         case WG_OP_DOWHILE: shape_ok = n.n_child == 1 && n.n_set == 4; break;
         case WG_OP_WAIT_UNTIL: shape_ok = n.n_child == 1 && n.n_set == 2; break;
+        case WG_OP_WRITE_TOKENS: shape_ok = n.n_child == 0 && n.n_set == 0 && n.data_len % 4 == 0; break;
         default: break;
         }
         if (!shape_ok) return WG_ERR_ARG;
@@ -175,6 +192,13 @@ int32_t validate(const wg_op_node *nodes, int32_t n_nodes, const int32_t *childr
             if (c < 0 || c >= n_nodes) return WG_ERR_ARG;
             if (used[c]) return WG_ERR_GRAMMAR;  // a node reached twice: not a tree
             used[c] = 1;
+        }
+        if (n.kind == WG_OP_WRITE_TOKENS) {
+            for (int j = 0; j < n.data_len / 4; ++j) {
+                int32_t tok;
+                memcpy(&tok, data + n.data_off + 4 * j, 4);
+                if (tok < 0) return WG_ERR_GRAMMAR;
+            }
         }
         if (n.kind == WG_OP_WAIT_UNTIL) {
             if (n.data_len < 1) return WG_ERR_GRAMMAR;
@@ -251,6 +275,11 @@ int32_t wg_lower_tree(const wg_op_node *nodes, int32_t n_nodes, const int32_t *c
                 q.push(e.to);
             }
         }
+        if (lw.forced_tok[s] >= 0 && new_id[lw.forced_next[s]] < 0) {
+            new_id[lw.forced_next[s]] = (int32_t)order.size();
+            order.push_back(lw.forced_next[s]);
+            q.push(lw.forced_next[s]);
+        }
     }
     if (new_id[done] < 0) {  // cannot happen for a valid tree, but keep DONE addressable
         new_id[done] = (int32_t)order.size();
@@ -321,7 +350,24 @@ int32_t wg_lower_tree(const wg_op_node *nodes, int32_t n_nodes, const int32_t *c
             out->table[(size_t)i * n_cls + c] = t;
         }
     }
+    out->forced_tok.clear();
+    out->forced_next.clear();
+    bool any_forced = false;
+    for (int32_t i = 0; i < S; ++i) any_forced |= lw.forced_tok[order[i]] >= 0;
+    if (any_forced) {
+        out->forced_tok.assign(S, -1);
+        out->forced_next.assign(S, 0);
+        for (int32_t i = 0; i < S; ++i) {
+            if (lw.forced_tok[order[i]] < 0) continue;
+            out->forced_tok[i] = lw.forced_tok[order[i]];
+            out->forced_next[i] = new_id[lw.forced_next[order[i]]];
+        }
+    }
     uint64_t h = 0xCBF29CE484222325ull;
+    if (any_forced) {
+        h = fnv1a(h, out->forced_tok.data(), out->forced_tok.size() * sizeof(int32_t));
+        h = fnv1a(h, out->forced_next.data(), out->forced_next.size() * sizeof(int32_t));
+    }
     h = fnv1a(h, &out->n_states, 4);
     h = fnv1a(h, &out->n_classes, 4);
     h = fnv1a(h, &out->done, 4);

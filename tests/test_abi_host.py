@@ -10,7 +10,7 @@ import pytest
 import oracle
 from cosim import co_reachable, mentioned_symbols
 from wg_workloads import (ALL_BYTES, EOS, Cond, DoWhile, IfElse, Sequence, SymSet, Wait, WaitUntil,
-                          Write, flatten, grammars)
+                          Write, WriteTokens, flatten, grammars, make_vocab)
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
@@ -123,3 +123,43 @@ def test_compile_rejects_malformed_arrays(wg):
 def test_large_enum_grammar_needs_wide_state_ids(wg):
     g = wg.Grammar(flatten(grammars.dynamic_snippet_template(0, n_args=8, enum_size=1000)))
     assert g.n_states > 40000
+
+
+def test_token_level_write_states_follow_the_checker_token_by_token(wg):
+    vocab = make_vocab(3000, seed=17)
+    toks = vocab.tokens()
+    digits = SymSet(b"0123456789")
+    op = Sequence(Write(b"id="), WriteTokens([500, 2, 501]),
+                  DoWhile(Sequence(WriteTokens([600]), Wait(digits, digits)),
+                          Cond(digits | b",.", SymSet(b","), SymSet(b"."))),
+                  WriteTokens([]), Write(b"ok"))
+    flat = flatten(op)
+    tree, g = oracle.Tree(flat), wg.Grammar(flat)
+    assert wg.Grammar(flat).content_hash == g.content_hash
+    rng = np.random.default_rng(3)
+    for _ in range(20):
+        cursor, sid = tree.start(), g.start_state
+        for _ in range(40):
+            words = oracle.mask(tree, vocab, cursor)
+            allowed = np.flatnonzero(np.unpackbits(words.view(np.uint8), bitorder="little")[:vocab.size])
+            assert allowed.size > 0
+            forced = g.forced_token(sid)
+            if forced is not None:
+                assert allowed.tolist() == [forced[0]]
+            # also try a few tokens that are not allowed: both sides must refuse them
+            for t in rng.integers(0, vocab.size, size=5):
+                rc, _ = oracle.advance(tree, vocab, cursor, int(t))
+                syms = [EOS] if t == vocab.eos_id else list(toks[t])
+                assert (rc == 0) == (g.step_token(sid, int(t), syms) != 0 and len(syms) > 0)
+            t = int(rng.choice(allowed))
+            rc, cursor = oracle.advance(tree, vocab, cursor, t)
+            sid = g.step_token(sid, t, [EOS] if t == vocab.eos_id else list(toks[t]))
+            assert rc == 0 and sid != 0
+            if cursor == oracle.DONE:
+                assert sid == g.done_state
+                break
+    bad = flatten(WriteTokens([3]))
+    bad.data[:] = np.frombuffer(np.array([-4], "<i4").tobytes(), np.uint8)
+    with pytest.raises(wg.WgError) as e:
+        wg.Grammar(bad)
+    assert e.value.status == wg.binding.WG_ERR_GRAMMAR

@@ -8,7 +8,8 @@ import pytest
 
 import oracle
 from cosim import co_reachable, mentioned_symbols, token_symbols
-from wg_workloads import (ALL_BYTES, BY_NAME, EOS, Sequence, SymSet, Wait, Write, flatten, grammars,
+from wg_workloads import (ALL_BYTES, BY_NAME, EOS, Cond, DoWhile, Sequence, SymSet, Wait, Write,
+                          WriteTokens, flatten, grammars,
                           has_structural_byte, make_logits, make_vocab, vocab_from_tokens)
 
 pytestmark = pytest.mark.gpu
@@ -243,7 +244,7 @@ class Sim:
             t = int(got_tok[r])
             rc, cur = oracle.advance(self.trees[gi], vocab, self.cursors[r], t)
             assert rc == 0, (self.step_no, r, t)
-            host_sid = self.grams[gi].walk(int(self.h_sid[r]), token_symbols(vocab, t))
+            host_sid = self.grams[gi].step_token(int(self.h_sid[r]), t, token_symbols(vocab, t))
             if cur == oracle.DONE:
                 cur = self.trees[gi].start()
                 host_sid = self.grams[gi].start_state
@@ -491,3 +492,45 @@ def test_degenerate_vocabularies_and_full_batches(wg, torch):
     want = oracle.masks([tree, tree], vocab, [tree.start(), tree.step(tree.start(), ord("c"))])
     assert (out.cpu().numpy().view(np.uint32) == want).all()
     assert want[0, 0] == 0b1110111 and want[1, 0] == 0
+
+
+def test_trajectory_with_token_level_writes(wg, torch):
+    vocab = make_vocab(8192, seed=14)
+    toks = vocab.tokens()
+    forced = [toks.index(b"<"), 700, 701, vocab.eos_id, 5000]
+    digits = SymSet(b"0123456789")
+    loop = DoWhile(Sequence(WriteTokens([900, 901]), Wait(digits, digits)),
+                   Cond(digits | b",;", SymSet(b","), SymSet(b";")))
+    ops = [Sequence(Write(b"ab"), WriteTokens(forced), Write(b"cd"), loop),
+           Sequence(WriteTokens([1, 3]), Wait(ALL_BYTES, SymSet(b"<")), WriteTokens([4000]))]
+    sim = Sim(wg, torch, vocab, ops, [0, 1, 0, 0], "bf16", cache_capacity=256, seed=11, steer=4.0)
+    for _ in range(60):
+        sim.step(fused=(sim.step_no % 2 == 0))
+    assert len(sim.visited) > 12
+    # states of a token-level Write allow exactly their token
+    g = sim.grams[0]
+    forced_states = [s for s in range(1, g.n_states) if g.forced_token(s)]
+    assert len(forced_states) == len(forced) + 2
+    B = len(forced_states)
+    out = torch.zeros((B, sim.dv.W), dtype=torch.int32, device="cuda")
+    ctx = wg.Context(sim.dv, 0, B)
+    wg.wg_build_masks(ctx, torch.full((B,), ctx.add_grammar(g), dtype=torch.int32, device="cuda"),
+                      to_dev(torch, np.array(forced_states, np.int32)), out, wg.WG_NO_CACHE)
+    bits = np.unpackbits(out.cpu().numpy().view(np.uint8), axis=1, bitorder="little")
+    assert (bits.sum(axis=1) == 1).all()
+    assert sorted(int(np.flatnonzero(b)[0]) for b in bits) == sorted(forced + [900, 901])
+
+
+def test_forced_token_beyond_the_vocabulary_gives_an_empty_mask(wg, torch):
+    vocab = make_vocab(1024, seed=14)
+    g = wg.Grammar(flatten(WriteTokens([vocab.size + 7])))
+    dv = wg.Vocab(vocab.offsets, vocab.data, vocab.eos_id)
+    ctx = wg.Context(dv, 4, 1)
+    gid = torch.full((1,), ctx.add_grammar(g), dtype=torch.int32, device="cuda")
+    sid = torch.full((1,), g.start_state, dtype=torch.int32, device="cuda")
+    mask = torch.ones((1, dv.W), dtype=torch.int32, device="cuda")
+    tok = torch.zeros(1, dtype=torch.int32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    wg.wg_decode_step(ctx, gid, sid, torch.zeros((1, vocab.size), device="cuda"), mask, tok, status)
+    assert (mask == 0).all() and tok.item() == -1
+    assert status.item() == wg.binding.WG_ERR_EMPTY_MASK and sid.item() == g.start_state

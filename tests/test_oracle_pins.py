@@ -19,7 +19,7 @@ import pytest
 import oracle
 import regex_ref
 from wg_workloads import (ALL_BYTES, DIGITS, EOS, Cond, DoWhile, IfElse, Sequence, Switch, SymSet,
-                          Wait, WaitUntil, Write, bf16_bits_to_f32, enum_trie, flatten, grammars,
+                          Wait, WaitUntil, Write, WriteTokens, bf16_bits_to_f32, enum_trie, flatten, grammars,
                           make_logits, make_vocab, vocab_from_tokens)
 
 
@@ -473,3 +473,41 @@ def test_wait_until_mask_closed_form(vocab32k):
                 n_cut += 1
         assert bool(got[t]) == want, tok
     assert got.mean() > 0.95
+
+
+# ---------------------------------------------------------------------------------------
+# token-level Write (the paper's own Write: predetermined token sequences)
+# ---------------------------------------------------------------------------------------
+def test_token_level_write_allows_exactly_the_next_token_at_token_boundaries():
+    tokens = [b"a", b"b", b"", b"ab", b"abX", b"X", b"c", b"cd", b"d", b"Xc", b"bX"]
+    vocab = vocab_from_tokens(tokens, eos_id=2)
+    X, EOS_ID, B = tokens.index(b"X"), 2, tokens.index(b"b")
+    tree = tree_of(Sequence(Write(b"ab"), WriteTokens([X, EOS_ID, B]), Write(b"cd")))
+
+    def allowed(cursor):
+        return [tokens[t] if t != 2 else b"<eos>" for t in
+                np.flatnonzero(unpack(oracle.mask(tree, vocab, cursor), vocab.size))]
+
+    c = tree.start()
+    # "abX" spells the literal and the forced token's bytes, but runs INTO the forced part
+    assert allowed(c) == [b"a", b"ab"]
+    rc, c1 = oracle.advance(tree, vocab, c, tokens.index(b"a"))
+    assert rc == 0 and allowed(c1) == [b"b"]                 # "bX" would run into it as well
+    rc, c = oracle.advance(tree, vocab, c, tokens.index(b"ab"))
+    assert rc == 0 and allowed(c) == [b"X"]                  # not "Xc": whole token X only
+    rc, c = oracle.advance(tree, vocab, c, X)
+    assert rc == 0 and allowed(c) == [b"<eos>"]              # the EOS id as a forced token
+    rc, c = oracle.advance(tree, vocab, c, EOS_ID)
+    assert rc == 0 and allowed(c) == [b"b"]
+    rc, bad = oracle.advance(tree, vocab, c, tokens.index(b"a"))
+    assert rc == oracle.ERR_REJECTED and bad == c
+    rc, c = oracle.advance(tree, vocab, c, B)
+    assert rc == 0 and allowed(c) == [b"c", b"cd"]           # byte level again
+    rc, c = oracle.advance(tree, vocab, c, tokens.index(b"cd"))
+    assert rc == 0 and allowed(c) == [b"<eos>"]
+    # a symbol can never enter a forced token
+    forced_cursor = tree.walk(tree.start(), list(b"ab"))
+    assert oracle.is_dead(tree.step(forced_cursor, ord("X")))
+    # an id beyond the vocabulary allows nothing
+    lone = tree_of(WriteTokens([99]))
+    assert not oracle.mask(lone, vocab, lone.start()).any()

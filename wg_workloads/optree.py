@@ -24,6 +24,7 @@ Per kind:
   SWITCH    sets     = [allow, deny, case_0..case_k-1]; children = [body_0..body_k-1]
   DOWHILE   sets     = [allow, deny, true, false];      children = [body]
   WAIT_UNTIL sets    = [allow, deny]; data = the string waited for; children = [body]
+  WRITE_TOKENS data  = the forced token ids, 4 little-endian bytes each
 
 IfElse is the two-case SWITCH: case_0 = true_waits -> if_body, case_1 =
 false_waits -> else_body.
@@ -45,6 +46,7 @@ KIND_WAIT = 2
 KIND_SWITCH = 3
 KIND_DOWHILE = 4
 KIND_WAIT_UNTIL = 5
+KIND_WRITE_TOKENS = 6
 
 SymbolsLike = Union[bytes, str, Iterable[int], "SymSet"]
 
@@ -144,6 +146,13 @@ class Wait(Op):
         self.allow = SymSet(self.allow)
         self.wait = SymSet(self.wait)
         self.deny = SymSet(self.deny)
+
+
+@dataclass
+class WriteTokens(Op):
+    """The paper's token-level Write: exactly these token ids, one per decode step."""
+
+    tokens: List[int]
 
 
 @dataclass
@@ -273,6 +282,13 @@ def flatten(root: Op) -> FlatTree:
             idx = new_node(KIND_WAIT)
             add_sets(idx, [op.allow, op.deny, op.wait])
             kids = [op.body]
+        elif isinstance(op, WriteTokens):
+            idx = new_node(KIND_WRITE_TOKENS)
+            raw = np.asarray(op.tokens, dtype="<i4").tobytes()
+            nodes[idx][5] = len(data)
+            nodes[idx][6] = len(raw)
+            data.extend(raw)
+            kids = []
         elif isinstance(op, WaitUntil):
             idx = new_node(KIND_WAIT_UNTIL)
             add_sets(idx, [op.allow, op.deny])
