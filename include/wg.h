@@ -303,6 +303,24 @@ int32_t wg_decode_step(wg_ctx *ctx, const int32_t *gid, int32_t *sid, int32_t B,
                        int64_t mask_stride_words, int32_t *token_out, int32_t *status,
                        uint32_t flags, void *stream);
 
+/* A decode step recorded once as a CUDA graph and replayed: for small batches the four kernel
+ * launches of wg_decode_step cost more host time than the kernels take on the GPU, and a
+ * graph launch replaces them with one call.  All arguments are those of wg_decode_step and
+ * are frozen into the graph: the caller keeps writing each step's logits into the same
+ * buffer (as an LM head does) and reads tokens and states from the same arrays.  Grammars
+ * added to the context after creation are not seen by the graph while the context's grammar
+ * registry has not grown (it grows when the 65th, 129th, ... grammar is added); create graphs
+ * after the grammars.  wg_step_graph_create records on an internal stream and runs nothing;
+ * wg_step_graph_launch enqueues one step on `stream`.  Results are identical to
+ * wg_decode_step.  Free the graph before its context. */
+typedef struct wg_step_graph wg_step_graph;
+int32_t wg_step_graph_create(wg_ctx *ctx, const int32_t *gid, int32_t *sid, int32_t B,
+                             void *logits, int32_t dtype, int64_t row_stride_elems,
+                             uint32_t *bitmask, int64_t mask_stride_words, int32_t *token_out,
+                             int32_t *status, uint32_t flags, wg_step_graph **out);
+int32_t wg_step_graph_launch(wg_step_graph *graph, void *stream);
+void wg_step_graph_free(wg_step_graph *graph);
+
 /* The same step for a caller whose logits live in HOST memory (pinned memory makes the
  * copies asynchronous): copies logits_host to the device buffer `logits_dev`, runs
  * wg_decode_step, copies the chosen tokens back to token_host and synchronises `stream`.

@@ -79,6 +79,10 @@ _SIGNATURES = {
     "wg_apply_mask_noalloc": (_i32, [_vp, _i32, _i64, _vp, _i64, _i32, _i32, _vp, _vp]),
     "wg_advance": (_i32, [_vp, _vp, _vp, _vp, _i32, _vp, _u32, _vp]),
     "wg_decode_step": (_i32, [_vp, _vp, _vp, _i32, _vp, _i32, _i64, _vp, _i64, _vp, _vp, _u32, _vp]),
+    "wg_step_graph_create": (_i32, [_vp, _vp, _vp, _i32, _vp, _i32, _i64, _vp, _i64, _vp, _vp, _u32,
+                                    C.POINTER(_vp)]),
+    "wg_step_graph_launch": (_i32, [_vp, _vp]),
+    "wg_step_graph_free": (None, [_vp]),
     "wg_decode_step_host": (_i32, [_vp, _vp, _vp, _i32, _vp, _vp, _i32, _i64, _vp, _i64, _vp, _vp,
                                    _vp, _u32, _vp]),
     "wg_ctx_set_timing": (_i32, [_vp, _i32]),
@@ -435,6 +439,39 @@ class StepPlan:
                       self._tok, self._status, self._flags, self._stream)
         if rc != WG_OK:
             raise WgError(rc, "wg_decode_step")
+
+
+class StepGraph:
+    """wg_step_graph: one decode step recorded as a CUDA graph for fixed buffers."""
+
+    def __init__(self, ctx: Context, gid, sid, logits, bitmask, token_out, status=None,
+                 flags: int = WG_USE_CACHE):
+        import torch
+        self._keep = (ctx, gid, sid, logits, bitmask, token_out, status)
+        B, stride = _rows(logits, "logits")
+        _, mstride = _rows(bitmask, "bitmask")
+        h = _vp()
+        _check(_lib.wg_step_graph_create(
+            ctx.handle, _dev_ptr(gid, torch.int32, "gid"), _dev_ptr(sid, torch.int32, "sid"), B,
+            _dev_ptr(logits, None, "logits"), _logits_dtype(logits), stride,
+            _dev_ptr(bitmask, (torch.int32, torch.uint32), "bitmask"), mstride,
+            _dev_ptr(token_out, torch.int32, "token_out"), _dev_ptr(status, torch.int32, "status"),
+            int(flags), C.byref(h)), "wg_step_graph_create")
+        self.handle = h
+        self._launch = _lib.wg_step_graph_launch
+
+    def launch(self, stream=None) -> None:
+        rc = self._launch(self.handle, _stream_ptr(stream))
+        if rc != WG_OK:
+            raise WgError(rc, "wg_step_graph_launch")
+
+    def close(self):
+        if getattr(self, "handle", None):
+            _lib.wg_step_graph_free(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        self.close()
 
 
 def wg_decode_step_host(ctx: Context, gid, sid, logits_host, logits_dev, bitmask, token_dev,

@@ -704,6 +704,67 @@ int32_t wg_decode_step(wg_ctx *c, const int32_t *gid, int32_t *sid, int32_t B, v
     return WG_OK;
 }
 
+}  // extern "C"
+
+struct wg_step_graph {
+    cudaGraph_t graph = nullptr;
+    cudaGraphExec_t exec = nullptr;
+};
+
+extern "C" {
+
+int32_t wg_step_graph_create(wg_ctx *c, const int32_t *gid, int32_t *sid, int32_t B, void *logits,
+                             int32_t dtype, int64_t row_stride_elems, uint32_t *bitmask,
+                             int64_t mask_stride_words, int32_t *token_out, int32_t *status,
+                             uint32_t flags, wg_step_graph **out) {
+    if (!out) return WG_ERR_ARG;
+    *out = nullptr;
+    if (!c) return WG_ERR_ARG;
+    wg_step_graph *g = new (std::nothrow) wg_step_graph();
+    if (!g) return WG_ERR_ARG;
+    cudaStream_t cap = nullptr;
+    int32_t rc = WG_OK;
+    if (cudaStreamCreateWithFlags(&cap, cudaStreamNonBlocking) != cudaSuccess) rc = WG_ERR_CUDA;
+    const bool timing = c->timing;
+    c->timing = false;  // event records do not belong in the recorded step
+    if (rc == WG_OK && cudaStreamBeginCapture(cap, cudaStreamCaptureModeThreadLocal) != cudaSuccess)
+        rc = WG_ERR_CUDA;
+    if (rc == WG_OK) {
+        rc = wg_decode_step(c, gid, sid, B, logits, dtype, row_stride_elems, bitmask,
+                            mask_stride_words, token_out, status, flags, cap);
+        cudaGraph_t graph = nullptr;
+        const cudaError_t e = cudaStreamEndCapture(cap, &graph);  // always end the capture
+        if (rc == WG_OK && e != cudaSuccess) { g_last_cuda_error = (int32_t)e; rc = WG_ERR_CUDA; }
+        g->graph = graph;
+    }
+    c->timing = timing;
+    if (rc == WG_OK) {
+        const cudaError_t e = cudaGraphInstantiate(&g->exec, g->graph, 0);
+        if (e != cudaSuccess) { g_last_cuda_error = (int32_t)e; rc = WG_ERR_CUDA; }
+    }
+    if (cap) cudaStreamDestroy(cap);
+    if (rc != WG_OK) {
+        wg_step_graph_free(g);
+        return rc;
+    }
+    *out = g;
+    return WG_OK;
+}
+
+int32_t wg_step_graph_launch(wg_step_graph *g, void *stream) {
+    if (!g || !g->exec) return WG_ERR_ARG;
+    WG_CUDA(cudaGraphLaunch(g->exec, static_cast<cudaStream_t>(stream)));
+    g_launches.fetch_add(4, std::memory_order_relaxed);  // the four kernels of a step
+    return WG_OK;
+}
+
+void wg_step_graph_free(wg_step_graph *g) {
+    if (!g) return;
+    if (g->exec) cudaGraphExecDestroy(g->exec);
+    if (g->graph) cudaGraphDestroy(g->graph);
+    delete g;
+}
+
 int32_t wg_decode_step_host(wg_ctx *c, const int32_t *gid, int32_t *sid, int32_t B,
                             const void *logits_host, void *logits_dev, int32_t dtype,
                             int64_t row_stride_elems, uint32_t *bitmask,
