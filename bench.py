@@ -32,6 +32,8 @@ from wg_workloads import BY_NAME, flatten, has_structural_byte, make_logits, mak
 # dram__bytes_read.sum + dram__bytes_write.sum of ONE launch of the dominant kernel, from the ncu
 # capture summarised under profiles/ (same launch shape as the timed run).  Set an entry to None
 # when its kernel changes and the capture has not been redone.
+BUILD_WARP_INSTR_PER_TOKEN = 0.42  # profiles/build_masks_kernel_cold_templates.md
+
 NCU_TRAFFIC_BYTES = {
     "json_warm": 222.2e6,       # profiles/apply_mask_kernel_json_warm.md
 }
@@ -333,6 +335,7 @@ def run_ours(args, w, steer: float) -> None:
     ctx.set_timing(True)
     timing_pass[0] = True
     kernel_pass_ms = run_steps(min(args.steps, 4096), True)
+    built_timed = ctx.stats()["masks_built"] - stats["masks_built"]
     kt = ctx.get_timing()
     ctx.set_timing(False)
     clocks = sampler.stop() if sampler else {}
@@ -385,10 +388,17 @@ def run_ours(args, w, steer: float) -> None:
                     "timed_by": "CUDA events recorded by the library around the kernel, in a "
                                 "second pass over the same steps"}
     else:
-        tok_per_s = built * V / (kt["build_ms"] * 1e-3) if kt["build_ms"] > 0 else 0.0
-        roofline = {"kernel": "build_masks_kernel", "bound": "alu", "achieved": tok_per_s / 1e9,
-                    "peak": None, "unit": "Gtokens-checked/s", "frac": None, "traffic": None,
-                    "avg_launch_ms": build_ms}
+        # Issue-slot bound of the build kernel: 148 SMs x 4 schedulers x 1 warp instruction per
+        # clock at the sampled SM clock, divided by the warp instructions the kernel spends per
+        # token checked (ncu: 16.3 M instructions for 256 x 151 936 tokens = 0.42 per token).
+        sm_mhz = clocks.get("sm_mhz") or 1965.0
+        peak_tok = 148 * 4 * sm_mhz * 1e6 / BUILD_WARP_INSTR_PER_TOKEN
+        tok_per_s = built_timed * V / (kt["build_ms"] * 1e-3) if kt["build_ms"] > 0 else 0.0
+        roofline = {"kernel": "build_masks_kernel (+ row reset)", "bound": "alu",
+                    "achieved": tok_per_s / 1e9, "peak": peak_tok / 1e9,
+                    "unit": "G tokens checked/s", "frac": tok_per_s / peak_tok,
+                    "peak_kind": "issue slots at the kernel's measured instructions per token",
+                    "traffic": None, "avg_launch_ms": build_ms}
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
