@@ -137,7 +137,7 @@ class OracleRun:
         self.oracle = oracle
         self.w, self.rows, self.steer = w, rows, steer
         self.vocab = make_vocab(w.V, w.vocab_seed)
-        self.bonus = has_structural_byte(self.vocab)
+        self.bonus = has_structural_byte(self.vocab, w.steer_bytes)
         n_gram = len({w.grammar_of_row(r) for r in range(rows)})
         self.trees = {}
         for r in range(rows):
@@ -266,7 +266,7 @@ def run_ours(args, w, steer: float) -> None:
     ring = args.ring or int(max(4, min(64, args.steps + args.warmup, (20 << 30) // (B * row_bytes))))
     gen = torch.Generator(device="cuda")
     gen.manual_seed(1234 + 7919 * rank)
-    bonus = torch.from_numpy(has_structural_byte(vocab)).cuda().to(torch.float32) * steer
+    bonus = torch.from_numpy(has_structural_byte(vocab, w.steer_bytes)).cuda().to(torch.float32) * steer
     pristine = []
     for _ in range(ring):
         x = torch.randn((B, V), generator=gen, device="cuda", dtype=torch.float32) * 2.0

@@ -23,6 +23,14 @@
  *     the wg_ctx was created, and must stay valid until the work queued on `stream` is done.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Device
  *     calls only enqueue work; they do not synchronise unless stated.
+ *   - A wg_ctx keeps per-call scratch: calls on one context must be issued from one thread at
+ *     a time and on one stream at a time (or on streams ordered by events).  Use one context
+ *     per concurrent stream; vocabularies and compiled grammars may be shared between them.
+ *   - Every object belongs to the CUDA device that was current when it was created; make
+ *     that device current before calling into it.
+ *   - The cache never evicts: when its pool is full, further new states are built straight
+ *     into the caller's bitmask on every step (counted as rows_uncached) until
+ *     wg_cache_clear is called.
  *   - Per-row problems found on the device (a refused token, an empty mask, an unknown
  *     state) are written to the optional per-row status array and counted in wg_stats; they
  *     never fault the GPU.

@@ -21,6 +21,15 @@ class Workload:
     n_grammars: int
     description: str
 
+    @property
+    def steer_bytes(self) -> bytes:
+        """Characters whose tokens get the steering bonus (empty = all structural ones).
+
+        The snippet workload only favours '<': a row then leaves a free-text slot on its next
+        step, so leaders keep meeting new states and the cache hit rate comes from the
+        followers (about one half), as the workload asks."""
+        return b"<" if self.name == "dynamic_snippets" else b""
+
     def grammar(self, g: int) -> Op:
         return _GRAMMARS[self.name](g)
 

@@ -115,10 +115,13 @@ def make_vocab(V: int, seed: int, eos_id: int = EOS_ID) -> Vocab:
     return vocab_from_tokens(tokens, eos_id)
 
 
-def has_structural_byte(vocab: Vocab) -> np.ndarray:
-    """bool [V]: the token contains one of the structural characters (input shaping only)."""
+def has_structural_byte(vocab: Vocab, chars: bytes = b"") -> np.ndarray:
+    """bool [V]: the token contains one of ``chars`` (default: the structural characters).
+
+    Input shaping only: the benchmark and the tests add a constant to the logits of these tokens
+    so that greedy decoding leaves free-text slots."""
     is_struct = np.zeros(256, dtype=bool)
-    is_struct[STRUCTURAL] = True
+    is_struct[np.frombuffer(chars, dtype=np.uint8) if chars else STRUCTURAL] = True
     hit = is_struct[vocab.data]
     csum = np.zeros(vocab.data.shape[0] + 1, dtype=np.int64)
     csum[1:] = np.cumsum(hit)
