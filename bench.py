@@ -56,6 +56,8 @@ def parse_args():
                    help="bonus added to tokens holding a structural character")
     p.add_argument("--graph", action="store_true",
                    help="replay each step as a recorded CUDA graph (small batches)")
+    p.add_argument("--separate", action="store_true",
+                   help="call wg_build_masks / wg_apply_mask / wg_advance instead of wg_decode_step")
     p.add_argument("--no-cpu-baseline", action="store_true")
     p.add_argument("--no-e2e", action="store_true")
     p.add_argument("--cpu-seconds", type=float, default=12.0)
@@ -296,8 +298,15 @@ def run_ours(args, w, steer: float) -> None:
                   for wbuf in work]
         stream_ptr = torch.cuda.current_stream()
 
+    ws = torch.empty(wg.wg_apply_workspace_bytes(B), dtype=torch.uint8, device="cuda")
+
     def step(i):
-        if graphs is not None and not timing_pass[0]:
+        if args.separate:
+            # the same step through the individual entry points (7 launches instead of 4)
+            wg.wg_build_masks(ctx, d_gid, d_sid, d_mask, flags & wg.WG_NO_CACHE)
+            wg.wg_apply_mask(work[i % ring], d_mask, V, d_tok, ws)
+            wg.wg_advance(ctx, d_gid, d_sid, d_tok, d_status, flags & wg.WG_RESTART_ON_DONE)
+        elif graphs is not None and not timing_pass[0]:
             graphs[i % ring].launch(stream_ptr)
         else:
             plan(work[i % ring])
@@ -405,7 +414,8 @@ def run_ours(args, w, steer: float) -> None:
         "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
         "config": {"workload": w.name, "V": V, "batch_per_gpu": B, "logits": w.dtype,
-                   "states": n_states, "launch": "cuda graph" if args.graph else "stream", "cache": "prewarmed" if w.prewarm else
+                   "states": n_states, "launch": "separate calls" if args.separate else
+                   ("cuda graph" if args.graph else "stream"), "cache": "prewarmed" if w.prewarm else
                    ("on" if w.use_cache else "off"), "steer": steer, "ring": ring,
                    "l2": "inputs larger than L2" if B * row_bytes > (126 << 20) else
                    "ring of distinct buffers; working set may sit in L2",

@@ -163,3 +163,14 @@ def test_token_level_write_states_follow_the_checker_token_by_token(wg):
     with pytest.raises(wg.WgError) as e:
         wg.Grammar(bad)
     assert e.value.status == wg.binding.WG_ERR_GRAMMAR
+
+
+def test_header_compiles_as_plain_c(tmp_path):
+    import subprocess
+    src = tmp_path / "use_wg.c"
+    src.write_text('#include "wg.h"\n'
+                   'int probe(void) { wg_stats s; wg_op_node n; (void)s; (void)n;\n'
+                   '  return WG_OK + WG_DTYPE_BF16 + WG_OP_WRITE_TOKENS + (int)sizeof(wg_op_node); }\n')
+    subprocess.check_call(["gcc", "-std=c99", "-Wall", "-Wextra", "-Werror", "-pedantic", "-c",
+                           "-I", os.path.join(ROOT, "include"), str(src), "-o",
+                           str(tmp_path / "use_wg.o")])

@@ -542,3 +542,37 @@ def test_forced_token_beyond_the_vocabulary_gives_an_empty_mask(wg, torch):
     wg.wg_decode_step(ctx, gid, sid, torch.zeros((1, vocab.size), device="cuda"), mask, tok, status)
     assert (mask == 0).all() and tok.item() == -1
     assert status.item() == wg.binding.WG_ERR_EMPTY_MASK and sid.item() == g.start_state
+
+
+def test_large_batch_stats_reset_and_kernel_timing(wg, torch):
+    vocab = make_vocab(2048, seed=15)
+    flat = flatten(grammars.json_reference_lookup(doc_nodes=40))
+    tree, g = oracle.Tree(flat), wg.Grammar(flat)
+    dv = wg.Vocab(vocab.offsets, vocab.data, vocab.eos_id)
+    B = 3000                                       # several passes of the one-block lookup kernel
+    ctx = wg.Context(dv, 512, B)
+    gid = torch.full((B,), ctx.add_grammar(g), dtype=torch.int32, device="cuda")
+    cursor_of = co_reachable(tree, g, mentioned_symbols(flat))
+    sids = sorted(cursor_of)
+    rows = np.array([sids[(7 * r) % len(sids)] for r in range(B)], np.int32)
+    sid = to_dev(torch, rows)
+    mask = torch.zeros((B, dv.W), dtype=torch.int32, device="cuda")
+    tok = torch.zeros(B, dtype=torch.int32, device="cuda")
+    status = torch.zeros(B, dtype=torch.int32, device="cuda")
+    host = make_logits(B, vocab.size, "bf16", [15, 0], 0)
+    want_masks = {s: oracle.mask(tree, vocab, cursor_of[s]) for s in set(rows.tolist())}
+    ctx.set_timing(True)
+    wg.wg_decode_step(ctx, gid, sid, dev_logits(torch, host, "bf16"), mask, tok, status)
+    t = ctx.get_timing()
+    assert t["steps"] == 1 and t["apply_ms"] > 0 and t["build_ms"] > 0
+    assert ctx.get_timing()["steps"] == 0             # reading forgets the recorded steps
+    ctx.set_timing(False)
+    got = mask.cpu().numpy().view(np.uint32)
+    want = np.stack([want_masks[s] for s in rows.tolist()])
+    assert (got == want).all()
+    assert (tok.cpu().numpy() == oracle.argmax(host, want, vocab.size)).all()
+    st = ctx.stats()
+    assert st["cache_misses"] == len(set(rows.tolist())) == st["masks_built"]
+    assert st["cache_hits"] == B - st["cache_misses"]
+    ctx.reset_stats()
+    assert all(v == 0 for k, v in ctx.stats().items() if k != "cache_entries")
