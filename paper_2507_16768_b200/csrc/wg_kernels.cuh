@@ -295,6 +295,9 @@ cache_lookup_insert_kernel(CtxDev ctx, const int32_t *gid, const int32_t *sid, i
             for (int probe = 0; probe < ctx.hash_size; ++probe, h = (h + 1) & mask) {
                 unsigned long long k = ctx.keys[h];
                 if (k == 0) {
+                    // a full pool takes no new keys, so the table never fills up with states
+                    // it cannot serve (the row is then built uncached)
+                    if (*(volatile int32_t *)ctx.n_slots >= ctx.capacity) break;
                     k = atomicCAS(&ctx.keys[h], 0ull, key);
                     if (k == 0) {  // this thread owns the new entry
                         const int32_t row = atomicAdd(ctx.n_slots, 1);
