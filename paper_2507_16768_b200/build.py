@@ -13,7 +13,7 @@ SOURCES = ["wg_api.cu", "wg_lower.cpp", "wg_regex.cpp"]
 HEADERS = [os.path.join(CSRC, "wg_kernels.cuh"), os.path.join(CSRC, "wg_internal.h"),
            os.path.join(ROOT, "include", "wg.h")]
 NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
-              "-Xcompiler", "-fPIC", "-shared", "-cudart", "shared"]
+              "-Xcompiler", "-fPIC", "-shared", "-cudart", "shared", "-ldl"]
 
 
 def _nvcc() -> str:
