@@ -511,3 +511,19 @@ def test_token_level_write_allows_exactly_the_next_token_at_token_boundaries():
     # an id beyond the vocabulary allows nothing
     lone = tree_of(WriteTokens([99]))
     assert not oracle.mask(lone, vocab, lone.start()).any()
+
+
+def test_golden_fixture_of_the_section_3_2_listing():
+    import os
+    path = os.path.join(os.path.dirname(__file__), "golden", "section_3_2_listing_language.txt")
+    tree = tree_of(grammars.paper_listing_example())
+    n = 0
+    for line in open(path):
+        line = line.rstrip("\n")
+        if not line or line.startswith("#"):
+            continue
+        verdict, text = line.split(" ", 1)
+        text = "" if text == "<empty>" else text
+        assert tree.accepts([ord(c) for c in text] + [EOS]) is (verdict == "accept"), line
+        n += 1
+    assert n >= 15

@@ -131,3 +131,17 @@ def test_patterns_outside_the_dialect_are_refused_with_a_reason(wg, pattern, why
         wg.Grammar.from_regex(pattern)
     assert e.value.status == wg.binding.WG_ERR_GRAMMAR
     assert why in str(e.value), str(e.value)
+
+
+def test_golden_fixture_through_the_regex_front_end(wg):
+    import os
+    path = os.path.join(os.path.dirname(__file__), "golden", "section_3_2_listing_language.txt")
+    g = wg.Grammar.from_regex(r"\d+(\.\d+)*")
+    for line in open(path):
+        line = line.rstrip("\n")
+        if not line or line.startswith("#"):
+            continue
+        verdict, text = line.split(" ", 1)
+        text = "" if text == "<empty>" else text
+        end = g.walk(g.start_state, [ord(c) for c in text] + [EOS])
+        assert (end == g.done_state) is (verdict == "accept"), line
