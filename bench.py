@@ -219,6 +219,9 @@ def run_ours(args, w, steer: float) -> None:
     import torch
     import torch.distributed as dist
 
+    from paper_2507_16768_b200 import build as lib_build
+    if int(os.environ.get("LOCAL_RANK", "0")) == 0:
+        lib_build.ensure()          # one rank builds if the library is missing
     import paper_2507_16768_b200 as wg
     from paper_2507_16768_b200.sharding import max_over_ranks
 

@@ -41,5 +41,18 @@ def build(force: bool = False, verbose: bool = False) -> str:
     return LIB
 
 
+def ensure() -> str:
+    """The library, built if it is missing; a library that only looks older than its sources
+    (file times change when a tree is copied) is rebuilt when nvcc is there and kept otherwise."""
+    if not os.path.exists(LIB):
+        return build(force=True)
+    if needs_build():
+        try:
+            return build(force=True)
+        except (OSError, subprocess.CalledProcessError):
+            pass
+    return LIB
+
+
 if __name__ == "__main__":
     print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))

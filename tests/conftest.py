@@ -27,3 +27,10 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(scope="session", autouse=True)
+def _built_library():
+    """The tests load libwg.so through the binding; build it first if that is needed."""
+    from paper_2507_16768_b200 import build
+    build.ensure()
