@@ -188,6 +188,15 @@ void wg_optree_free(wg_optree *tree);
 int32_t wg_compile_regex(const char *pattern, int32_t length, wg_grammar **out);
 const char *wg_regex_error(void);
 
+/* Returns in *out a grammar with the same language in which states that behave alike are
+ * merged (classical DFA minimisation by partition refinement).  The paper caches masks per
+ * operator state (Section 3.3); merged states share one cached mask, and grammars that
+ * repeat a tail (enum entries with a common ending, the tails a regular expression's
+ * alternatives carry) shrink a lot.  State ids change: states taken from the input grammar
+ * do not carry over.  Host side; cost about n_states * n_classes * log(n_states) per round of
+ * refinement.  The input is left as it is; free both. */
+int32_t wg_grammar_minimize(const wg_grammar *grammar, wg_grammar **out);
+
 /* Host-side facts about a compiled grammar.  Any output pointer may be NULL.
  * content_hash identifies the table: two compilations with equal tables hash equally. */
 int32_t wg_grammar_info(const wg_grammar *grammar, int32_t *n_states, int32_t *start_state,

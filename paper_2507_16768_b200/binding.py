@@ -54,6 +54,7 @@ _SIGNATURES = {
     "wg_vocab_free": (None, [_vp]),
     "wg_compile_grammar": (_i32, [_vp, _i32, _vp, _i32, _vp, _i32, _vp, _i32, _i32, C.POINTER(_vp)]),
     "wg_grammar_free": (None, [_vp]),
+    "wg_grammar_minimize": (_i32, [_vp, C.POINTER(_vp)]),
     "wg_regex_to_optree": (_i32, [C.c_char_p, _i32, C.POINTER(_vp)]),
     "wg_optree_sizes": (_i32, [_vp, C.POINTER(_i32), C.POINTER(_i32), C.POINTER(_i32),
                                C.POINTER(_i32), C.POINTER(_i32)]),
@@ -225,6 +226,12 @@ class Grammar:
         if rc != WG_OK:
             raise WgError(rc, "wg_compile_regex: " + _lib.wg_regex_error().decode())
         return cls(_handle=h)
+
+    def minimized(self) -> "Grammar":
+        """wg_grammar_minimize: the same language with equivalent states merged."""
+        h = _vp()
+        _check(_lib.wg_grammar_minimize(self.handle, C.byref(h)), "wg_grammar_minimize")
+        return Grammar(_handle=h)
 
     def step(self, state: int, symbol: int) -> int:
         return int(_lib.wg_grammar_step(self.handle, int(state), int(symbol)))

@@ -253,6 +253,25 @@ int32_t wg_compile_grammar(const wg_op_node *nodes, int32_t n_nodes, const int32
 
 void wg_grammar_free(wg_grammar *g) { delete g; }
 
+int32_t wg_grammar_minimize(const wg_grammar *g, wg_grammar **out) {
+    if (!g || !out) return WG_ERR_ARG;
+    *out = nullptr;
+    wg_grammar *m = new (std::nothrow) wg_grammar();
+    if (!m) return WG_ERR_ARG;
+    int32_t rc;
+    try {
+        rc = wg_minimize_grammar(*g, m);
+    } catch (const std::bad_alloc &) {
+        rc = WG_ERR_CAPACITY;
+    }
+    if (rc != WG_OK) {
+        delete m;
+        return rc;
+    }
+    *out = m;
+    return WG_OK;
+}
+
 int32_t wg_grammar_info(const wg_grammar *g, int32_t *n_states, int32_t *start_state,
                         int32_t *done_state, int32_t *n_classes, uint64_t *content_hash) {
     if (!g) return WG_ERR_ARG;

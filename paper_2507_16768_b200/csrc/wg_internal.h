@@ -30,6 +30,9 @@ struct wg_grammar {
     uint64_t hash = 0;
 };
 
+// Merges states with equal behaviour (wg_lower.cpp).  out may not alias in.
+int32_t wg_minimize_grammar(const wg_grammar &in, wg_grammar *out);
+
 // Lowering entry (wg_lower.cpp).
 int32_t wg_lower_tree(const wg_op_node *nodes, int32_t n_nodes, const int32_t *children,
                       int32_t n_children, const uint32_t *sets, int32_t n_sets,

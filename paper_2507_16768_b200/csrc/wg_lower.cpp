@@ -226,6 +226,21 @@ uint64_t fnv1a(uint64_t h, const void *p, size_t n) {
     return h;
 }
 
+uint64_t content_hash(const wg_grammar &g) {
+    uint64_t h = 0xCBF29CE484222325ull;
+    if (!g.forced_tok.empty()) {
+        h = fnv1a(h, g.forced_tok.data(), g.forced_tok.size() * sizeof(int32_t));
+        h = fnv1a(h, g.forced_next.data(), g.forced_next.size() * sizeof(int32_t));
+    }
+    h = fnv1a(h, &g.n_states, 4);
+    h = fnv1a(h, &g.n_classes, 4);
+    h = fnv1a(h, &g.done, 4);
+    h = fnv1a(h, &g.eos_class, 4);
+    h = fnv1a(h, g.byte_class, 256);
+    h = fnv1a(h, g.table.data(), g.table.size() * sizeof(int32_t));
+    return h;
+}
+
 }  // namespace
 
 int32_t wg_lower_tree(const wg_op_node *nodes, int32_t n_nodes, const int32_t *children,
@@ -363,17 +378,84 @@ int32_t wg_lower_tree(const wg_op_node *nodes, int32_t n_nodes, const int32_t *c
             out->forced_next[i] = new_id[lw.forced_next[order[i]]];
         }
     }
-    uint64_t h = 0xCBF29CE484222325ull;
-    if (any_forced) {
-        h = fnv1a(h, out->forced_tok.data(), out->forced_tok.size() * sizeof(int32_t));
-        h = fnv1a(h, out->forced_next.data(), out->forced_next.size() * sizeof(int32_t));
+    out->hash = content_hash(*out);
+    return WG_OK;
+}
+
+// Moore's partition refinement: start from {DEAD}, {DONE}, the forced-token states grouped by
+// token id, and everything else; split blocks by the blocks their transitions lead to until
+// nothing splits any more.  States of one final block accept the same continuations, so they
+// get one state (and one cached mask) in the output.
+int32_t wg_minimize_grammar(const wg_grammar &in, wg_grammar *out) {
+    const int32_t S = in.n_states, C = in.n_classes;
+    const bool forced = !in.forced_tok.empty();
+    std::vector<int32_t> block(S, 0);
+    int32_t n_blocks = 0;
+    {
+        std::unordered_map<int64_t, int32_t> first;
+        for (int32_t s = 0; s < S; ++s) {
+            int64_t key = s == 0 ? -1 : (s == in.done ? -2 : -3);
+            if (s != 0 && forced && in.forced_tok[s] >= 0) key = in.forced_tok[s];
+            auto it = first.find(key);
+            if (it == first.end()) it = first.emplace(key, n_blocks++).first;
+            block[s] = it->second;
+        }
     }
-    h = fnv1a(h, &out->n_states, 4);
-    h = fnv1a(h, &out->n_classes, 4);
-    h = fnv1a(h, &out->done, 4);
-    h = fnv1a(h, &out->eos_class, 4);
-    h = fnv1a(h, out->byte_class, 256);
-    h = fnv1a(h, out->table.data(), out->table.size() * sizeof(int32_t));
-    out->hash = h;
+    const int width = C + 2;
+    std::vector<int32_t> sig((size_t)S * width);
+    std::vector<int32_t> order(S), next_block(S);
+    for (;;) {
+        for (int32_t s = 0; s < S; ++s) {
+            int32_t *row = &sig[(size_t)s * width];
+            row[0] = block[s];
+            for (int32_t c = 0; c < C; ++c) row[1 + c] = block[in.table[(size_t)s * C + c]];
+            row[1 + C] = (forced && in.forced_tok[s] >= 0) ? block[in.forced_next[s]] : -1;
+        }
+        for (int32_t s = 0; s < S; ++s) order[s] = s;
+        std::sort(order.begin(), order.end(), [&](int32_t a, int32_t b) {
+            const int cmp = memcmp(&sig[(size_t)a * width], &sig[(size_t)b * width], sizeof(int32_t) * width);
+            return cmp != 0 ? cmp < 0 : a < b;
+        });
+        int32_t n_next = 0;
+        for (int32_t i = 0; i < S; ++i) {
+            if (i > 0 && memcmp(&sig[(size_t)order[i] * width], &sig[(size_t)order[i - 1] * width],
+                                sizeof(int32_t) * width) != 0)
+                ++n_next;
+            next_block[order[i]] = n_next;
+        }
+        ++n_next;
+        block.swap(next_block);
+        if (n_next == n_blocks) break;  // refinement only splits: an equal count is a fixpoint
+        n_blocks = n_next;
+    }
+    // new ids in order of first appearance (the input is numbered breadth-first from the start
+    // state, so locality survives); DEAD stays 0
+    std::vector<int32_t> new_id(n_blocks, -1), rep;
+    rep.reserve(n_blocks);
+    for (int32_t s = 0; s < S; ++s)
+        if (new_id[block[s]] < 0) { new_id[block[s]] = (int32_t)rep.size(); rep.push_back(s); }
+    const int32_t M = (int32_t)rep.size();
+    out->n_states = M;
+    out->n_classes = C;
+    out->start = new_id[block[in.start]];
+    out->done = new_id[block[in.done]];
+    out->eos_class = in.eos_class;
+    memcpy(out->byte_class, in.byte_class, sizeof(in.byte_class));
+    out->table.assign((size_t)M * C, 0);
+    for (int32_t m = 0; m < M; ++m)
+        for (int32_t c = 0; c < C; ++c)
+            out->table[(size_t)m * C + c] = new_id[block[in.table[(size_t)rep[m] * C + c]]];
+    out->forced_tok.clear();
+    out->forced_next.clear();
+    if (forced) {
+        out->forced_tok.assign(M, -1);
+        out->forced_next.assign(M, 0);
+        for (int32_t m = 0; m < M; ++m)
+            if (in.forced_tok[rep[m]] >= 0) {
+                out->forced_tok[m] = in.forced_tok[rep[m]];
+                out->forced_next[m] = new_id[block[in.forced_next[rep[m]]]];
+            }
+    }
+    out->hash = content_hash(*out);
     return WG_OK;
 }

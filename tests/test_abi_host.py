@@ -174,3 +174,31 @@ def test_header_compiles_as_plain_c(tmp_path):
     subprocess.check_call(["gcc", "-std=c99", "-Wall", "-Wextra", "-Werror", "-pedantic", "-c",
                            "-I", os.path.join(ROOT, "include"), str(src), "-o",
                            str(tmp_path / "use_wg.o")])
+
+
+@pytest.mark.parametrize("name", ["listing", "html", "json_doc", "template1", "snippets",
+                                  "html_tags", "overlapping_until", "empty_bodies"])
+def test_minimized_grammar_keeps_the_language(wg, name):
+    flat = flatten(GRAMMARS[name]())
+    tree = oracle.Tree(flat)
+    g = wg.Grammar(flat)
+    m = g.minimized()
+    assert m.n_states <= g.n_states and m.start_state == 1
+    symbols = range(257) if flat.n_nodes < 60 else mentioned_symbols(flat)
+    cursor_of = co_reachable(tree, m, symbols)          # checks every transition against the checker
+    assert sorted(cursor_of) == list(range(1, m.n_states))
+    assert cursor_of[m.done_state] == oracle.DONE
+    again = m.minimized()
+    assert again.n_states == m.n_states and again.content_hash == m.content_hash
+
+
+def test_minimization_merges_repeated_tails(wg):
+    g = wg.Grammar(flatten(grammars.json_reference_lookup()))
+    assert g.minimized().n_states < g.n_states // 4
+    r = wg.Grammar.from_regex(r"(a\d*|b)c(x|y)?z")      # the front end copies tails into branches
+    assert r.minimized().n_states < r.n_states
+    # forced tokens stay apart by token id
+    t = wg.Grammar(flatten(Sequence(WriteTokens([5, 6, 5, 6]), Write(b"ab"))))
+    m = t.minimized()
+    assert m.n_states == t.n_states
+    assert [m.forced_token(s)[0] for s in range(1, 5)] == [5, 6, 5, 6]

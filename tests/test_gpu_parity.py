@@ -160,11 +160,13 @@ class Sim:
     """One workload driven on both sides: same vocabulary, grammars, logits and tokens."""
 
     def __init__(self, wg, torch, vocab, ops, row_grammar, dtype, cache_capacity, use_cache=True,
-                 seed=0, steer=6.0, delays=None):
+                 seed=0, steer=6.0, delays=None, minimize=False):
         self.wg, self.torch, self.vocab, self.dtype = wg, torch, vocab, dtype
         self.flats = [op if hasattr(op, "nodes") else flatten(op) for op in ops]
         self.trees = [oracle.Tree(f) for f in self.flats]
         self.grams = [wg.Grammar(f) for f in self.flats]
+        if minimize:
+            self.grams = [g.minimized() for g in self.grams]
         self.dv = wg.Vocab(vocab.offsets, vocab.data, vocab.eos_id)
         self.B = len(row_grammar)
         self.ctx = wg.Context(self.dv, cache_capacity, self.B)
@@ -576,3 +578,14 @@ def test_large_batch_stats_reset_and_kernel_timing(wg, torch):
     assert st["cache_hits"] == B - st["cache_misses"]
     ctx.reset_stats()
     assert all(v == 0 for k, v in ctx.stats().items() if k != "cache_entries")
+
+
+def test_trajectory_on_minimized_grammars(wg, torch):
+    vocab = make_vocab(8192, seed=16)
+    ops = [grammars.json_reference_lookup(doc_nodes=200), grammars.dynamic_snippet_template(1, n_args=3, enum_size=12)]
+    sim = Sim(wg, torch, vocab, ops, [0, 1, 0, 1, 0], "bf16", cache_capacity=1024, seed=9, steer=5.0,
+              minimize=True)
+    assert sim.grams[0].n_states < wg.Grammar(sim.flats[0]).n_states
+    for _ in range(50):
+        sim.step()
+    assert len(sim.visited) > 30
