@@ -58,6 +58,8 @@ def parse_args():
                    help="replay each step as a recorded CUDA graph (small batches)")
     p.add_argument("--separate", action="store_true",
                    help="call wg_build_masks / wg_apply_mask / wg_advance instead of wg_decode_step")
+    p.add_argument("--steer-all", action="store_true",
+                   help="steer every structural character (rows then dwell in free-text slots)")
     p.add_argument("--no-cpu-baseline", action="store_true")
     p.add_argument("--no-e2e", action="store_true")
     p.add_argument("--cpu-seconds", type=float, default=12.0)
@@ -271,7 +273,8 @@ def run_ours(args, w, steer: float) -> None:
     ring = args.ring or int(max(4, min(64, args.steps + args.warmup, (20 << 30) // (B * row_bytes))))
     gen = torch.Generator(device="cuda")
     gen.manual_seed(1234 + 7919 * rank)
-    bonus = torch.from_numpy(has_structural_byte(vocab, w.steer_bytes)).cuda().to(torch.float32) * steer
+    steer_bytes = b"" if args.steer_all else w.steer_bytes
+    bonus = torch.from_numpy(has_structural_byte(vocab, steer_bytes)).cuda().to(torch.float32) * steer
     pristine = []
     for _ in range(ring):
         x = torch.randn((B, V), generator=gen, device="cuda", dtype=torch.float32) * 2.0

@@ -391,6 +391,14 @@ int32_t wg_ctx_add_grammar(wg_ctx *c, const wg_grammar *g, int32_t *grammar_id) 
     const bool wide = g->n_states > 65535;
     GrammarSlot slot{g->hash, g->table, g->forced_tok, g->forced_next, g->n_states, g->n_classes,
                      nullptr, nullptr, nullptr, nullptr, nullptr};
+    struct Guard {  // frees the uploads again if any later step fails
+        GrammarSlot *s;
+        ~Guard() {
+            if (!s) return;
+            cudaFree(s->d_table); cudaFree(s->d_cls); cudaFree(s->d_first_ok);
+            cudaFree(s->d_leaves); cudaFree(s->d_forced);
+        }
+    } guard{&slot};
     if (!g->forced_tok.empty()) {
         std::vector<int2> forced(g->n_states);
         for (int32_t st = 0; st < g->n_states; ++st) forced[st] = make_int2(g->forced_tok[st], g->forced_next[st]);
@@ -450,6 +458,7 @@ int32_t wg_ctx_add_grammar(wg_ctx *c, const wg_grammar *g, int32_t *grammar_id) 
     }
     WG_CUDA(cudaMemcpy(c->d_grammars + id, &gd, sizeof(GrammarDev), cudaMemcpyHostToDevice));
     c->grammars.push_back(gd);
+    guard.s = nullptr;  // the context owns the uploads from here on
     c->slots.push_back(std::move(slot));
     c->dev.n_grammars = id + 1;
     *grammar_id = id;
