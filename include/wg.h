@@ -102,7 +102,7 @@ enum {
  *             level such a token is a string.  Accepts text over (allow \ deny) and the
  *             string's own bytes up to and including the FIRST occurrence of the string.)
  *   WRITE_TOKENS data  = the forced token ids, 4 little-endian bytes each (ids >= 0)
- *             (paper Section 3.2: Write "outputs predetermined token sequences"; Section 3.3:
+ *             (paper Section 3.2: Write emits a token sequence fixed in advance; Section 3.3:
  *             a chain of Waits each expecting one token.  Exactly these ids, one per decode
  *             step; entered and left at token boundaries only, so no token's bytes may run
  *             into or out of it.  An id beyond the vocabulary yields an empty mask.) */
@@ -161,8 +161,8 @@ int32_t wg_compile_grammar(const wg_op_node *nodes, int32_t n_nodes, const int32
                            const uint8_t *data, int32_t n_data, int32_t root, wg_grammar **out);
 void wg_grammar_free(wg_grammar *grammar);
 
-/* Regular-expression front end (paper Section 3.2, "From Regular Expressions to Wait/Write
- * Operator Composition"; the syntax-prior path of Section 4.1's "WGrammar (online)").
+/* Regular-expression front end (paper Section 3.2, the paragraph on translating regular
+ * expressions into Wait / Write compositions; the syntax-prior variant evaluated in Section 4.1).
  * Translates a pattern into an operator tree: classes and characters become Wait, literal runs
  * Write, repetition and branching DoWhile / IfElse(Switch) / Sequence, followed by EOS.
  * Dialect (bytes): literals, '.', escapes \d \w \s \D \W \S \n \t \r \f \v \0 \xHH
@@ -246,7 +246,7 @@ int32_t wg_reset_stats(wg_ctx *ctx, void *stream);
 int32_t wg_mask_cache_lookup(wg_ctx *ctx, const int32_t *gid, const int32_t *sid, int32_t B,
                              int32_t *slot, void *stream);
 
-/* Mask creation (paper Section 1 "mask creation", Section 3.3).
+/* Mask creation (paper Section 1, the third stage of constrained decoding; Section 3.3).
  *   gid, sid          device, B entries
  *   bitmask           device, B rows of W words, row r at bitmask + r * row_stride_words
  *   row_stride_words  >= W
@@ -258,7 +258,8 @@ int32_t wg_mask_cache_lookup(wg_ctx *ctx, const int32_t *gid, const int32_t *sid
 int32_t wg_build_masks(wg_ctx *ctx, const int32_t *gid, const int32_t *sid, int32_t B,
                        uint32_t *bitmask, int64_t row_stride_words, uint32_t flags, void *stream);
 
-/* Mask application (paper Section 1: applied to the logits prior to sampling), in place.
+/* Mask application (paper Section 1: the mask acts on the logits before a token is sampled),
+ * in place.
  *   logits            device, B rows of V elements, row r at logits + r * row_stride_elems
  *   dtype             WG_DTYPE_BF16 or WG_DTYPE_FP32
  *   bitmask           device, as written by wg_build_masks

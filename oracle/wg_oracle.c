@@ -26,8 +26,8 @@
  *                                 (Section 3.2: waits are tokens, e.g. a closing tag): any text
  *                                 over (A \ D) and the bytes of u, up to and including the FIRST
  *                                 occurrence of u, then L(body)
- *   WriteTokens(t1..tn)           the paper's own Write (Section 3.2: "outputs predetermined token
- *                                 sequences"; Section 3.3: a chain of Waits each expecting one
+ *   WriteTokens(t1..tn)           the paper's own Write (Section 3.2: it emits a token sequence fixed
+ *                                 in advance; Section 3.3: a chain of Waits each expecting one
  *                                 token): exactly these token ids, one per decode step.  It is
  *                                 entered and left only at token boundaries: no token's bytes
  *                                 may run into it or out of it.

@@ -1,5 +1,5 @@
-// Regular expression -> operator tree (paper Section 3.2, "From Regular Expressions to
-// Wait/Write Operator Composition"; the syntax-prior path the paper calls WGrammar (online)).
+// Regular expression -> operator tree (paper Section 3.2, the paragraph on translating regular
+// expressions into Wait / Write compositions; the syntax-prior variant evaluated in Section 4.1).
 //
 // Character classes and single characters become Wait operators, literal runs become Write,
 // repetition and branching become DoWhile / IfElse(Switch) / Sequence.  Because the operators

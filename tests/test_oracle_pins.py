@@ -476,7 +476,7 @@ def test_wait_until_mask_closed_form(vocab32k):
 
 
 # ---------------------------------------------------------------------------------------
-# token-level Write (the paper's own Write: predetermined token sequences)
+# token-level Write (the paper's own Write: a token sequence fixed in advance)
 # ---------------------------------------------------------------------------------------
 def test_token_level_write_allows_exactly_the_next_token_at_token_boundaries():
     tokens = [b"a", b"b", b"", b"ab", b"abX", b"X", b"c", b"cd", b"d", b"Xc", b"bX"]
