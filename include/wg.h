@@ -197,6 +197,18 @@ const char *wg_regex_error(void);
  * refinement.  The input is left as it is; free both. */
 int32_t wg_grammar_minimize(const wg_grammar *grammar, wg_grammar **out);
 
+/* A compiled grammar as a flat byte blob, so that tables compiled offline can be stored and
+ * loaded at start-up instead of being recompiled (paper Section 3.1: the static structure is
+ * processed once, offline, into an artefact that requests reuse).
+ * wg_grammar_save: writes at most `capacity` bytes to `blob` and always stores the size the
+ *   blob needs in *needed; returns WG_ERR_CAPACITY (nothing written) if capacity is too
+ *   small, so a first call with blob = NULL, capacity = 0 asks for the size.
+ * wg_grammar_load: rebuilds a grammar from such a blob after checking it (magic, version,
+ *   sizes, every table entry and state id in range); a damaged blob gives WG_ERR_ARG.
+ * The format is little-endian and private to this library version. */
+int32_t wg_grammar_save(const wg_grammar *grammar, void *blob, size_t capacity, size_t *needed);
+int32_t wg_grammar_load(const void *blob, size_t size, wg_grammar **out);
+
 /* Host-side facts about a compiled grammar.  Any output pointer may be NULL.
  * content_hash identifies the table: two compilations with equal tables hash equally. */
 int32_t wg_grammar_info(const wg_grammar *grammar, int32_t *n_states, int32_t *start_state,

@@ -55,6 +55,8 @@ _SIGNATURES = {
     "wg_compile_grammar": (_i32, [_vp, _i32, _vp, _i32, _vp, _i32, _vp, _i32, _i32, C.POINTER(_vp)]),
     "wg_grammar_free": (None, [_vp]),
     "wg_grammar_minimize": (_i32, [_vp, C.POINTER(_vp)]),
+    "wg_grammar_save": (_i32, [_vp, _vp, C.c_size_t, C.POINTER(C.c_size_t)]),
+    "wg_grammar_load": (_i32, [C.c_char_p, C.c_size_t, C.POINTER(_vp)]),
     "wg_regex_to_optree": (_i32, [C.c_char_p, _i32, C.POINTER(_vp)]),
     "wg_optree_sizes": (_i32, [_vp, C.POINTER(_i32), C.POINTER(_i32), C.POINTER(_i32),
                                C.POINTER(_i32), C.POINTER(_i32)]),
@@ -225,6 +227,20 @@ class Grammar:
         rc = _lib.wg_compile_regex(pattern, len(pattern), C.byref(h))
         if rc != WG_OK:
             raise WgError(rc, "wg_compile_regex: " + _lib.wg_regex_error().decode())
+        return cls(_handle=h)
+
+    def save(self) -> bytes:
+        """wg_grammar_save: the compiled table as a blob for wg_grammar_load."""
+        need = C.c_size_t()
+        _lib.wg_grammar_save(self.handle, None, 0, C.byref(need))
+        buf = C.create_string_buffer(need.value)
+        _check(_lib.wg_grammar_save(self.handle, buf, need.value, C.byref(need)), "wg_grammar_save")
+        return buf.raw
+
+    @classmethod
+    def load(cls, blob: bytes) -> "Grammar":
+        h = _vp()
+        _check(_lib.wg_grammar_load(blob, len(blob), C.byref(h)), "wg_grammar_load")
         return cls(_handle=h)
 
     def minimized(self) -> "Grammar":

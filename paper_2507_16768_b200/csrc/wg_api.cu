@@ -272,6 +272,81 @@ int32_t wg_grammar_minimize(const wg_grammar *g, wg_grammar **out) {
     return WG_OK;
 }
 
+namespace {
+constexpr uint32_t BLOB_MAGIC = 0x31474757u;  // "WGG1"
+struct BlobHeader {
+    uint32_t magic, version;
+    int32_t n_states, n_classes, start, done, eos_class, has_forced;
+    uint64_t hash;
+};
+}  // namespace
+
+int32_t wg_grammar_save(const wg_grammar *g, void *blob, size_t capacity, size_t *needed) {
+    if (!g || !needed) return WG_ERR_ARG;
+    const size_t n_table = g->table.size() * sizeof(int32_t);
+    const size_t n_forced = g->forced_tok.size() * sizeof(int32_t);
+    const size_t total = sizeof(BlobHeader) + 256 + n_table + 2 * n_forced;
+    *needed = total;
+    if (capacity < total || !blob) return WG_ERR_CAPACITY;
+    uint8_t *p = static_cast<uint8_t *>(blob);
+    const BlobHeader h{BLOB_MAGIC, 1u, g->n_states, g->n_classes, g->start, g->done, g->eos_class,
+                       g->forced_tok.empty() ? 0 : 1, g->hash};
+    memcpy(p, &h, sizeof(h)); p += sizeof(h);
+    memcpy(p, g->byte_class, 256); p += 256;
+    memcpy(p, g->table.data(), n_table); p += n_table;
+    if (n_forced) {
+        memcpy(p, g->forced_tok.data(), n_forced); p += n_forced;
+        memcpy(p, g->forced_next.data(), n_forced);
+    }
+    return WG_OK;
+}
+
+int32_t wg_grammar_load(const void *blob, size_t size, wg_grammar **out) {
+    if (!out) return WG_ERR_ARG;
+    *out = nullptr;
+    if (!blob || size < sizeof(BlobHeader) + 256) return WG_ERR_ARG;
+    const uint8_t *p = static_cast<const uint8_t *>(blob);
+    BlobHeader h;
+    memcpy(&h, p, sizeof(h)); p += sizeof(h);
+    if (h.magic != BLOB_MAGIC || h.version != 1u) return WG_ERR_ARG;
+    if (h.n_states < 2 || h.n_classes < 1 || h.n_classes > WG_N_SYMBOLS) return WG_ERR_ARG;
+    if (h.start < 1 || h.start >= h.n_states || h.done < 1 || h.done >= h.n_states ||
+        h.eos_class < 0 || h.eos_class >= h.n_classes)
+        return WG_ERR_ARG;
+    const size_t cells = (size_t)h.n_states * (size_t)h.n_classes;
+    const size_t n_forced = h.has_forced ? (size_t)h.n_states * sizeof(int32_t) : 0;
+    if (size != sizeof(BlobHeader) + 256 + cells * sizeof(int32_t) + 2 * n_forced) return WG_ERR_ARG;
+    wg_grammar *g = new (std::nothrow) wg_grammar();
+    if (!g) return WG_ERR_ARG;
+    bool ok = true;
+    try {
+        g->n_states = h.n_states; g->n_classes = h.n_classes; g->start = h.start; g->done = h.done;
+        g->eos_class = h.eos_class; g->hash = h.hash;
+        memcpy(g->byte_class, p, 256); p += 256;
+        for (int b = 0; b < 256 && ok; ++b) ok = g->byte_class[b] < h.n_classes;
+        g->table.resize(cells);
+        memcpy(g->table.data(), p, cells * sizeof(int32_t)); p += cells * sizeof(int32_t);
+        for (size_t i = 0; i < cells && ok; ++i) ok = g->table[i] >= 0 && g->table[i] < h.n_states;
+        for (int32_t c = 0; c < h.n_classes && ok; ++c) ok = g->table[c] == 0;  // DEAD stays dead
+        if (n_forced) {
+            g->forced_tok.resize(h.n_states);
+            g->forced_next.resize(h.n_states);
+            memcpy(g->forced_tok.data(), p, n_forced); p += n_forced;
+            memcpy(g->forced_next.data(), p, n_forced);
+            for (int32_t st = 0; st < h.n_states && ok; ++st)
+                ok = g->forced_tok[st] >= -1 && g->forced_next[st] >= 0 && g->forced_next[st] < h.n_states;
+        }
+    } catch (const std::bad_alloc &) {
+        ok = false;
+    }
+    if (!ok) {
+        delete g;
+        return WG_ERR_ARG;
+    }
+    *out = g;
+    return WG_OK;
+}
+
 int32_t wg_grammar_info(const wg_grammar *g, int32_t *n_states, int32_t *start_state,
                         int32_t *done_state, int32_t *n_classes, uint64_t *content_hash) {
     if (!g) return WG_ERR_ARG;

@@ -202,3 +202,27 @@ def test_minimization_merges_repeated_tails(wg):
     m = t.minimized()
     assert m.n_states == t.n_states
     assert [m.forced_token(s)[0] for s in range(1, 5)] == [5, 6, 5, 6]
+
+
+def test_saved_grammar_loads_back_identical_and_damage_is_refused(wg):
+    for op in (grammars.json_reference_lookup(doc_nodes=50), Sequence(Write(b"a"), WriteTokens([7, 9]))):
+        g = wg.Grammar(flatten(op))
+        blob = g.save()
+        back = wg.Grammar.load(blob)
+        assert (back.n_states, back.n_classes, back.start_state, back.done_state, back.content_hash) == \
+               (g.n_states, g.n_classes, g.start_state, g.done_state, g.content_hash)
+        for s_ in range(g.n_states):
+            assert back.forced_token(s_) == g.forced_token(s_)
+            for sym in (0, 34, 48, 97, 255, EOS):
+                assert back.step(s_, sym) == g.step(s_, sym)
+        assert wg.Grammar.load(back.save()).save() == blob
+        for damaged in (blob[:-1], blob + b"x", b"\0" * len(blob), blob[:4] + b"\x09" + blob[5:]):
+            with pytest.raises(wg.WgError) as e:
+                wg.Grammar.load(damaged)
+            assert e.value.status == wg.binding.WG_ERR_ARG
+        # a table entry pointing outside the table
+        bad = bytearray(blob)
+        off = 40 + 256 + 4 * g.n_classes            # first cell of state 1
+        bad[off:off + 4] = (g.n_states + 5).to_bytes(4, "little")
+        with pytest.raises(wg.WgError):
+            wg.Grammar.load(bytes(bad))
