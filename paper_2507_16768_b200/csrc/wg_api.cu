@@ -82,6 +82,7 @@ struct wg_vocab {
     VocabDev dev{};
     void *d_rec = nullptr, *d_len = nullptr, *d_offsets = nullptr, *d_bytes = nullptr;
     void *d_first_mask = nullptr, *d_fold_mask = nullptr, *d_valid_mask = nullptr;
+    std::vector<uint8_t> host_rec;  // the 16-byte records, kept for per-grammar class mapping
     int device = 0;
 };
 
@@ -93,8 +94,14 @@ struct GrammarSlot {
     void *d_table, *d_cls, *d_first_ok, *d_leaves, *d_forced;
 };
 
+struct ClassMappedRecords {
+    uint8_t byte_class[256];
+    void *d_rec;  // uint4[V]
+};
+
 struct wg_ctx {
     const wg_vocab *vocab = nullptr;
+    std::vector<ClassMappedRecords> class_records;  // one per distinct byte_class map
     CtxDev dev{};
     std::vector<GrammarDev> grammars;  // host mirror of dev.grammars
     std::vector<GrammarSlot> slots;
@@ -208,6 +215,7 @@ int32_t wg_load_vocab(const uint32_t *offsets, const uint8_t *bytes, int32_t V, 
     v->dev.valid_mask = static_cast<const uint32_t *>(v->d_valid_mask);
     v->dev.offsets = static_cast<const uint32_t *>(v->d_offsets);
     v->dev.bytes = static_cast<const uint8_t *>(v->d_bytes);
+    v->host_rec = std::move(rec);
     v->dev.V = V;
     v->dev.W = (V + 31) / 32;
     v->dev.eos_id = eos_id;
@@ -439,6 +447,7 @@ void wg_ctx_free(wg_ctx *c) {
     if (!c) return;
     cudaDeviceSynchronize();
     for (void *p : c->owned) cudaFree(p);
+    for (ClassMappedRecords &r : c->class_records) cudaFree(r.d_rec);
     for (cudaEvent_t e : c->events) cudaEventDestroy(e);
     for (GrammarSlot &s : c->slots) {
         cudaFree(s.d_table);
@@ -513,10 +522,31 @@ int32_t wg_ctx_add_grammar(wg_ctx *c, const wg_grammar *g, int32_t *grammar_id) 
         WG_CUDA(cudaMemcpy(slot.d_leaves, leaves.data(), leaves.size() * sizeof(unsigned long long),
                            cudaMemcpyHostToDevice));
     }
+    // the vocabulary's records with bytes replaced by this grammar's classes (shared between
+    // grammars whose class maps are equal)
+    const void *d_rec_class = nullptr;
+    for (const ClassMappedRecords &r : c->class_records)
+        if (memcmp(r.byte_class, g->byte_class, 256) == 0) d_rec_class = r.d_rec;
+    if (!d_rec_class) {
+        const std::vector<uint8_t> &src = c->vocab->host_rec;
+        std::vector<uint8_t> mapped(src.size());
+        for (size_t i = 0; i < src.size(); ++i) mapped[i] = g->byte_class[src[i]];
+        ClassMappedRecords r;
+        memcpy(r.byte_class, g->byte_class, 256);
+        r.d_rec = nullptr;
+        WG_CUDA(cudaMalloc(&r.d_rec, mapped.size() ? mapped.size() : 1));
+        if (cudaMemcpy(r.d_rec, mapped.data(), mapped.size(), cudaMemcpyHostToDevice) != cudaSuccess) {
+            cudaFree(r.d_rec);
+            return WG_ERR_CUDA;
+        }
+        c->class_records.push_back(r);
+        d_rec_class = r.d_rec;
+    }
     GrammarDev gd{slot.d_table, static_cast<const uint8_t *>(slot.d_cls),
                   static_cast<const uint32_t *>(slot.d_first_ok),
                   static_cast<const unsigned long long *>(slot.d_leaves),
-                  static_cast<const int2 *>(slot.d_forced), g->n_states,
+                  static_cast<const int2 *>(slot.d_forced),
+                  static_cast<const uint4 *>(d_rec_class), g->n_states,
                   g->n_classes, g->start, g->done, g->eos_class, wide ? 1 : 0};
     const int32_t id = (int32_t)c->slots.size();
     if (id >= c->grammar_cap) {  // grow the registry; queued kernels still read the old one

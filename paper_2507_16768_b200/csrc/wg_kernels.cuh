@@ -19,6 +19,9 @@ struct GrammarDev {
                                        // lead anywhere but back to the state itself
     const int2 *forced;         // [n_states] (token id or -1, next state), or NULL: states of a
                                 // token-level Write accept exactly one whole token
+    const uint4 *rec_class;     // [V] the vocabulary's 16-byte records with every byte replaced by
+                                // its class under THIS grammar's byte_class (shared by grammars
+                                // with equal class maps): saves the class look-up in the walk
     int32_t n_states, n_classes, start, done, eos_class, wide;
 };
 
@@ -75,6 +78,28 @@ __device__ __forceinline__ uint32_t walk_record(const T *__restrict__ tab, int C
         if (j >= n || s == 0) break;
         const uint32_t b = (w[j >> 2] >> (8 * (j & 3))) & 0xFFu;
         s = tab[(size_t)s * C + cls[b]];
+    }
+    return s;
+}
+
+// The walk of the build kernel: the first 16 bytes come as classes straight from the
+// grammar's class-mapped record, so every step is one dependent table look-up.
+template <typename T>
+__device__ __forceinline__ uint32_t walk_token_classes(const VocabDev &v, const uint4 *rec_class,
+                                                       const T *__restrict__ tab, int C,
+                                                       const uint8_t *cls, uint32_t s, int t) {
+    const int n = v.len[t];
+    if (n == 0) return 0;
+    const uint4 rec = __ldg(&rec_class[t]);
+    const uint32_t w[4] = {rec.x, rec.y, rec.z, rec.w};
+#pragma unroll
+    for (int j = 0; j < WG_REC_BYTES; ++j) {
+        if (j >= n || s == 0) break;
+        s = tab[(size_t)s * C + ((w[j >> 2] >> (8 * (j & 3))) & 0xFFu)];
+    }
+    if (n > WG_REC_BYTES && s != 0) {
+        const uint32_t b = v.offsets[t] + WG_REC_BYTES, e = v.offsets[t + 1];
+        for (uint32_t i = b; i < e && s != 0; ++i) s = tab[(size_t)s * C + cls[v.bytes[i]]];
     }
     return s;
 }
@@ -225,11 +250,12 @@ build_masks_kernel(VocabDev v, CtxDev ctx, BuildWork work) {
         const int n = n_todo;
         for (int i = threadIdx.x; i < n; i += BUILD_THREADS) {
             const int rel = todo[i];
+            // (the EOS token is never queued: it has no bytes)
             const uint32_t end = g.wide
-                ? walk_token<uint32_t>(v, static_cast<const uint32_t *>(g.table), g.n_classes,
-                                       g.eos_class, cls, s0, t_begin + rel)
-                : walk_token<uint16_t>(v, static_cast<const uint16_t *>(g.table), g.n_classes,
-                                       g.eos_class, cls, s0, t_begin + rel);
+                ? walk_token_classes<uint32_t>(v, g.rec_class, static_cast<const uint32_t *>(g.table),
+                                               g.n_classes, cls, s0, t_begin + rel)
+                : walk_token_classes<uint16_t>(v, g.rec_class, static_cast<const uint16_t *>(g.table),
+                                               g.n_classes, cls, s0, t_begin + rel);
             if (end != 0) atomicOr(&words[rel >> 5], 1u << (rel & 31));
         }
         __syncthreads();
