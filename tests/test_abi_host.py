@@ -226,3 +226,16 @@ def test_saved_grammar_loads_back_identical_and_damage_is_refused(wg):
         bad[off:off + 4] = (g.n_states + 5).to_bytes(4, "little")
         with pytest.raises(wg.WgError):
             wg.Grammar.load(bytes(bad))
+
+
+def test_random_trees_lower_to_tables_that_match_the_checker(wg):
+    from test_oracle_pins import _random_tree
+    rng = np.random.default_rng(77)
+    symbols = list(b"abcd,;x") + [EOS]
+    for _ in range(80):
+        flat = flatten(_random_tree(rng, 3))
+        tree, g = oracle.Tree(flat), wg.Grammar(flat)
+        cursor_of = co_reachable(tree, g, symbols)
+        assert sorted(cursor_of) == list(range(1, g.n_states))
+        m = g.minimized()
+        assert sorted(co_reachable(tree, m, symbols)) == list(range(1, m.n_states))

@@ -527,3 +527,75 @@ def test_golden_fixture_of_the_section_3_2_listing():
         assert tree.accepts([ord(c) for c in text] + [EOS]) is (verdict == "accept"), line
         n += 1
     assert n >= 15
+
+
+# ---------------------------------------------------------------------------------------
+# random operator trees against the regular-expression restatement
+# ---------------------------------------------------------------------------------------
+def _random_tree(rng, depth):
+    alphabet = b"abcd,;"
+
+    def pick_sets(k):
+        """k pairwise disjoint non-empty deciding sets and a stay set disjoint from them."""
+        syms = list(alphabet)
+        rng.shuffle(syms)
+        cases = [SymSet([syms.pop()]) for _ in range(k)]
+        if syms and rng.random() < 0.4:
+            cases[0] = cases[0] | [syms.pop()]
+        stay = SymSet([s for s in syms if rng.random() < 0.5])
+        return cases, stay
+
+    def node(d):
+        kind = rng.integers(0, 7) if d > 0 else rng.integers(0, 3)
+        if kind == 0:
+            n = int(rng.integers(1, 4))
+            return Write(bytes(rng.choice(list(alphabet), size=n).tolist()))
+        if kind == 1:
+            (w,), stay = pick_sets(1)
+            return Wait(allow=stay | w, wait=w, body=node(d - 1) if d > 0 and rng.random() < 0.3 else None)
+        if kind == 2:
+            return WaitUntil(SymSet(b"ab,"), bytes(rng.choice(list(b"ab"), size=int(rng.integers(1, 4))).tolist()))
+        if kind == 3:
+            k = int(rng.integers(2, 4))
+            cases, stay = pick_sets(k)
+            union = stay
+            for c in cases:
+                union = union | c
+            return Switch(allow=union, cases=cases,
+                          bodies=[node(d - 1) if rng.random() < 0.7 else None for _ in range(k)])
+        if kind == 4:
+            (t, f), stay = pick_sets(2)
+            return DoWhile(node(d - 1) if rng.random() < 0.85 else None,
+                           Cond(allow=stay | t | f, true_waits=t, false_waits=f))
+        return Sequence([node(d - 1) for _ in range(int(rng.integers(0, 4)))])
+
+    return Sequence(node(depth), node(depth - 1))
+
+
+def test_random_trees_agree_with_their_regular_expression():
+    rng = np.random.default_rng(2024)
+    alphabet = list(b"abcd,;") + [EOS]
+    n_members = 0
+    for _ in range(60):
+        op = _random_tree(rng, 3)
+        tree = tree_of(op)
+        prog = regex_ref.program(op)
+        for _ in range(120):
+            # a random walk that mostly follows accepted symbols, so that deep states are reached
+            cursor, text = tree.start(), []
+            for _ in range(int(rng.integers(1, 25))):
+                options = [s for s in alphabet if not oracle.is_dead(tree.step(cursor, s))]
+                if options and rng.random() < 0.85:
+                    s = options[int(rng.integers(0, len(options)))]
+                else:
+                    s = alphabet[int(rng.integers(0, len(alphabet)))]
+                nxt = tree.step(cursor, s)
+                data = regex_ref.to_bytes(text + [s])
+                assert oracle.is_dead(nxt) == (not regex_ref.viable(prog, data)), (op, data)
+                if oracle.is_dead(nxt):
+                    break
+                cursor, text = nxt, text + [s]
+            member = regex_ref.member(prog, regex_ref.to_bytes(text))
+            assert (cursor == oracle.DONE) == member, (op, text)
+            n_members += member
+    assert n_members > 200
