@@ -589,3 +589,35 @@ def test_trajectory_on_minimized_grammars(wg, torch):
     for _ in range(50):
         sim.step()
     assert len(sim.visited) > 30
+
+
+def test_masks_of_random_trees_on_a_dense_small_alphabet_vocabulary(wg, torch):
+    import itertools
+    from test_oracle_pins import _random_tree
+    rng = np.random.default_rng(31)
+    alphabet = b"abcd,;"
+    tokens = [b""]                                                   # id 0 = EOS
+    for n in (1, 2, 3):
+        tokens += [bytes(t) for t in itertools.product(alphabet, repeat=n)]
+    tokens += [bytes(rng.choice(list(alphabet), size=int(rng.integers(4, 24))).tolist())
+               for _ in range(900)]
+    tokens += [b"x", b"ax", b""]
+    vocab = vocab_from_tokens(tokens, eos_id=0)
+    dv = wg.Vocab(vocab.offsets, vocab.data, vocab.eos_id)
+    symbols = list(alphabet) + [ord("x"), EOS]
+    ctx = wg.Context(dv, 4096, 512)
+    n_states = 0
+    for _ in range(25):
+        flat = flatten(_random_tree(rng, 3))
+        tree, g = oracle.Tree(flat), wg.Grammar(flat)
+        cursor_of = co_reachable(tree, g, symbols)
+        sids = sorted(cursor_of)[:512]
+        gid = ctx.add_grammar(g)
+        want = oracle.masks([tree] * len(sids), vocab, [cursor_of[s] for s in sids], n_threads=8)
+        for flags in (wg.WG_NO_CACHE, wg.WG_USE_CACHE):
+            out = torch.zeros((len(sids), dv.W), dtype=torch.int32, device="cuda")
+            wg.wg_build_masks(ctx, torch.full((len(sids),), gid, dtype=torch.int32, device="cuda"),
+                              to_dev(torch, np.array(sids, np.int32)), out, flags)
+            assert (out.cpu().numpy().view(np.uint32) == want).all()
+        n_states += len(sids)
+    assert n_states > 150
