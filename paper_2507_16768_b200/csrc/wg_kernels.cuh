@@ -3,6 +3,7 @@
 // tensor-core instruction appears.
 #pragma once
 
+#include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <cstdint>
 
@@ -493,6 +494,13 @@ __device__ __forceinline__ void block_argmax_commit(unsigned long long best,
 // Per-lane running maximum as (float value, id): a strict float compare keeps the first of
 // equal values and treats -0.0 and +0.0 as equal; !(v <= best) also takes the very first
 // allowed element, whatever its value (best starts as NaN).
+__device__ __forceinline__ __nv_bfloat162 as_bf162(uint32_t w) {
+    return *reinterpret_cast<const __nv_bfloat162 *>(&w);
+}
+__device__ __forceinline__ uint32_t bf162_bits(__nv_bfloat162 v) {
+    return *reinterpret_cast<const uint32_t *>(&v);
+}
+
 struct LaneBest {
     float v;
     int idx;
@@ -595,38 +603,55 @@ apply_mask_kernel(ApplyArgs a, CtxDev ctx, unsigned long long *argkey) {
                 if (chunk0 + c >= full_chunks || bits[q] == 0 || (!ARGMAX && bits[q] == FULL))
                     bits[q] = SKIP;
                 else
-                    val[q] = __ldcs(reinterpret_cast<const uint4 *>(row) + chunk0 + c);
+                    // a plain load, not a streaming one: a mixed chunk is stored back right
+                    // away and should still find its line
+                    val[q] = *(reinterpret_cast<const uint4 *>(row) + chunk0 + c);
             }
 #pragma unroll
             for (int q = 0; q < GROUP; ++q) {
                 if (bits[q] == SKIP) continue;
                 const int chunk = chunk0 + (p0 + q) * 32 + lane;
                 uint32_t w[4] = {val[q].x, val[q].y, val[q].z, val[q].w};
-                const int t0 = chunk * EPC;
-                if (sizeof(E) == 2) {
+                if (bits[q] != FULL) {  // disallowed elements become -inf
+                    if (sizeof(E) == 2) {
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        if ((bits[q] >> i) & 1u) {
-                            if (ARGMAX)
-                                best.offer((i & 1) ? (w[i >> 1] & 0xFFFF0000u) : (w[i >> 1] << 16),
-                                           t0 + i);
-                        } else {
-                            w[i >> 1] = (i & 1) ? ((w[i >> 1] & 0x0000FFFFu) | 0xFF800000u)
-                                                : ((w[i >> 1] & 0xFFFF0000u) | 0x0000FF80u);
+                        for (int i = 0; i < 4; ++i) {
+                            const uint32_t two = (bits[q] >> (2 * i)) & 3u;
+                            const uint32_t keep = ((two & 1u) ? 0x0000FFFFu : 0u) | ((two & 2u) ? 0xFFFF0000u : 0u);
+                            w[i] = (w[i] & keep) | (NEG_INF_BF16X2 & ~keep);
                         }
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 4; ++i)
+                            if (!((bits[q] >> i) & 1u)) w[i] = NEG_INF_F32;
                     }
-                } else {
+                    __stcs(reinterpret_cast<uint4 *>(row) + chunk, make_uint4(w[0], w[1], w[2], w[3]));
+                }
+                if (ARGMAX) {
+                    // The maximum of the chunk over the patched values (disallowed ones are -inf
+                    // now) costs a few max instructions; the element is looked up only when it
+                    // beats the lane's running maximum, which soon becomes rare.
+                    float m;
+                    if (sizeof(E) == 2) {
+                        const __nv_bfloat162 m2 = __hmax2(__hmax2(as_bf162(w[0]), as_bf162(w[1])),
+                                                          __hmax2(as_bf162(w[2]), as_bf162(w[3])));
+                        const uint32_t u = bf162_bits(m2);
+                        m = fmaxf(__uint_as_float(u << 16), __uint_as_float(u & 0xFFFF0000u));
+                    } else {
+                        m = fmaxf(fmaxf(__uint_as_float(w[0]), __uint_as_float(w[1])),
+                                  fmaxf(__uint_as_float(w[2]), __uint_as_float(w[3])));
+                    }
+                    if (!(m <= best.v)) {
+                        const int t0 = chunk * EPC;
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        if ((bits[q] >> i) & 1u) {
-                            if (ARGMAX) best.offer(w[i], t0 + i);
-                        } else {
-                            w[i] = NEG_INF_F32;
+                        for (int i = EPC - 1; i >= 0; --i) {  // descending: the lowest id stays
+                            const uint32_t e = sizeof(E) == 2
+                                ? ((i & 1) ? (w[i >> 1] & 0xFFFF0000u) : (w[i >> 1] << 16)) : w[i];
+                            if (((bits[q] >> i) & 1u) && __uint_as_float(e) == m) best.idx = t0 + i;
                         }
+                        best.v = m;
                     }
                 }
-                if (bits[q] != FULL)
-                    __stcs(reinterpret_cast<uint4 *>(row) + chunk, make_uint4(w[0], w[1], w[2], w[3]));
             }
         }
     }
