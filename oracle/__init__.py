@@ -192,3 +192,31 @@ def advance(tree: Tree, vocab, cursor, token: int):
 
 def max_threads() -> int:
     return int(lib().wgo_max_threads())
+
+
+# ---- adaptive token-set storage of a mask (paper Section 3.3) ---------------------------------
+# A Wait keeps either the few tokens it refuses ("denies", when most of the vocabulary is
+# accepted) or the few it accepts ("allows", when most is refused).  Written out plainly: count
+# the allowed tokens among ids 0..V-1 and keep the smaller side as a sorted id list.  A tie keeps
+# the allowed side.
+ALLOWS = 0
+DENIES = 1
+
+
+def adaptive_token_set(mask_words: np.ndarray, V: int) -> Tuple[int, np.ndarray]:
+    """(kind, sorted token ids) for one packed mask row."""
+    allowed = [t for t in range(V) if (int(mask_words[t >> 5]) >> (t & 31)) & 1]
+    if 2 * len(allowed) <= V:
+        return ALLOWS, np.asarray(allowed, np.int32)
+    taken = set(allowed)
+    return DENIES, np.asarray([t for t in range(V) if t not in taken], np.int32)
+
+
+def apply_token_set(logits: np.ndarray, kind: int, ids: np.ndarray, V: int) -> None:
+    """Masks one row of raw logit bit patterns (uint16 = bf16, uint32 = fp32) in place from a
+    token set: with ALLOWS every id that is not listed becomes -inf, with DENIES every listed one."""
+    ninf = {np.dtype(np.uint16): 0xFF80, np.dtype(np.uint32): 0xFF800000}[logits.dtype]
+    listed = set(int(t) for t in ids)
+    for t in range(V):
+        if (t in listed) == (kind == DENIES):
+            logits[t] = ninf

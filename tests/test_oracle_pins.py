@@ -409,6 +409,58 @@ def test_argmax_ties_signed_zero_and_all_minus_inf():
     assert oracle.argmax(bf, words, V)[0] == 50
 
 
+# ---------------------------------------------------------------------------------------
+# adaptive allows / denies storage (Section 3.3) and the apply that works from such a set
+# ---------------------------------------------------------------------------------------
+def test_adaptive_token_set_hand_examples():
+    # V = 10, allowed = {1, 4, 9}: reject-heavy, so the allowed side is kept
+    words = np.array([(1 << 1) | (1 << 4) | (1 << 9)], np.uint32)
+    kind, ids = oracle.adaptive_token_set(words, 10)
+    assert kind == oracle.ALLOWS and ids.tolist() == [1, 4, 9]
+    # allowed = everything but {0, 7}: accept-heavy, so the refused side is kept
+    words = np.array([0x3FF & ~((1 << 0) | (1 << 7))], np.uint32)
+    kind, ids = oracle.adaptive_token_set(words, 10)
+    assert kind == oracle.DENIES and ids.tolist() == [0, 7]
+    # exactly half: the allowed side; bits at and beyond V are never listed
+    words = np.array([0b0101010101 | (1 << 20)], np.uint32)
+    kind, ids = oracle.adaptive_token_set(words, 10)
+    assert kind == oracle.ALLOWS and ids.tolist() == [0, 2, 4, 6, 8]
+    # nothing allowed / everything allowed, across a word boundary
+    kind, ids = oracle.adaptive_token_set(np.zeros(2, np.uint32), 40)
+    assert kind == oracle.ALLOWS and ids.size == 0
+    kind, ids = oracle.adaptive_token_set(np.array([0xFFFFFFFF, 0xFF], np.uint32), 40)
+    assert kind == oracle.DENIES and ids.size == 0
+    kind, ids = oracle.adaptive_token_set(np.array([0xFFFFFFFF, 0x7F], np.uint32), 40)
+    assert kind == oracle.DENIES and ids.tolist() == [39]
+
+
+def test_apply_from_a_token_set_hand_example_and_against_the_dense_apply():
+    x = np.arange(1, 7, dtype=np.float32).view(np.uint32).copy()
+    y = x.copy()
+    oracle.apply_token_set(y, oracle.ALLOWS, np.array([0, 3], np.int32), 6)
+    assert y.view(np.float32).tolist() == [1.0, -np.inf, -np.inf, 4.0, -np.inf, -np.inf]
+    y = x.copy()
+    oracle.apply_token_set(y, oracle.DENIES, np.array([0, 3], np.int32), 6)
+    assert y.view(np.float32).tolist() == [-np.inf, 2.0, 3.0, -np.inf, 5.0, 6.0]
+    # both storage forms describe the same mask: the result equals the dense apply
+    rng = np.random.default_rng(11)
+    V = 1003
+    for dtype, density in (("bf16", 0.02), ("fp32", 0.97), ("bf16", 0.5)):
+        keep = rng.random(V) < density
+        words = np.zeros((1, (V + 31) // 32), np.uint32)
+        for t in np.nonzero(keep)[0]:
+            words[0, t >> 5] |= np.uint32(1 << (t & 31))
+        kind, ids = oracle.adaptive_token_set(words[0], V)
+        assert kind == (oracle.ALLOWS if 2 * keep.sum() <= V else oracle.DENIES)
+        assert ids.size == min(keep.sum(), V - keep.sum())
+        logits = make_logits(1, V, dtype, 3)
+        raw = logits.view(np.uint32) if dtype == "fp32" else logits
+        a, b = raw.copy(), raw.copy()
+        oracle.apply_mask(a, words, V)
+        oracle.apply_token_set(b[0], kind, ids, V)
+        assert (a == b).all()
+
+
 def test_enum_trie_accepts_exactly_its_strings():
     names = [b'alpha"', b'alps"', b'beta"', b'be"', b'gamma-1"', b'gamma-2"', b'g"']
     op = Sequence(Write(b'"'), enum_trie(names), Write(b";"))
