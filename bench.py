@@ -60,6 +60,8 @@ def parse_args():
                    help="call wg_build_masks / wg_apply_mask / wg_advance instead of wg_decode_step")
     p.add_argument("--steer-all", action="store_true",
                    help="steer every structural character (rows then dwell in free-text slots)")
+    p.add_argument("--cache-mode", default="dense", choices=["dense", "compact"],
+                   help="storage of cached masks: packed rows, or allows / denies entries")
     p.add_argument("--no-cpu-baseline", action="store_true")
     p.add_argument("--no-e2e", action="store_true")
     p.add_argument("--cpu-seconds", type=float, default=12.0)
@@ -252,7 +254,8 @@ def run_ours(args, w, steer: float) -> None:
     n_states = sum(c.n_states for c in compiled.values())
     # every state of every grammar, but never more rows than a run can visit
     capacity = min(n_states + 64, 1 << 16) if w.use_cache else 0
-    ctx = wg.Context(dv, capacity, B)
+    ctx = wg.Context(dv, capacity, B, wg.WG_CACHE_COMPACT if args.cache_mode == "compact"
+                     else wg.WG_CACHE_DENSE)
     gid_of = {g: ctx.add_grammar(c) for g, c in compiled.items()}
     if w.prewarm:
         for g in grammar_ids:
@@ -423,7 +426,8 @@ def run_ours(args, w, steer: float) -> None:
         "config": {"workload": w.name, "V": V, "batch_per_gpu": B, "logits": w.dtype,
                    "states": n_states, "launch": "separate calls" if args.separate else
                    ("cuda graph" if args.graph else "stream"), "cache": "prewarmed" if w.prewarm else
-                   ("on" if w.use_cache else "off"), "steer": steer, "ring": ring,
+                   ("on" if w.use_cache else "off"), "cache_mode": args.cache_mode, "steer": steer,
+                   "ring": ring,
                    "l2": "inputs larger than L2" if B * row_bytes > (126 << 20) else
                    "ring of distinct buffers; working set may sit in L2",
                    "timing": "CUDA events per chunk of <= ring steps; logits restored between "
@@ -432,7 +436,7 @@ def run_ours(args, w, steer: float) -> None:
         "kernel_ms": {"lookup_and_build": build_ms, "apply": apply_ms},
         "tokens_checked_per_s": (built * V) / (ms * 1e-3) if built else 0.0,
         "cache": {k: stats[k] for k in ("cache_hits", "cache_misses", "masks_built",
-                                         "rows_uncached", "cache_entries")},
+                                         "rows_uncached", "cache_entries", "cache_bytes")},
         "rows_with_error_status": bad,
         "e2e": e2e, "gpu_launches": launches, "clocks": clocks, "wall_s": wall,
     }

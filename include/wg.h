@@ -118,6 +118,16 @@ typedef struct wg_vocab wg_vocab;     /* token byte strings, resident on one dev
 typedef struct wg_grammar wg_grammar; /* a compiled transition table, host side     */
 typedef struct wg_ctx wg_ctx;         /* device tables, mask cache and scratch      */
 
+/* Storage of the mask cache (wg_ctx_create_ex) and the two forms of a compact entry. */
+enum {
+    WG_CACHE_DENSE = 0,  /* one packed mask row of W words per cached state                    */
+    WG_CACHE_COMPACT = 1 /* adaptive allows / denies entries (paper Section 3.3)               */
+};
+enum {
+    WG_ENTRY_ALLOWS = 0, /* reject-heavy state: the entry keeps the allowed tokens             */
+    WG_ENTRY_DENIES = 1  /* accept-heavy state: the entry keeps the refused tokens             */
+};
+
 typedef struct wg_stats {
     int64_t cache_hits;      /* rows served from the cache                                  */
     int64_t cache_misses;    /* rows whose mask had to be built (first sight of the state)  */
@@ -127,6 +137,7 @@ typedef struct wg_stats {
     int64_t empty_masks;     /* rows whose argmax found no allowed token                    */
     int64_t bad_states;      /* rows with a grammar or state id out of range                */
     int64_t cache_entries;   /* states held by the cache now                                */
+    int64_t cache_bytes;     /* device memory those cached masks occupy                     */
 } wg_stats;
 
 /* ---- setup ------------------------------------------------------------------------- */
@@ -231,6 +242,34 @@ int32_t wg_grammar_forced_token(const wg_grammar *grammar, int32_t state, int32_
 int32_t wg_ctx_create(const wg_vocab *vocab, int32_t cache_capacity, int32_t max_batch,
                       wg_ctx **out);
 void wg_ctx_free(wg_ctx *ctx);
+
+/* wg_ctx_create with a choice of cache storage.
+ * WG_CACHE_DENSE is wg_ctx_create.  WG_CACHE_COMPACT stores every cached mask the way the
+ * paper's Wait operator keeps its token sets (Section 3.3: a few refused tokens in `denies`
+ * when most of the vocabulary is accepted, the accepted ones in `allows` when most is
+ * refused): the side with fewer tokens is kept -- allows when at most half of the V tokens
+ * are allowed, denies otherwise.  On the device an entry holds its listed tokens grouped by
+ * 32-token mask word (only the words that contain a listed token are stored, behind a small
+ * per-span index), so an entry never takes more room than the id list and a row is masked
+ * straight from it.  Masks of literal states and of free-text slots shrink from V/8 bytes to
+ * a few hundred bytes, which is what lets grammars with hundreds of thousands of states stay
+ * cached.  Results of every call are identical in both modes.
+ *   arena_bytes  device memory for the entries; 0 = a quarter of what cache_capacity dense
+ *                rows would take.  When the arena is full, further new states are built on
+ *                every step (counted as rows_uncached), as with a full dense pool.
+ * Errors: WG_ERR_ARG (also: unknown cache_mode, V above 1 048 576 in compact mode), WG_ERR_CUDA. */
+int32_t wg_ctx_create_ex(const wg_vocab *vocab, int32_t cache_capacity, int32_t max_batch,
+                         int32_t cache_mode, size_t arena_bytes, wg_ctx **out);
+
+/* Reads one cached entry of a WG_CACHE_COMPACT context back to the host as the paper's token
+ * set: *kind = WG_ENTRY_ALLOWS or WG_ENTRY_DENIES (or -1 when (grammar_id, state) is not
+ * cached), *n_listed = number of tokens on the kept side, ids_host[0 .. min(n_listed,
+ * ids_capacity)) = those token ids in ascending order, *entry_bytes = device bytes the entry
+ * occupies.  Any output pointer may be NULL.  For tests and tooling; synchronises `stream`.
+ * Errors: WG_ERR_ARG (also for a dense context), WG_ERR_CUDA. */
+int32_t wg_cache_entry_read(wg_ctx *ctx, int32_t grammar_id, int32_t state, int32_t *kind,
+                            int32_t *n_listed, int32_t *ids_host, int32_t ids_capacity,
+                            int64_t *entry_bytes, void *stream);
 
 /* Uploads a compiled grammar's table and returns its id in this context.  A grammar whose
  * content_hash and tables equal one already added gets that grammar's id, so requests

@@ -30,6 +30,10 @@ WG_DTYPE_FP32 = 1
 WG_USE_CACHE = 0
 WG_NO_CACHE = 1
 WG_RESTART_ON_DONE = 2
+WG_CACHE_DENSE = 0
+WG_CACHE_COMPACT = 1
+WG_ENTRY_ALLOWS = 0
+WG_ENTRY_DENIES = 1
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(
@@ -42,7 +46,7 @@ _lib = C.CDLL(LIB_PATH)
 class WgStats(C.Structure):
     _fields_ = [(n, C.c_int64) for n in (
         "cache_hits", "cache_misses", "masks_built", "rows_uncached", "tokens_rejected",
-        "empty_masks", "bad_states", "cache_entries")]
+        "empty_masks", "bad_states", "cache_entries", "cache_bytes")]
 
     def as_dict(self):
         return {n: int(getattr(self, n)) for n, _ in self._fields_}
@@ -69,7 +73,10 @@ _SIGNATURES = {
     "wg_grammar_step": (_i32, [_vp, _i32, _i32]),
     "wg_grammar_forced_token": (_i32, [_vp, _i32, C.POINTER(_i32), C.POINTER(_i32)]),
     "wg_ctx_create": (_i32, [_vp, _i32, _i32, C.POINTER(_vp)]),
+    "wg_ctx_create_ex": (_i32, [_vp, _i32, _i32, _i32, C.c_size_t, C.POINTER(_vp)]),
     "wg_ctx_free": (None, [_vp]),
+    "wg_cache_entry_read": (_i32, [_vp, _i32, _i32, C.POINTER(_i32), C.POINTER(_i32), _vp, _i32,
+                                   C.POINTER(_i64), _vp]),
     "wg_ctx_add_grammar": (_i32, [_vp, _vp, C.POINTER(_i32)]),
     "wg_cache_prewarm": (_i32, [_vp, _i32, _vp]),
     "wg_cache_clear": (_i32, [_vp, _vp]),
@@ -283,13 +290,31 @@ class Grammar:
 class Context:
     """wg_ctx: device tables, the mask cache and per-batch scratch."""
 
-    def __init__(self, vocab: Vocab, cache_capacity: int, max_batch: int):
+    def __init__(self, vocab: Vocab, cache_capacity: int, max_batch: int,
+                 cache_mode: int = WG_CACHE_DENSE, arena_bytes: int = 0):
         self.vocab = vocab
         self.max_batch = int(max_batch)
         h = _vp()
-        _check(_lib.wg_ctx_create(vocab.handle, int(cache_capacity), int(max_batch), C.byref(h)),
-               "wg_ctx_create")
+        if cache_mode == WG_CACHE_DENSE and not arena_bytes:
+            _check(_lib.wg_ctx_create(vocab.handle, int(cache_capacity), int(max_batch),
+                                      C.byref(h)), "wg_ctx_create")
+        else:
+            _check(_lib.wg_ctx_create_ex(vocab.handle, int(cache_capacity), int(max_batch),
+                                         int(cache_mode), int(arena_bytes), C.byref(h)),
+                   "wg_ctx_create_ex")
         self.handle = h
+
+    def cache_entry(self, grammar_id: int, state: int, stream=None):
+        """wg_cache_entry_read: (kind, sorted token ids, device bytes) of one compact cache
+        entry, or None when the state is not cached."""
+        kind, n, nbytes = _i32(), _i32(), _i64()
+        ids = np.zeros(self.vocab.V, np.int32)
+        _check(_lib.wg_cache_entry_read(self.handle, int(grammar_id), int(state), C.byref(kind),
+                                        C.byref(n), _np_ptr(ids), ids.shape[0], C.byref(nbytes),
+                                        _stream_ptr(stream)), "wg_cache_entry_read")
+        if kind.value < 0:
+            return None
+        return kind.value, ids[:n.value].copy(), int(nbytes.value)
 
     def close(self):
         if getattr(self, "handle", None):

@@ -385,10 +385,17 @@ int32_t wg_grammar_step(const wg_grammar *g, int32_t state, int32_t symbol) {
 
 int32_t wg_ctx_create(const wg_vocab *vocab, int32_t cache_capacity, int32_t max_batch,
                       wg_ctx **out) {
+    return wg_ctx_create_ex(vocab, cache_capacity, max_batch, WG_CACHE_DENSE, 0, out);
+}
+
+int32_t wg_ctx_create_ex(const wg_vocab *vocab, int32_t cache_capacity, int32_t max_batch,
+                         int32_t cache_mode, size_t arena_bytes, wg_ctx **out) {
     if (!out) return WG_ERR_ARG;
     *out = nullptr;
     if (!vocab || cache_capacity < 0 || max_batch <= 0 || cache_capacity > (1 << 28))
         return WG_ERR_ARG;
+    if (cache_mode != WG_CACHE_DENSE && cache_mode != WG_CACHE_COMPACT) return WG_ERR_ARG;
+    const bool compact = cache_mode == WG_CACHE_COMPACT && cache_capacity > 0;
     wg_ctx *c = new (std::nothrow) wg_ctx();
     if (!c) return WG_ERR_ARG;
     c->vocab = vocab;
@@ -410,7 +417,25 @@ int32_t wg_ctx_create(const wg_vocab *vocab, int32_t cache_capacity, int32_t max
     };
     take(&d.keys, (size_t)d.hash_size);
     take(&d.vals, (size_t)d.hash_size);
-    take(&d.pool, (size_t)d.capacity * (size_t)d.pool_stride);
+    if (compact) {
+        d.compact = 1;
+        d.hdr_stride = (vocab->dev.W + 31) / 32;
+        // at least one mask with every word stored; word offsets must fit in 31 bits
+        size_t words = arena_bytes ? arena_bytes / sizeof(uint32_t)
+                                   : (size_t)d.capacity * (size_t)d.pool_stride / 4;
+        if (words < (size_t)d.pool_stride) words = (size_t)d.pool_stride;
+        if (words > 0x7FFFFFFFull) words = 0x7FFFFFFFull;
+        d.arena_words = (long long)words;
+        take(&d.arena, (size_t)d.arena_words);
+        take(&d.arena_top, 1);
+        take(&d.ent_hdr, (size_t)d.capacity * (size_t)d.hdr_stride);
+        take(&d.ent_fail, (size_t)d.capacity);
+        take(&d.ent_stage, (size_t)d.capacity);
+        take(&d.stage, (size_t)max_batch * (size_t)d.pool_stride);
+        take(&d.bl_row, (size_t)max_batch);
+    } else {
+        take(&d.pool, (size_t)d.capacity * (size_t)d.pool_stride);
+    }
     take(&d.n_slots, 1);
     take(&d.ent, (size_t)max_batch);
     take(&d.slot, (size_t)max_batch);
@@ -433,6 +458,10 @@ int32_t wg_ctx_create(const wg_vocab *vocab, int32_t cache_capacity, int32_t max
             cudaMemset(d.bl_count, 0, sizeof(int32_t)) != cudaSuccess ||
             cudaMemset(d.argkey, 0, sizeof(unsigned long long) * (size_t)max_batch) != cudaSuccess ||
             cudaMemset(d.stats, 0, sizeof(unsigned long long) * ST_COUNT) != cudaSuccess)
+            rc = WG_ERR_CUDA;
+        if (compact && rc == WG_OK &&
+            (cudaMemset(d.arena_top, 0, sizeof(unsigned long long)) != cudaSuccess ||
+             cudaMemset(d.ent_fail, 0, sizeof(int32_t) * (size_t)d.capacity) != cudaSuccess))
             rc = WG_ERR_CUDA;
     }
     if (rc != WG_OK) {
@@ -584,8 +613,12 @@ int32_t wg_get_stats(wg_ctx *c, wg_stats *out, void *stream) {
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     unsigned long long h[ST_COUNT];
     int32_t n_slots = 0;
+    unsigned long long arena_top = 0;
     WG_CUDA(cudaMemcpyAsync(h, c->dev.stats, sizeof(h), cudaMemcpyDeviceToHost, st));
     WG_CUDA(cudaMemcpyAsync(&n_slots, c->dev.n_slots, sizeof(n_slots), cudaMemcpyDeviceToHost, st));
+    if (c->dev.compact)
+        WG_CUDA(cudaMemcpyAsync(&arena_top, c->dev.arena_top, sizeof(arena_top),
+                                cudaMemcpyDeviceToHost, st));
     WG_CUDA(cudaStreamSynchronize(st));
     out->cache_hits = (int64_t)h[ST_HITS];
     out->cache_misses = (int64_t)h[ST_MISSES];
@@ -595,6 +628,10 @@ int32_t wg_get_stats(wg_ctx *c, wg_stats *out, void *stream) {
     out->empty_masks = (int64_t)h[ST_EMPTY];
     out->bad_states = (int64_t)h[ST_BAD_STATE];
     out->cache_entries = n_slots;
+    if (arena_top > (unsigned long long)c->dev.arena_words) arena_top = (unsigned long long)c->dev.arena_words;
+    out->cache_bytes = c->dev.compact
+        ? (int64_t)(arena_top * sizeof(uint32_t)) + (int64_t)n_slots * c->dev.hdr_stride * (int64_t)sizeof(uint2)
+        : (int64_t)n_slots * c->dev.pool_stride * (int64_t)sizeof(uint32_t);
     return WG_OK;
 }
 
@@ -621,11 +658,11 @@ int32_t launch_build(wg_ctx *c, const BuildWork &work, int max_entries, cudaStre
     long long grid = (long long)sm_count() * 8;  // 8 resident blocks of 256 threads per SM
     if (items < grid) grid = items;
     if (grid < 1) grid = 1;
+    auto kernel = c->dev.compact ? build_masks_kernel<true> : build_masks_kernel<false>;
     if (pdl)
-        WG_CUDA(launch_pdl(build_masks_kernel, dim3((unsigned)grid), dim3(BUILD_THREADS), st, v,
-                           c->dev, w));
+        WG_CUDA(launch_pdl(kernel, dim3((unsigned)grid), dim3(BUILD_THREADS), st, v, c->dev, w));
     else
-        build_masks_kernel<<<(unsigned)grid, BUILD_THREADS, 0, st>>>(v, c->dev, w);
+        kernel<<<(unsigned)grid, BUILD_THREADS, 0, st>>>(v, c->dev, w);
     WG_LAUNCHED();
     return WG_OK;
 }
@@ -714,7 +751,11 @@ int32_t wg_build_masks(wg_ctx *c, const int32_t *gid, const int32_t *sid, int32_
     int32_t rc = launch_build(c, work, B, st);
     if (rc != WG_OK) return rc;
     dim3 grid((unsigned)((W + 1023) / 1024), (unsigned)B);
-    cache_gather_kernel<<<grid, 256, 0, st>>>(c->dev, W, bitmask, row_stride_words);
+    if (c->dev.compact)
+        cache_gather_compact_kernel<<<grid, 256, 0, st>>>(c->dev, c->vocab->dev.V, W, bitmask,
+                                                          row_stride_words);
+    else
+        cache_gather_kernel<<<grid, 256, 0, st>>>(c->dev, W, bitmask, row_stride_words);
     WG_LAUNCHED();
     return WG_OK;
 }
@@ -859,6 +900,7 @@ int32_t wg_decode_step(wg_ctx *c, const int32_t *gid, int32_t *sid, int32_t B, v
 struct wg_step_graph {
     cudaGraph_t graph = nullptr;
     cudaGraphExec_t exec = nullptr;
+    int64_t kernels = 0;  // kernel launches one replay stands for
 };
 
 extern "C" {
@@ -880,8 +922,12 @@ int32_t wg_step_graph_create(wg_ctx *c, const int32_t *gid, int32_t *sid, int32_
     if (rc == WG_OK && cudaStreamBeginCapture(cap, cudaStreamCaptureModeThreadLocal) != cudaSuccess)
         rc = WG_ERR_CUDA;
     if (rc == WG_OK) {
+        const int64_t before = g_launches.load(std::memory_order_relaxed);
         rc = wg_decode_step(c, gid, sid, B, logits, dtype, row_stride_elems, bitmask,
                             mask_stride_words, token_out, status, flags, cap);
+        // the launches were recorded, not run: take them off the count of launches made
+        g->kernels = g_launches.load(std::memory_order_relaxed) - before;
+        g_launches.fetch_sub(g->kernels, std::memory_order_relaxed);
         cudaGraph_t graph = nullptr;
         const cudaError_t e = cudaStreamEndCapture(cap, &graph);  // always end the capture
         if (rc == WG_OK && e != cudaSuccess) { g_last_cuda_error = (int32_t)e; rc = WG_ERR_CUDA; }
@@ -904,7 +950,7 @@ int32_t wg_step_graph_create(wg_ctx *c, const int32_t *gid, int32_t *sid, int32_
 int32_t wg_step_graph_launch(wg_step_graph *g, void *stream) {
     if (!g || !g->exec) return WG_ERR_ARG;
     WG_CUDA(cudaGraphLaunch(g->exec, static_cast<cudaStream_t>(stream)));
-    g_launches.fetch_add(4, std::memory_order_relaxed);  // the four kernels of a step
+    g_launches.fetch_add(g->kernels, std::memory_order_relaxed);  // the kernels of one step
     return WG_OK;
 }
 
@@ -960,6 +1006,59 @@ int32_t wg_ctx_get_timing(wg_ctx *c, double *build_ms, double *apply_ms, int64_t
     if (apply_ms) *apply_ms = a;
     if (steps) *steps = (int64_t)c->timed_steps;
     c->timed_steps = 0;
+    return WG_OK;
+}
+
+int32_t wg_cache_entry_read(wg_ctx *c, int32_t grammar_id, int32_t state, int32_t *kind,
+                            int32_t *n_listed, int32_t *ids_host, int32_t ids_capacity,
+                            int64_t *entry_bytes, void *stream) {
+    if (!c || !c->dev.compact || ids_capacity < 0 || (ids_capacity > 0 && !ids_host)) return WG_ERR_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const VocabDev &v = c->vocab->dev;
+    if (kind) *kind = -1;
+    if (n_listed) *n_listed = 0;
+    if (entry_bytes) *entry_bytes = 0;
+    // find the cache row with the device's own probe and let the device expand the entry into
+    // a scratch row, exactly as a decode step reads it
+    iota_states_kernel<<<1, 32, 0, st>>>(c->d_stage_gid, c->d_stage_sid, grammar_id, state, 1);
+    WG_LAUNCHED();
+    cache_lookup_kernel<<<1, 32, 0, st>>>(c->dev, c->d_stage_gid, c->d_stage_sid, 1, c->dev.slot);
+    WG_LAUNCHED();
+    int32_t row = -1;
+    WG_CUDA(cudaMemcpyAsync(&row, c->dev.slot, sizeof(row), cudaMemcpyDeviceToHost, st));
+    WG_CUDA(cudaStreamSynchronize(st));
+    if (row < 0) return WG_OK;
+    cache_gather_compact_kernel<<<dim3((unsigned)((v.W + 1023) / 1024), 1), 256, 0, st>>>(
+        c->dev, v.V, v.W, c->dev.stage, c->dev.pool_stride);
+    WG_LAUNCHED();
+    std::vector<uint32_t> words((size_t)v.W);
+    std::vector<uint2> hdr((size_t)c->dev.hdr_stride);
+    WG_CUDA(cudaMemcpyAsync(words.data(), c->dev.stage, words.size() * sizeof(uint32_t),
+                            cudaMemcpyDeviceToHost, st));
+    WG_CUDA(cudaMemcpyAsync(hdr.data(), c->dev.ent_hdr + (size_t)row * c->dev.hdr_stride,
+                            hdr.size() * sizeof(uint2), cudaMemcpyDeviceToHost, st));
+    WG_CUDA(cudaStreamSynchronize(st));
+    // the paper's rule for the mask as a whole: keep the side with fewer tokens
+    int64_t allowed = 0;
+    for (uint32_t w : words) allowed += __builtin_popcount(w);
+    const int32_t k = 2 * allowed <= (int64_t)v.V ? WG_ENTRY_ALLOWS : WG_ENTRY_DENIES;
+    int32_t written = 0, total = 0;
+    for (int w = 0; w < v.W; ++w) {
+        const int tail = v.V & 31;
+        const uint32_t full = (w == v.W - 1 && tail) ? ((1u << tail) - 1u) : 0xFFFFFFFFu;
+        uint32_t listed = (k == WG_ENTRY_ALLOWS ? words[w] : ~words[w]) & full;
+        while (listed) {
+            const int b = __builtin_ctz(listed);
+            listed &= listed - 1;
+            if (written < ids_capacity) ids_host[written++] = w * 32 + b;
+            ++total;
+        }
+    }
+    size_t stored = 0;
+    for (const uint2 &h : hdr) stored += (size_t)__builtin_popcount(h.x);
+    if (kind) *kind = k;
+    if (n_listed) *n_listed = total;
+    if (entry_bytes) *entry_bytes = (int64_t)(hdr.size() * sizeof(uint2) + stored * sizeof(uint32_t));
     return WG_OK;
 }
 

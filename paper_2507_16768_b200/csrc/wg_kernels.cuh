@@ -60,7 +60,23 @@ struct CtxDev {
     int32_t *bl_count;
     unsigned long long *argkey;  // [max_batch] packed (value key, ~id) maxima
     unsigned long long *stats;   // [ST_COUNT]
+    // compact cache (allows / denies storage instead of dense pool rows); pool is NULL then
+    int32_t compact;
+    uint2 *ent_hdr;                  // [capacity][hdr_stride] per cache row and span of 32 mask
+                                     // words: (bitmap of the stored words, where they start in
+                                     // the arena | the span's default in bit 31)
+    int32_t hdr_stride;              // spans per mask = ceil(W / 32)
+    uint32_t *arena;                 // [arena_words] the stored words of all entries
+    unsigned long long *arena_top;   // words handed out so far (beyond arena_words: full)
+    long long arena_words;           // < 2^31
+    int32_t *ent_fail;               // [capacity] 1: part of the entry found no room in the arena;
+                                     // the state stays uncached from then on
+    int32_t *ent_stage;              // [capacity] staging row that holds the dense mask during
+                                     // the call that built the entry
+    uint32_t *stage;                 // [max_batch][pool_stride] dense masks built in this call
+    int32_t *bl_row;                 // [max_batch] cache row of each build-list entry, or -1
 };
+
 
 constexpr uint32_t NEG_INF_F32 = 0xFF800000u;
 constexpr uint32_t NEG_INF_BF16X2 = 0xFF80FF80u;
@@ -123,6 +139,60 @@ __device__ __forceinline__ uint32_t walk_token(const VocabDev &v, const T *__res
 }
 
 // ---------------------------------------------------------------------------------------
+// Compact cache entries: the adaptive allows / denies storage.  A mask is kept span by span
+// (a span = 32 mask words = 1024 tokens).  Each span makes the paper's choice for itself: when
+// fewer of its words differ from zero than from all-ones it keeps the allowed side (default
+// word 0), otherwise the refused side (default word all-ones below V); only the words that
+// differ from the default are stored, back to back in the arena.  The per-span header says
+// which words are stored, where they start, and which default applies.  A listed token costs
+// at most one stored word, so a mask never takes more room than its id list, and a reader
+// finds word w with one header load and one popcount instead of a search.
+// ---------------------------------------------------------------------------------------
+constexpr uint32_t HDR_DEFAULT_ONES = 0x80000000u;
+
+__device__ __forceinline__ uint32_t full_word(int w, int V, int W) {  // all tokens of word w
+    if (w >= W) return 0u;
+    const int tail = V & 31;
+    return (w == W - 1 && tail) ? ((1u << tail) - 1u) : 0xFFFFFFFFu;
+}
+
+// Mask word `span * 32 + lane` of a compact entry (called by all 32 lanes of a warp).
+__device__ __forceinline__ uint32_t entry_word(const uint2 *hdr_row, const uint32_t *arena, int span,
+                                               int lane, int V, int W) {
+    const uint2 hdr = hdr_row[span];
+    if ((hdr.x >> lane) & 1u)
+        return arena[(hdr.y & ~HDR_DEFAULT_ONES) + __popc(hdr.x & ((1u << lane) - 1u))];
+    return (hdr.y & HDR_DEFAULT_ONES) ? full_word(span * 32 + lane, V, W) : 0u;
+}
+
+// Stores one finished span (32 mask words, one per lane) of cache row `row`; called by a whole
+// warp.  The room is taken with one atomic add that is never given back: the first span that
+// does not fit leaves the top beyond the end, and from then on the arena counts as full.
+__device__ __forceinline__ void store_span(uint2 *hdr_row, uint32_t *arena,
+                                           unsigned long long *arena_top, long long arena_words,
+                                           int32_t *fail_flag, unsigned long long *uncached_stat,
+                                           int span, uint32_t word, int lane, int V, int W) {
+    const uint32_t b0 = __ballot_sync(0xFFFFFFFFu, word != 0u);
+    const uint32_t b1 = __ballot_sync(0xFFFFFFFFu, word != full_word(span * 32 + lane, V, W));
+    const bool ones = __popc(b1) < __popc(b0);
+    uint32_t bits = ones ? b1 : b0;
+    const int n = __popc(bits);
+    unsigned long long off = 0ull;
+    if (n > 0) {
+        if (lane == 0) off = atomicAdd(arena_top, (unsigned long long)n);
+        off = __shfl_sync(0xFFFFFFFFu, off, 0);
+        if (off + (unsigned long long)n > (unsigned long long)arena_words) {
+            if (lane == 0 && atomicExch(fail_flag, 1) == 0) atomicAdd(uncached_stat, 1ull);
+            bits = 0u;
+            off = 0ull;
+        } else if ((bits >> lane) & 1u) {
+            arena[off + __popc(bits & ((1u << lane) - 1u))] = word;
+        }
+    }
+    if (lane == 0) hdr_row[span] = make_uint2(bits, (uint32_t)off | (ones ? HDR_DEFAULT_ONES : 0u));
+}
+
+// ---------------------------------------------------------------------------------------
 // K1: mask build.  Work item = (mask m, chunk of tokens); a fixed-size grid strides over the
 // items, so a launch with nothing to build costs a few empty blocks.
 //
@@ -141,6 +211,21 @@ constexpr int BUILD_THREADS = 256;
 constexpr int BUILD_CHUNK_MAX = 8192;  // tokens per work item (the launch picks 2048 or 8192)
 constexpr int BUILD_MAX_FOLDS = 20;    // more leaving folds than this: queue every P token
 
+// The spans of one finished chunk (n_words mask words in shared memory, beginning at span
+// first_span) into a cache row.
+__device__ __forceinline__ void store_chunk_spans(uint2 *hdr_row, uint32_t *arena,
+                                               unsigned long long *arena_top, long long arena_words,
+                                               int32_t *fail_flag, unsigned long long *uncached_stat,
+                                               int first_span, int n_words, const uint32_t *words,
+                                               int V, int W) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int sl = warp; sl * 32 < n_words; sl += (int)(blockDim.x >> 5)) {
+        const int wl = sl * 32 + lane;
+        store_span(hdr_row, arena, arena_top, arena_words, fail_flag, uncached_stat, first_span + sl,
+                   wl < n_words ? words[wl] : 0u, lane, V, W);
+    }
+}
+
 struct BuildWork {
     const int32_t *gid, *sid;   // per entry
     uint32_t *const *dst_list;  // per entry destination, or NULL: use dst_base + m * dst_stride
@@ -151,7 +236,9 @@ struct BuildWork {
     int32_t chunk;              // tokens per work item: a multiple of 32, <= BUILD_CHUNK_MAX
 };
 
-__global__ void __launch_bounds__(BUILD_THREADS, 6)
+// COMPACT: the cache keeps allows / denies entries; finished chunks are also stored as spans.
+template <bool COMPACT>
+__global__ void __launch_bounds__(BUILD_THREADS, COMPACT ? 5 : 6)
 build_masks_kernel(VocabDev v, CtxDev ctx, BuildWork work) {
     __shared__ uint8_t cls[256];
     __shared__ int cls_gid;
@@ -263,6 +350,15 @@ build_masks_kernel(VocabDev v, CtxDev ctx, BuildWork work) {
         // phase 3: whole words out
         for (int wl = threadIdx.x; wl < n_words; wl += BUILD_THREADS)
             dst[(t_begin >> 5) + wl] = words[wl];
+        // Compact cache: the chunk's spans go into the cache entry straight from shared memory
+        // (chunks are whole spans; the dense words above only serve the call that built them).
+        if (COMPACT && work.dst_list) {
+            const int row = ctx.bl_row[m];
+            if (row >= 0)
+                store_chunk_spans(ctx.ent_hdr + (int64_t)row * ctx.hdr_stride, ctx.arena, ctx.arena_top,
+                                  ctx.arena_words, ctx.ent_fail + row, ctx.stats + ST_UNCACHED,
+                                  t_begin >> 10, n_words, words, v.V, v.W);
+        }
     }
 }
 
@@ -295,6 +391,7 @@ __global__ void cache_lookup_kernel(CtxDev ctx, const int32_t *gid, const int32_
             if (k == key) { found = ctx.vals[h]; break; }
             if (k == 0) break;
         }
+        if (ctx.compact && found >= 0 && ctx.ent_fail[found]) found = -1;
     }
     slot[r] = found;
 }
@@ -333,7 +430,14 @@ cache_lookup_insert_kernel(CtxDev ctx, const int32_t *gid, const int32_t *sid, i
                             const int i = atomicAdd(ctx.bl_count, 1);
                             ctx.bl_gid[i] = g;
                             ctx.bl_sid[i] = s;
-                            ctx.bl_dst[i] = ctx.pool + (int64_t)row * ctx.pool_stride;
+                            if (ctx.compact) {  // built into a staging row; its spans also go to the arena
+                                ctx.bl_dst[i] = ctx.stage + (int64_t)i * ctx.pool_stride;
+                                ctx.bl_row[i] = row;
+                                ctx.ent_fail[row] = 0;
+                                ctx.ent_stage[row] = i;
+                            } else {
+                                ctx.bl_dst[i] = ctx.pool + (int64_t)row * ctx.pool_stride;
+                            }
                         } else {
                             atomicSub(ctx.n_slots, 1);
                             ctx.vals[h] = -1;
@@ -352,7 +456,11 @@ cache_lookup_insert_kernel(CtxDev ctx, const int32_t *gid, const int32_t *sid, i
     int hits = 0, misses = 0, uncached = 0;
     for (int r = threadIdx.x; r < B; r += blockDim.x) {
         const int32_t e = ctx.ent[r];
-        const int32_t row = e >= 0 ? ctx.vals[e & ~ENT_NEW] : -1;
+        int32_t row = e >= 0 ? ctx.vals[e & ~ENT_NEW] : -1;
+        // a state whose entry found no room in the arena is rebuilt on every step
+        // a state whose entry found no room in the arena is rebuilt on every step (a row
+        // inserted by this very call still has the flag clear here)
+        if (ctx.compact && row >= 0 && ctx.ent_fail[row]) row = -1;
         ctx.slot[r] = row;
         // a hit is a row served from a pool row that some earlier row or call already owned
         if (row >= 0 && !(e & ENT_NEW)) ++hits; else ++misses;
@@ -363,6 +471,7 @@ cache_lookup_insert_kernel(CtxDev ctx, const int32_t *gid, const int32_t *sid, i
                 ctx.bl_gid[i] = gid[r];
                 ctx.bl_sid[i] = sid[r];
                 ctx.bl_dst[i] = bitmask + (int64_t)r * mask_stride;
+                if (ctx.compact) ctx.bl_row[i] = -1;
             }
         }
     }
@@ -390,12 +499,37 @@ __global__ void reset_rows_kernel(CtxDev ctx, int B) {
 __global__ void cache_clear_kernel(CtxDev ctx) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i < ctx.hash_size) { ctx.keys[i] = 0ull; ctx.vals[i] = -1; }
-    if (i == 0) *ctx.n_slots = 0;
+    if (i == 0) {
+        *ctx.n_slots = 0;
+        if (ctx.compact) *ctx.arena_top = 0ull;
+    }
 }
 
 __global__ void iota_states_kernel(int32_t *gid, int32_t *sid, int g, int first, int n) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i < n) { gid[i] = g; sid[i] = first + i; }
+}
+
+// K3 for the compact cache: expand entries into bitmask rows.  grid = (chunks of 32 spans, B).
+__global__ void __launch_bounds__(256)
+cache_gather_compact_kernel(CtxDev ctx, int V, int W, uint32_t *bitmask, int64_t mask_stride) {
+    const int r = blockIdx.y;
+    const int32_t row = ctx.slot[r];
+    if (row < 0) return;  // built straight into the bitmask
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int n_spans = (W + 31) / 32;
+    const bool failed = ctx.ent_fail[row] != 0;
+    const uint2 *hdr_row = ctx.ent_hdr + (int64_t)row * ctx.hdr_stride;
+    uint32_t *dst = bitmask + (int64_t)r * mask_stride;
+    for (int span = blockIdx.x * 32 + warp; span < min(n_spans, (int)(blockIdx.x + 1) * 32); span += 8) {
+        const int w = span * 32 + lane;
+        uint32_t word;
+        if (!failed)
+            word = entry_word(hdr_row, ctx.arena, span, lane, V, W);
+        else  // built in this call and the arena had no room: the staging row still holds it
+            word = w < W ? ctx.stage[(int64_t)ctx.ent_stage[row] * ctx.pool_stride + w] : 0u;
+        if (w < W) dst[w] = word;
+    }
 }
 
 // K3: copy cached rows out.  grid = (chunks, B).
@@ -536,9 +670,19 @@ apply_mask_kernel(ApplyArgs a, CtxDev ctx, unsigned long long *argkey) {
     E *row = static_cast<E *>(a.logits) + (int64_t)r * a.row_stride;
     const uint32_t *own = a.bitmask + (int64_t)r * a.mask_stride;
     const uint32_t *mrow = own;
+    const uint2 *entry = nullptr;  // header row of the state's compact cache entry, if any
+    bool entry_failed = false;     // no room in the arena: the staging row holds the mask
     if (GATHER) {
         const int32_t slot = ctx.slot[r];
-        if (slot >= 0) mrow = ctx.pool + (int64_t)slot * ctx.pool_stride;
+        if (slot >= 0 && !ctx.compact) {
+            mrow = ctx.pool + (int64_t)slot * ctx.pool_stride;
+        } else if (slot >= 0) {
+            // The entry is read without waiting for its failure flag (the header row of a cache
+            // row in use only ever names stored words); a failed entry is read again below.
+            entry = ctx.ent_hdr + (int64_t)slot * ctx.hdr_stride;
+            entry_failed = ctx.ent_fail[slot] != 0;
+            mrow = nullptr;
+        }
     }
     const bool copy_out = GATHER && mrow != own;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -555,9 +699,28 @@ apply_mask_kernel(ApplyArgs a, CtxDev ctx, unsigned long long *argkey) {
     for (int k = 0; k < APPLY_SPANS_PER_WARP; ++k) {
         const int w = (span_begin + warp + k * APPLY_WARPS) * 32 + lane;
         words[k] = 0;
-        if (span_begin + warp + k * APPLY_WARPS < span_end && w < a.W) {
-            words[k] = mrow[w];
-            if (copy_out) a.bitmask_out[(int64_t)r * a.mask_stride + w] = words[k];
+        if (span_begin + warp + k * APPLY_WARPS < span_end) {
+            if (GATHER && entry)
+                words[k] = entry_word(entry, ctx.arena, span_begin + warp + k * APPLY_WARPS, lane,
+                                      a.V, a.W);
+            else if (w < a.W)
+                words[k] = mrow[w];
+        }
+    }
+    if (GATHER && entry_failed) {  // built in this call, no room in the arena (uniform per block)
+        const uint32_t *srow = ctx.stage + (int64_t)ctx.ent_stage[ctx.slot[r]] * ctx.pool_stride;
+#pragma unroll
+        for (int k = 0; k < APPLY_SPANS_PER_WARP; ++k) {
+            const int w = (span_begin + warp + k * APPLY_WARPS) * 32 + lane;
+            if (span_begin + warp + k * APPLY_WARPS < span_end && w < a.W) words[k] = srow[w];
+        }
+    }
+    if (copy_out) {
+#pragma unroll
+        for (int k = 0; k < APPLY_SPANS_PER_WARP; ++k) {
+            const int w = (span_begin + warp + k * APPLY_WARPS) * 32 + lane;
+            if (span_begin + warp + k * APPLY_WARPS < span_end && w < a.W)
+                a.bitmask_out[(int64_t)r * a.mask_stride + w] = words[k];
         }
     }
     // Sweep 1: every chunk whose bits are all clear is a pure store; chunks that will have to
@@ -657,8 +820,13 @@ apply_mask_kernel(ApplyArgs a, CtxDev ctx, unsigned long long *argkey) {
     }
     unsigned long long packed = best.packed();
     // elements after the last whole chunk (V not a multiple of the chunk size)
-    if (blockIdx.x == gridDim.x - 1 && full_chunks * EPC < a.V)
+    if (blockIdx.x == gridDim.x - 1 && full_chunks * EPC < a.V) {
+        if (GATHER && entry) {  // the row's last words were written out by this very block
+            __syncthreads();
+            mrow = own;
+        }
         apply_scalar<E, ARGMAX>(row, mrow, full_chunks * EPC, a.V, packed);
+    }
     block_argmax_commit<ARGMAX>(packed, argkey + r);
 }
 
@@ -671,12 +839,30 @@ apply_mask_unaligned_kernel(ApplyArgs a, CtxDev ctx, unsigned long long *argkey)
     E *row = static_cast<E *>(a.logits) + (int64_t)r * a.row_stride;
     const uint32_t *own = a.bitmask + (int64_t)r * a.mask_stride;
     const uint32_t *mrow = own;
-    if (GATHER) {
-        const int32_t slot = ctx.slot[r];
-        if (slot >= 0) mrow = ctx.pool + (int64_t)slot * ctx.pool_stride;
-    }
     const int per_block = ((a.V + gridDim.x - 1) / gridDim.x + 31) & ~31;
     const int begin = blockIdx.x * per_block, end = min(begin + per_block, a.V);
+    if (GATHER) {
+        const int32_t slot = ctx.slot[r];
+        if (slot >= 0 && !ctx.compact) {
+            mrow = ctx.pool + (int64_t)slot * ctx.pool_stride;
+        } else if (slot >= 0) {
+            if (ctx.ent_fail[slot]) {
+                mrow = ctx.stage + (int64_t)ctx.ent_stage[slot] * ctx.pool_stride;
+            } else if (begin < end) {
+                // expand the block's words of the compact entry into the row's own bitmask,
+                // then mask from there
+                const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+                const int w_begin = begin >> 5, w_end = (end + 31) >> 5;
+                const uint2 *hdr_row = ctx.ent_hdr + (int64_t)slot * ctx.hdr_stride;
+                for (int span = (w_begin >> 5) + warp; span * 32 < w_end; span += APPLY_WARPS) {
+                    const uint32_t word = entry_word(hdr_row, ctx.arena, span, lane, a.V, a.W);
+                    const int w = span * 32 + lane;
+                    if (w >= w_begin && w < w_end) a.bitmask_out[(int64_t)r * a.mask_stride + w] = word;
+                }
+                __syncthreads();
+            }
+        }
+    }
     if (GATHER && mrow != own)
         for (int i = (begin >> 5) + (int)threadIdx.x; i < (end + 31) >> 5; i += APPLY_THREADS)
             a.bitmask_out[(int64_t)r * a.mask_stride + i] = mrow[i];

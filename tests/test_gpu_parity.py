@@ -160,7 +160,7 @@ class Sim:
     """One workload driven on both sides: same vocabulary, grammars, logits and tokens."""
 
     def __init__(self, wg, torch, vocab, ops, row_grammar, dtype, cache_capacity, use_cache=True,
-                 seed=0, steer=6.0, delays=None, minimize=False):
+                 seed=0, steer=6.0, delays=None, minimize=False, cache_mode=0, arena_bytes=0):
         self.wg, self.torch, self.vocab, self.dtype = wg, torch, vocab, dtype
         self.flats = [op if hasattr(op, "nodes") else flatten(op) for op in ops]
         self.trees = [oracle.Tree(f) for f in self.flats]
@@ -169,7 +169,7 @@ class Sim:
             self.grams = [g.minimized() for g in self.grams]
         self.dv = wg.Vocab(vocab.offsets, vocab.data, vocab.eos_id)
         self.B = len(row_grammar)
-        self.ctx = wg.Context(self.dv, cache_capacity, self.B)
+        self.ctx = wg.Context(self.dv, cache_capacity, self.B, cache_mode, arena_bytes)
         self.gids = [self.ctx.add_grammar(g) for g in self.grams]
         self.row_grammar = list(row_grammar)
         self.flags = (wg.WG_USE_CACHE if use_cache else wg.WG_NO_CACHE) | wg.WG_RESTART_ON_DONE
@@ -577,7 +577,7 @@ def test_large_batch_stats_reset_and_kernel_timing(wg, torch):
     assert st["cache_misses"] == len(set(rows.tolist())) == st["masks_built"]
     assert st["cache_hits"] == B - st["cache_misses"]
     ctx.reset_stats()
-    assert all(v == 0 for k, v in ctx.stats().items() if k != "cache_entries")
+    assert all(v == 0 for k, v in ctx.stats().items() if k not in ("cache_entries", "cache_bytes"))
 
 
 def test_trajectory_on_minimized_grammars(wg, torch):
