@@ -85,7 +85,8 @@ enum {
     WG_OP_SWITCH = 3, /* IfElse and its k-way generalisation */
     WG_OP_DOWHILE = 4,
     WG_OP_WAIT_UNTIL = 5,  /* a Wait whose wait "token" is a multi-byte string */
-    WG_OP_WRITE_TOKENS = 6 /* the paper's token-level Write: forced token ids        */
+    WG_OP_WRITE_TOKENS = 6, /* the paper's token-level Write: forced token ids       */
+    WG_OP_HOLE = 7          /* templates only: the place of a run-time argument      */
 };
 
 /* One node of a flattened operator tree.  Children, symbol sets and literal bytes live in
@@ -105,7 +106,8 @@ enum {
  *             (paper Section 3.2: Write emits a token sequence fixed in advance; Section 3.3:
  *             a chain of Waits each expecting one token.  Exactly these ids, one per decode
  *             step; entered and left at token boundaries only, so no token's bytes may run
- *             into or out of it.  An id beyond the vocabulary yields an empty mask.) */
+ *             into or out of it.  An id beyond the vocabulary yields an empty mask.)
+ *   HOLE      reserved = index of the argument that fills it (wg_template_compile only) */
 typedef struct wg_op_node {
     int32_t kind;
     int32_t n_child, child_off;
@@ -197,7 +199,43 @@ int32_t wg_optree_copy(const wg_optree *tree, wg_op_node *nodes, int32_t *childr
                        uint8_t *data);
 void wg_optree_free(wg_optree *tree);
 int32_t wg_compile_regex(const char *pattern, int32_t length, wg_grammar **out);
+/* The same for a pattern that is an ARGUMENT of a template (wg_template_instantiate): no EOS
+ * follows it, and because the operators decide on the symbol that follows a repetition, the
+ * pattern itself must close its last repetition (`[0-9]+"` is a fragment, `[0-9]+` is not:
+ * WG_ERR_GRAMMAR). */
+int32_t wg_compile_regex_fragment(const char *pattern, int32_t length, wg_grammar **out);
 const char *wg_regex_error(void);
+
+/* Templates: the static part of a structure compiled once, arguments spliced in per request
+ * (paper Section 3.1: the structure factory holds structures that are parameterised but not yet
+ * instantiated, and a request's arguments are combined with it into the request's state
+ * machine; contribution 2: static structure precompiled offline, dynamic arguments injected at
+ * run time and composed from predefined grammar snippets).
+ * wg_template_compile lowers an operator tree that may contain HOLE nodes (arrays as in
+ *   wg_compile_grammar); the same argument index may occur at several holes.
+ * wg_template_instantiate fills every hole with a compiled grammar -- args[i] for the holes
+ *   of argument i -- by copying table rows, without lowering anything again: a hole's entries
+ *   lead to the start of a private copy of the argument's states, and where the argument's
+ *   language is complete control continues after the hole.  The result is an ordinary grammar
+ *   whose language is that of the tree with each hole replaced by its argument's tree.  An
+ *   argument must be compiled from a tree that mentions EOS in no set (arguments sit inside
+ *   the output, they do not end it); anything else gives WG_ERR_GRAMMAR.  Argument grammars
+ *   can be compiled once and reused across requests and holes (predefined snippets), come from
+ *   wg_compile_regex, or be loaded from blobs.  Cost: proportional to the rows copied
+ *   (states x symbol classes), typically a small fraction of lowering the whole tree.
+ * Errors: WG_ERR_ARG (null, n_args different from the template's, malformed arrays),
+ *   WG_ERR_GRAMMAR, WG_ERR_CAPACITY. */
+typedef struct wg_template wg_template;
+int32_t wg_template_compile(const wg_op_node *nodes, int32_t n_nodes, const int32_t *children,
+                            int32_t n_children, const uint32_t *sets, int32_t n_sets,
+                            const uint8_t *data, int32_t n_data, int32_t root, wg_template **out);
+/* n_states counts the template's own states (placeholders included); n_holes the hole sites
+ * that can be reached; n_args = 1 + the largest argument index.  Any pointer may be NULL. */
+int32_t wg_template_info(const wg_template *tmpl, int32_t *n_states, int32_t *n_holes,
+                         int32_t *n_args);
+int32_t wg_template_instantiate(const wg_template *tmpl, const wg_grammar *const *args,
+                                int32_t n_args, wg_grammar **out);
+void wg_template_free(wg_template *tmpl);
 
 /* Returns in *out a grammar with the same language in which states that behave alike are
  * merged (classical DFA minimisation by partition refinement).  The paper caches masks per

@@ -59,6 +59,10 @@ _SIGNATURES = {
     "wg_compile_grammar": (_i32, [_vp, _i32, _vp, _i32, _vp, _i32, _vp, _i32, _i32, C.POINTER(_vp)]),
     "wg_grammar_free": (None, [_vp]),
     "wg_grammar_minimize": (_i32, [_vp, C.POINTER(_vp)]),
+    "wg_template_compile": (_i32, [_vp, _i32, _vp, _i32, _vp, _i32, _vp, _i32, _i32, C.POINTER(_vp)]),
+    "wg_template_info": (_i32, [_vp, C.POINTER(_i32), C.POINTER(_i32), C.POINTER(_i32)]),
+    "wg_template_instantiate": (_i32, [_vp, C.POINTER(_vp), _i32, C.POINTER(_vp)]),
+    "wg_template_free": (None, [_vp]),
     "wg_grammar_save": (_i32, [_vp, _vp, C.c_size_t, C.POINTER(C.c_size_t)]),
     "wg_grammar_load": (_i32, [C.c_char_p, C.c_size_t, C.POINTER(_vp)]),
     "wg_regex_to_optree": (_i32, [C.c_char_p, _i32, C.POINTER(_vp)]),
@@ -67,6 +71,7 @@ _SIGNATURES = {
     "wg_optree_copy": (_i32, [_vp, _vp, _vp, _vp, _vp]),
     "wg_optree_free": (None, [_vp]),
     "wg_compile_regex": (_i32, [C.c_char_p, _i32, C.POINTER(_vp)]),
+    "wg_compile_regex_fragment": (_i32, [C.c_char_p, _i32, C.POINTER(_vp)]),
     "wg_regex_error": (C.c_char_p, []),
     "wg_grammar_info": (_i32, [_vp, C.POINTER(_i32), C.POINTER(_i32), C.POINTER(_i32),
                                C.POINTER(_i32), C.POINTER(C.c_uint64)]),
@@ -227,11 +232,13 @@ class Grammar:
         self.n_classes, self.content_hash = c.value, hs.value
 
     @classmethod
-    def from_regex(cls, pattern) -> "Grammar":
+    def from_regex(cls, pattern, fragment: bool = False) -> "Grammar":
+        """wg_compile_regex, or wg_compile_regex_fragment for a template argument."""
         if isinstance(pattern, str):
             pattern = pattern.encode("utf-8")
         h = _vp()
-        rc = _lib.wg_compile_regex(pattern, len(pattern), C.byref(h))
+        fn = _lib.wg_compile_regex_fragment if fragment else _lib.wg_compile_regex
+        rc = fn(pattern, len(pattern), C.byref(h))
         if rc != WG_OK:
             raise WgError(rc, "wg_compile_regex: " + _lib.wg_regex_error().decode())
         return cls(_handle=h)
@@ -281,6 +288,42 @@ class Grammar:
     def close(self):
         if getattr(self, "handle", None):
             _lib.wg_grammar_free(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        self.close()
+
+
+class Template:
+    """wg_template_compile: an operator tree with holes, lowered once; ``instantiate`` splices
+    one compiled grammar per argument into the holes (wg_template_instantiate)."""
+
+    def __init__(self, flat):
+        nodes = np.ascontiguousarray(flat.nodes, np.int32)
+        children = np.ascontiguousarray(flat.children, np.int32)
+        sets = np.ascontiguousarray(flat.sets, np.uint32)
+        data = np.ascontiguousarray(flat.data, np.uint8)
+        h = _vp()
+        _check(_lib.wg_template_compile(_np_ptr(nodes), nodes.shape[0], _np_ptr(children),
+                                        children.shape[0], _np_ptr(sets), sets.shape[0],
+                                        _np_ptr(data), data.shape[0], int(flat.root), C.byref(h)),
+               "wg_template_compile")
+        self.handle = h
+        n, k, a = _i32(), _i32(), _i32()
+        _check(_lib.wg_template_info(h, C.byref(n), C.byref(k), C.byref(a)), "wg_template_info")
+        self.n_states, self.n_holes, self.n_args = n.value, k.value, a.value
+
+    def instantiate(self, args) -> Grammar:
+        args = list(args)
+        arr = (_vp * max(1, len(args)))(*[g.handle for g in args])
+        h = _vp()
+        _check(_lib.wg_template_instantiate(self.handle, arr, len(args), C.byref(h)),
+               "wg_template_instantiate")
+        return Grammar(_handle=h)
+
+    def close(self):
+        if getattr(self, "handle", None):
+            _lib.wg_template_free(self.handle)
             self.handle = None
 
     def __del__(self):

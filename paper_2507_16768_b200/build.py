@@ -9,7 +9,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libwg.so")
-SOURCES = ["wg_api.cu", "wg_lower.cpp", "wg_regex.cpp"]
+SOURCES = ["wg_api.cu", "wg_lower.cpp", "wg_regex.cpp", "wg_template.cpp"]
 HEADERS = [os.path.join(CSRC, "wg_kernels.cuh"), os.path.join(CSRC, "wg_internal.h"),
            os.path.join(ROOT, "include", "wg.h")]
 NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",

@@ -261,6 +261,65 @@ int32_t wg_compile_grammar(const wg_op_node *nodes, int32_t n_nodes, const int32
 
 void wg_grammar_free(wg_grammar *g) { delete g; }
 
+int32_t wg_template_compile(const wg_op_node *nodes, int32_t n_nodes, const int32_t *children,
+                            int32_t n_children, const uint32_t *sets, int32_t n_sets,
+                            const uint8_t *data, int32_t n_data, int32_t root, wg_template **out) {
+    NvtxRange nvtx_range("wg_template_compile");
+    if (!out) return WG_ERR_ARG;
+    *out = nullptr;
+    wg_template *t = new (std::nothrow) wg_template();
+    if (!t) return WG_ERR_ARG;
+    int32_t rc;
+    try {
+        rc = wg_lower_tree(nodes, n_nodes, children, n_children, sets, n_sets, data, n_data, root,
+                           &t->base, &t->sites);
+        if (rc == WG_OK)  // every HOLE node counts, also one that no path reaches
+            for (int32_t i = 0; i < n_nodes; ++i)
+                if (nodes[i].kind == WG_OP_HOLE && nodes[i].reserved + 1 > t->n_args)
+                    t->n_args = nodes[i].reserved + 1;
+    } catch (const std::bad_alloc &) {
+        rc = WG_ERR_CAPACITY;
+    }
+    if (rc != WG_OK) {
+        delete t;
+        return rc;
+    }
+    *out = t;
+    return WG_OK;
+}
+
+int32_t wg_template_info(const wg_template *t, int32_t *n_states, int32_t *n_holes, int32_t *n_args) {
+    if (!t) return WG_ERR_ARG;
+    if (n_states) *n_states = t->base.n_states;
+    if (n_holes) *n_holes = (int32_t)t->sites.size();
+    if (n_args) *n_args = t->n_args;
+    return WG_OK;
+}
+
+int32_t wg_template_instantiate(const wg_template *t, const wg_grammar *const *args, int32_t n_args,
+                                wg_grammar **out) {
+    NvtxRange nvtx_range("wg_template_instantiate");
+    if (!out) return WG_ERR_ARG;
+    *out = nullptr;
+    if (!t) return WG_ERR_ARG;
+    wg_grammar *g = new (std::nothrow) wg_grammar();
+    if (!g) return WG_ERR_ARG;
+    int32_t rc;
+    try {
+        rc = wg_instantiate_template(*t, args, n_args, g);
+    } catch (const std::bad_alloc &) {
+        rc = WG_ERR_CAPACITY;
+    }
+    if (rc != WG_OK) {
+        delete g;
+        return rc;
+    }
+    *out = g;
+    return WG_OK;
+}
+
+void wg_template_free(wg_template *t) { delete t; }
+
 int32_t wg_grammar_minimize(const wg_grammar *g, wg_grammar **out) {
     if (!g || !out) return WG_ERR_ARG;
     *out = nullptr;
@@ -284,7 +343,7 @@ namespace {
 constexpr uint32_t BLOB_MAGIC = 0x31474757u;  // "WGG1"
 struct BlobHeader {
     uint32_t magic, version;
-    int32_t n_states, n_classes, start, done, eos_class, has_forced;
+    int32_t n_states, n_classes, start, done, eos_class, has_forced, tail, reserved;
     uint64_t hash;
 };
 }  // namespace
@@ -297,8 +356,8 @@ int32_t wg_grammar_save(const wg_grammar *g, void *blob, size_t capacity, size_t
     *needed = total;
     if (capacity < total || !blob) return WG_ERR_CAPACITY;
     uint8_t *p = static_cast<uint8_t *>(blob);
-    const BlobHeader h{BLOB_MAGIC, 1u, g->n_states, g->n_classes, g->start, g->done, g->eos_class,
-                       g->forced_tok.empty() ? 0 : 1, g->hash};
+    const BlobHeader h{BLOB_MAGIC, 2u, g->n_states, g->n_classes, g->start, g->done, g->eos_class,
+                       g->forced_tok.empty() ? 0 : 1, g->tail, 0, g->hash};
     memcpy(p, &h, sizeof(h)); p += sizeof(h);
     memcpy(p, g->byte_class, 256); p += 256;
     memcpy(p, g->table.data(), n_table); p += n_table;
@@ -316,7 +375,8 @@ int32_t wg_grammar_load(const void *blob, size_t size, wg_grammar **out) {
     const uint8_t *p = static_cast<const uint8_t *>(blob);
     BlobHeader h;
     memcpy(&h, p, sizeof(h)); p += sizeof(h);
-    if (h.magic != BLOB_MAGIC || h.version != 1u) return WG_ERR_ARG;
+    if (h.magic != BLOB_MAGIC || h.version != 2u) return WG_ERR_ARG;
+    if (h.tail < -1 || h.tail == 0 || h.tail >= h.n_states) return WG_ERR_ARG;
     if (h.n_states < 2 || h.n_classes < 1 || h.n_classes > WG_N_SYMBOLS) return WG_ERR_ARG;
     if (h.start < 1 || h.start >= h.n_states || h.done < 1 || h.done >= h.n_states ||
         h.eos_class < 0 || h.eos_class >= h.n_classes)
@@ -329,7 +389,7 @@ int32_t wg_grammar_load(const void *blob, size_t size, wg_grammar **out) {
     bool ok = true;
     try {
         g->n_states = h.n_states; g->n_classes = h.n_classes; g->start = h.start; g->done = h.done;
-        g->eos_class = h.eos_class; g->hash = h.hash;
+        g->eos_class = h.eos_class; g->hash = h.hash; g->tail = h.tail;
         memcpy(g->byte_class, p, 256); p += 256;
         for (int b = 0; b < 256 && ok; ++b) ok = g->byte_class[b] < h.n_classes;
         g->table.resize(cells);

@@ -27,8 +27,28 @@ struct wg_grammar {
     // (as a whole token) and continues in forced_next[s]; its table row is all DEAD.  Both
     // vectors are empty when the grammar has no such state.
     std::vector<int32_t> forced_tok, forced_next;
+    // The state reached when the tree's own language is complete and only the implicit
+    // end-of-sequence is still to come; -1 when the tree mentions EOS itself (there is no
+    // implicit one then).  Splicing a grammar into a template redirects entries of this state.
+    int32_t tail = -1;
     uint64_t hash = 0;
 };
+
+// One hole of a template: a placeholder state, the argument that fills it and the state
+// where control continues once the argument's language is complete.
+struct wg_hole_site {
+    int32_t state, arg, next;
+};
+
+// A template (paper Section 3.1: a structure of the factory, parameterised but not yet
+// instantiated): the table of its static part, with one placeholder state per hole.
+struct wg_template {
+    wg_grammar base;
+    std::vector<wg_hole_site> sites;
+    int32_t n_args = 0;
+};
+
+uint64_t wg_grammar_content_hash(const wg_grammar &g);
 
 // Merges states with equal behaviour (wg_lower.cpp).  out may not alias in.
 int32_t wg_minimize_grammar(const wg_grammar &in, wg_grammar *out);
@@ -36,4 +56,9 @@ int32_t wg_minimize_grammar(const wg_grammar &in, wg_grammar *out);
 // Lowering entry (wg_lower.cpp).
 int32_t wg_lower_tree(const wg_op_node *nodes, int32_t n_nodes, const int32_t *children,
                       int32_t n_children, const uint32_t *sets, int32_t n_sets,
-                      const uint8_t *data, int32_t n_data, int32_t root, wg_grammar *out);
+                      const uint8_t *data, int32_t n_data, int32_t root, wg_grammar *out,
+                      std::vector<wg_hole_site> *sites = nullptr);
+
+// Splices one compiled grammar per argument into the template's holes (wg_template.cpp).
+int32_t wg_instantiate_template(const wg_template &t, const wg_grammar *const *args, int32_t n_args,
+                                wg_grammar *out);

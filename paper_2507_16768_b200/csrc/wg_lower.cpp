@@ -46,6 +46,7 @@ struct Lowerer {
     const uint8_t *data;
     std::vector<std::vector<Edge>> states;  // outgoing edges; symbols on no edge go to DEAD
     std::vector<int32_t> forced_tok, forced_next;  // per state; -1 = an ordinary state
+    std::vector<wg_hole_site> holes;               // placeholder states of a template
 
     int32_t new_state() {
         states.emplace_back();
@@ -97,6 +98,13 @@ struct Lowerer {
             }
             SymSet stay = stay_set(n);
             if (!stay.empty()) states[s].push_back({stay, s});
+            return s;
+        }
+        case WG_OP_HOLE: {
+            // A placeholder with no way out; instantiation replaces it by the entry of the
+            // argument's automaton lowered against k.
+            const int32_t s = new_state();
+            holes.push_back({s, n.reserved, k});
             return s;
         }
         case WG_OP_WRITE_TOKENS: {
@@ -161,7 +169,7 @@ struct Lowerer {
 
 int32_t validate(const wg_op_node *nodes, int32_t n_nodes, const int32_t *children,
                  int32_t n_children, const SymSet *sets, int32_t n_sets, const uint8_t *data,
-                 int32_t n_data, int32_t root) {
+                 int32_t n_data, int32_t root, bool allow_holes) {
     std::vector<uint8_t> used(n_nodes, 0);
     used[root] = 1;
     for (int32_t i = 0; i < n_nodes; ++i) {
@@ -180,6 +188,10 @@ int32_t validate(const wg_op_node *nodes, int32_t n_nodes, const int32_t *childr
         case WG_OP_DOWHILE: shape_ok = n.n_child == 1 && n.n_set == 4; break;
         case WG_OP_WAIT_UNTIL: shape_ok = n.n_child == 1 && n.n_set == 2; break;
         case WG_OP_WRITE_TOKENS: shape_ok = n.n_child == 0 && n.n_set == 0 && n.data_len % 4 == 0; break;
+        case WG_OP_HOLE:
+            if (!allow_holes) return WG_ERR_GRAMMAR;  // holes exist in templates only
+            shape_ok = n.n_child == 0 && n.n_set == 0 && n.data_len == 0 && n.reserved >= 0;
+            break;
         default: break;
         }
         if (!shape_ok) return WG_ERR_ARG;
@@ -220,44 +232,54 @@ int32_t validate(const wg_op_node *nodes, int32_t n_nodes, const int32_t *childr
     return WG_OK;
 }
 
-uint64_t fnv1a(uint64_t h, const void *p, size_t n) {
+// FNV-1a over 8-byte words (the tables hashed here are megabytes), then over the last bytes.
+static uint64_t fnv1a_bytes(uint64_t h, const void *p, size_t n) {
     const uint8_t *b = (const uint8_t *)p;
-    for (size_t i = 0; i < n; ++i) h = (h ^ b[i]) * 0x100000001B3ull;
-    return h;
-}
-
-uint64_t content_hash(const wg_grammar &g) {
-    uint64_t h = 0xCBF29CE484222325ull;
-    if (!g.forced_tok.empty()) {
-        h = fnv1a(h, g.forced_tok.data(), g.forced_tok.size() * sizeof(int32_t));
-        h = fnv1a(h, g.forced_next.data(), g.forced_next.size() * sizeof(int32_t));
+    size_t i = 0;
+    for (; i + 8 <= n; i += 8) {
+        uint64_t w;
+        memcpy(&w, b + i, 8);
+        h = (h ^ w) * 0x100000001B3ull;
+        h ^= h >> 29;
     }
-    h = fnv1a(h, &g.n_states, 4);
-    h = fnv1a(h, &g.n_classes, 4);
-    h = fnv1a(h, &g.done, 4);
-    h = fnv1a(h, &g.eos_class, 4);
-    h = fnv1a(h, g.byte_class, 256);
-    h = fnv1a(h, g.table.data(), g.table.size() * sizeof(int32_t));
+    for (; i < n; ++i) h = (h ^ b[i]) * 0x100000001B3ull;
     return h;
 }
 
 }  // namespace
 
+uint64_t wg_grammar_content_hash(const wg_grammar &g) {
+    uint64_t h = 0xCBF29CE484222325ull;
+    if (!g.forced_tok.empty()) {
+        h = fnv1a_bytes(h, g.forced_tok.data(), g.forced_tok.size() * sizeof(int32_t));
+        h = fnv1a_bytes(h, g.forced_next.data(), g.forced_next.size() * sizeof(int32_t));
+    }
+    h = fnv1a_bytes(h, &g.n_states, 4);
+    h = fnv1a_bytes(h, &g.n_classes, 4);
+    h = fnv1a_bytes(h, &g.done, 4);
+    h = fnv1a_bytes(h, &g.eos_class, 4);
+    h = fnv1a_bytes(h, g.byte_class, 256);
+    h = fnv1a_bytes(h, g.table.data(), g.table.size() * sizeof(int32_t));
+    return h;
+}
+
 int32_t wg_lower_tree(const wg_op_node *nodes, int32_t n_nodes, const int32_t *children,
                       int32_t n_children, const uint32_t *sets_raw, int32_t n_sets,
-                      const uint8_t *data, int32_t n_data, int32_t root, wg_grammar *out) {
+                      const uint8_t *data, int32_t n_data, int32_t root, wg_grammar *out,
+                      std::vector<wg_hole_site> *sites) {
     if (!nodes || n_nodes <= 0 || root < 0 || root >= n_nodes || n_children < 0 || n_sets < 0 ||
         n_data < 0 || (n_children > 0 && !children) || (n_sets > 0 && !sets_raw) ||
         (n_data > 0 && !data))
         return WG_ERR_ARG;
     const SymSet *sets = reinterpret_cast<const SymSet *>(sets_raw);
-    int32_t rc = validate(nodes, n_nodes, children, n_children, sets, n_sets, data, n_data, root);
+    int32_t rc = validate(nodes, n_nodes, children, n_children, sets, n_sets, data, n_data, root,
+                          sites != nullptr);
     if (rc != WG_OK) return rc;
 
     bool mentions_eos = false;
     for (int32_t s = 0; s < n_sets; ++s) mentions_eos |= sets[s].has(WG_SYM_EOS);
 
-    Lowerer lw{nodes, n_nodes, children, sets, data, {}};
+    Lowerer lw{nodes, n_nodes, children, sets, data, {}, {}, {}, {}};
     const int32_t dead = lw.new_state();  // 0: no edges
     (void)dead;
     const int32_t done = lw.new_state();
@@ -271,6 +293,8 @@ int32_t wg_lower_tree(const wg_op_node *nodes, int32_t n_nodes, const int32_t *c
 
     // breadth-first renumbering from the start state; DEAD stays 0
     const int32_t n_raw = (int32_t)lw.states.size();
+    std::vector<int32_t> hole_next(n_raw, -1);
+    for (const wg_hole_site &h : lw.holes) hole_next[h.state] = h.next;
     std::vector<int32_t> new_id(n_raw, -1);
     std::vector<int32_t> order;
     order.reserve(n_raw);
@@ -294,6 +318,11 @@ int32_t wg_lower_tree(const wg_op_node *nodes, int32_t n_nodes, const int32_t *c
             new_id[lw.forced_next[s]] = (int32_t)order.size();
             order.push_back(lw.forced_next[s]);
             q.push(lw.forced_next[s]);
+        }
+        if (hole_next[s] >= 0 && new_id[hole_next[s]] < 0) {  // what follows a hole is reachable
+            new_id[hole_next[s]] = (int32_t)order.size();
+            order.push_back(hole_next[s]);
+            q.push(hole_next[s]);
         }
     }
     if (new_id[done] < 0) {  // cannot happen for a valid tree, but keep DONE addressable
@@ -378,7 +407,14 @@ int32_t wg_lower_tree(const wg_op_node *nodes, int32_t n_nodes, const int32_t *c
             out->forced_next[i] = new_id[lw.forced_next[order[i]]];
         }
     }
-    out->hash = content_hash(*out);
+    out->tail = (!mentions_eos && new_id[k] >= 0) ? new_id[k] : -1;
+    if (sites) {
+        sites->clear();
+        for (const wg_hole_site &h : lw.holes)
+            if (new_id[h.state] >= 0)  // a hole that no path reaches needs no filling
+                sites->push_back({new_id[h.state], h.arg, new_id[h.next]});
+    }
+    out->hash = wg_grammar_content_hash(*out);
     return WG_OK;
 }
 
@@ -439,6 +475,7 @@ int32_t wg_minimize_grammar(const wg_grammar &in, wg_grammar *out) {
     out->n_classes = C;
     out->start = new_id[block[in.start]];
     out->done = new_id[block[in.done]];
+    out->tail = in.tail >= 0 ? new_id[block[in.tail]] : -1;
     out->eos_class = in.eos_class;
     memcpy(out->byte_class, in.byte_class, sizeof(in.byte_class));
     out->table.assign((size_t)M * C, 0);
@@ -456,6 +493,6 @@ int32_t wg_minimize_grammar(const wg_grammar &in, wg_grammar *out) {
                 out->forced_next[m] = new_id[block[in.forced_next[rep[m]]]];
             }
     }
-    out->hash = content_hash(*out);
+    out->hash = wg_grammar_content_hash(*out);
     return WG_OK;
 }

@@ -615,7 +615,18 @@ extern "C" {
 
 const char *wg_regex_error(void) { return g_regex_error.c_str(); }
 
+namespace {
+int32_t regex_to_optree(const char *pattern, int32_t length, bool fragment, wg_optree **out);
+}
+
 int32_t wg_regex_to_optree(const char *pattern, int32_t length, wg_optree **out) {
+    return regex_to_optree(pattern, length, false, out);
+}
+
+namespace {
+// fragment: the pattern is an argument that sits inside a larger output, so no end-of-sequence
+// symbol follows it and its last repetition must be closed by the pattern itself.
+int32_t regex_to_optree(const char *pattern, int32_t length, bool fragment, wg_optree **out) {
     if (!out) return WG_ERR_ARG;
     *out = nullptr;
     if (!pattern || length < 0 || length > (1 << 20)) return WG_ERR_ARG;
@@ -628,13 +639,18 @@ int32_t wg_regex_to_optree(const char *pattern, int32_t length, wg_optree **out)
         if (ps.more()) ps.fail("unbalanced )");
         // the program is the pattern followed by the end-of-sequence symbol
         std::vector<int> items = {root};
-        arena.push_back(Re{R_SET, Set{}, {}});
-        arena.back().set.add(WG_SYM_EOS);
-        items.push_back((int)arena.size() - 1);
+        if (!fragment) {
+            arena.push_back(Re{R_SET, Set{}, {}});
+            arena.back().set.add(WG_SYM_EOS);
+            items.push_back((int)arena.size() - 1);
+        }
         Gen gen{arena};
         Chain chain;
         Set open = gen.gen(items, 0, Set{}, chain);
-        if (!open.empty()) throw Fail{"internal: repetition left open at the end"};
+        if (!open.empty())
+            throw Fail{fragment ? "a fragment must end with a character or class that closes its "
+                                  "last repetition (the operators decide on the symbol that follows)"
+                                : "internal: repetition left open at the end"};
         auto tree = std::make_unique<wg_optree>();
         tree->root = tree->flat.emit_chain(chain);
         if (tree->root < 0) throw Fail{"internal: empty program"};
@@ -648,6 +664,7 @@ int32_t wg_regex_to_optree(const char *pattern, int32_t length, wg_optree **out)
         return WG_ERR_CAPACITY;
     }
 }
+}  // namespace
 
 void wg_optree_free(wg_optree *tree) { delete tree; }
 
@@ -673,11 +690,24 @@ int32_t wg_optree_copy(const wg_optree *tree, wg_op_node *nodes, int32_t *childr
     return WG_OK;
 }
 
+namespace {
+int32_t compile_regex(const char *pattern, int32_t length, bool fragment, wg_grammar **out);
+}
+
 int32_t wg_compile_regex(const char *pattern, int32_t length, wg_grammar **out) {
+    return compile_regex(pattern, length, false, out);
+}
+
+int32_t wg_compile_regex_fragment(const char *pattern, int32_t length, wg_grammar **out) {
+    return compile_regex(pattern, length, true, out);
+}
+
+namespace {
+int32_t compile_regex(const char *pattern, int32_t length, bool fragment, wg_grammar **out) {
     if (!out) return WG_ERR_ARG;
     *out = nullptr;
     wg_optree *tree = nullptr;
-    int32_t rc = wg_regex_to_optree(pattern, length, &tree);
+    int32_t rc = regex_to_optree(pattern, length, fragment, &tree);
     if (rc != WG_OK) return rc;
     const Flat &f = tree->flat;
     rc = wg_compile_grammar(f.nodes.data(), (int32_t)f.nodes.size(), f.children.data(),
@@ -687,5 +717,6 @@ int32_t wg_compile_regex(const char *pattern, int32_t length, wg_grammar **out) 
     wg_optree_free(tree);
     return rc;
 }
+}  // namespace
 
 }  // extern "C"

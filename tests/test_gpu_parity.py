@@ -160,11 +160,13 @@ class Sim:
     """One workload driven on both sides: same vocabulary, grammars, logits and tokens."""
 
     def __init__(self, wg, torch, vocab, ops, row_grammar, dtype, cache_capacity, use_cache=True,
-                 seed=0, steer=6.0, delays=None, minimize=False, cache_mode=0, arena_bytes=0):
+                 seed=0, steer=6.0, delays=None, minimize=False, cache_mode=0, arena_bytes=0,
+                 grams=None):
         self.wg, self.torch, self.vocab, self.dtype = wg, torch, vocab, dtype
         self.flats = [op if hasattr(op, "nodes") else flatten(op) for op in ops]
         self.trees = [oracle.Tree(f) for f in self.flats]
-        self.grams = [wg.Grammar(f) for f in self.flats]
+        # grams: library grammars made some other way than by lowering the trees (templates)
+        self.grams = list(grams) if grams is not None else [wg.Grammar(f) for f in self.flats]
         if minimize:
             self.grams = [g.minimized() for g in self.grams]
         self.dv = wg.Vocab(vocab.offsets, vocab.data, vocab.eos_id)

@@ -11,8 +11,8 @@ from typing import List
 
 import numpy as np
 
-from .optree import (ALL_BYTES, DIGITS, Cond, DoWhile, IfElse, Op, Sequence, Switch, SymSet,
-                     Wait, WaitUntil, Write, enum_trie)
+from .optree import (ALL_BYTES, DIGITS, Cond, DoWhile, Hole, IfElse, Op, Sequence, Switch, SymSet,
+                     Wait, WaitUntil, Write, enum_trie, substitute)
 
 LT = ord("<")
 
@@ -185,23 +185,33 @@ def random_template(seed: int, min_segments: int = 10, max_segments: int = 30) -
 ENUM_ALPHABET = np.frombuffer(b"abcdefghijklmnopqrstuvwxyz0123456789-_", dtype=np.uint8)
 
 
-def dynamic_snippet_template(seed: int, n_args: int = 64, enum_size: int = 40,
-                             len_min: int = 3, len_max: int = 12) -> Op:
-    """Config 5: an HTML template whose arguments are enums instantiated per request.
+def dynamic_snippet_parts(seed: int, n_args: int = 64, enum_size: int = 40,
+                          len_min: int = 3, len_max: int = 12):
+    """Config 5 as (template, arguments): the static HTML structure with one hole per section
+    (Section 3.1: parameterised, not yet instantiated) and the per-request enums that fill them.
 
-    Section ``i`` is ``<sec name="`` + one of ``enum_size`` random strings + ``">`` +
-    free text + ``</sec>``.  The enum is a trie of k-way Switch nodes; the closing quote is
-    part of every string so that no entry is a prefix of another.
+    Section ``i`` is ``<sec name="`` + one of ``enum_size`` random strings + ``">`` + free text +
+    ``</sec>``.  Each enum is a trie of k-way Switch nodes; the closing quote is part of every
+    string so that no entry is a prefix of another.  The static part does not depend on the seed.
     """
     rng = np.random.Generator(np.random.Philox(key=[seed, 0x736E6970]))
     parts: List[Op] = []
-    for _ in range(n_args):
+    args: List[Op] = []
+    for i in range(n_args):
         names = set()
         while len(names) < enum_size:
             n = int(rng.integers(len_min, len_max + 1))
             names.add(ENUM_ALPHABET[rng.integers(0, ENUM_ALPHABET.size, size=n)].tobytes() + b'"')
         parts.append(Write(b'<sec name="'))
-        parts.append(enum_trie(sorted(names)))
+        parts.append(Hole(i))
+        args.append(enum_trie(sorted(names)))
         parts.append(Write(b">"))
         parts.extend(text_slot(b"</sec>\n"))
-    return Sequence(parts)
+    return Sequence(parts), args
+
+
+def dynamic_snippet_template(seed: int, n_args: int = 64, enum_size: int = 40,
+                             len_min: int = 3, len_max: int = 12) -> Op:
+    """Config 5 as one tree: ``dynamic_snippet_parts`` with the arguments filled in."""
+    template, args = dynamic_snippet_parts(seed, n_args, enum_size, len_min, len_max)
+    return substitute(template, args)

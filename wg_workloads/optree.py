@@ -25,6 +25,9 @@ Per kind:
   DOWHILE   sets     = [allow, deny, true, false];      children = [body]
   WAIT_UNTIL sets    = [allow, deny]; data = the string waited for; children = [body]
   WRITE_TOKENS data  = the forced token ids, 4 little-endian bytes each
+  HOLE      last column of the node row = index of the argument that fills it
+            (templates only: paper Section 3.1, structures that are parameterised but not
+            yet instantiated)
 
 IfElse is the two-case SWITCH: case_0 = true_waits -> if_body, case_1 =
 false_waits -> else_body.
@@ -47,6 +50,7 @@ KIND_SWITCH = 3
 KIND_DOWHILE = 4
 KIND_WAIT_UNTIL = 5
 KIND_WRITE_TOKENS = 6
+KIND_HOLE = 7
 
 SymbolsLike = Union[bytes, str, Iterable[int], "SymSet"]
 
@@ -153,6 +157,13 @@ class WriteTokens(Op):
     """The paper's token-level Write: exactly these token ids, one per decode step."""
 
     tokens: List[int]
+
+
+@dataclass
+class Hole(Op):
+    """The place of run-time argument ``arg`` in a template tree."""
+
+    arg: int
 
 
 @dataclass
@@ -289,6 +300,10 @@ def flatten(root: Op) -> FlatTree:
             nodes[idx][6] = len(raw)
             data.extend(raw)
             kids = []
+        elif isinstance(op, Hole):
+            idx = new_node(KIND_HOLE)
+            nodes[idx][7] = int(op.arg)
+            kids = []
         elif isinstance(op, WaitUntil):
             idx = new_node(KIND_WAIT_UNTIL)
             add_sets(idx, [op.allow, op.deny])
@@ -361,3 +376,25 @@ def enum_trie(strings: Seq[bytes]) -> Op:
     out = build(strings, 0)
     assert out is not None
     return out
+
+
+def substitute(op: Optional[Op], args: Seq[Optional[Op]]) -> Optional[Op]:
+    """The tree with every ``Hole(i)`` replaced by ``args[i]`` (a fresh copy per occurrence)."""
+    import copy
+    if op is None:
+        return None
+    if isinstance(op, Hole):
+        return copy.deepcopy(args[op.arg])
+    if isinstance(op, Sequence):
+        return Sequence([substitute(p, args) for p in op.parts])
+    if isinstance(op, Switch):
+        return Switch(allow=op.allow, cases=list(op.cases), deny=op.deny,
+                      bodies=[substitute(b, args) for b in op.bodies])
+    if isinstance(op, DoWhile):
+        return DoWhile(body=substitute(op.body, args), condition=op.condition)
+    if isinstance(op, Wait):
+        return Wait(allow=op.allow, wait=op.wait, deny=op.deny, body=substitute(op.body, args))
+    if isinstance(op, WaitUntil):
+        return WaitUntil(allow=op.allow, until=op.until, deny=op.deny,
+                         body=substitute(op.body, args))
+    return op  # Write, WriteTokens: leaves without holes
