@@ -625,27 +625,12 @@ __device__ __forceinline__ void block_argmax_commit(unsigned long long best,
     }
 }
 
-// Per-lane running maximum as (float value, id): a strict float compare keeps the first of
-// equal values and treats -0.0 and +0.0 as equal; !(v <= best) also takes the very first
-// allowed element, whatever its value (best starts as NaN).
 __device__ __forceinline__ __nv_bfloat162 as_bf162(uint32_t w) {
     return *reinterpret_cast<const __nv_bfloat162 *>(&w);
 }
 __device__ __forceinline__ uint32_t bf162_bits(__nv_bfloat162 v) {
     return *reinterpret_cast<const uint32_t *>(&v);
 }
-
-struct LaneBest {
-    float v;
-    int idx;
-    __device__ __forceinline__ void offer(uint32_t f32_bits, int t) {
-        const float x = __uint_as_float(f32_bits);
-        if (!(x <= v)) { v = x; idx = t; }
-    }
-    __device__ __forceinline__ unsigned long long packed() const {
-        return idx < 0 ? 0ull : pack_best(order_key(__float_as_uint(v)), idx);
-    }
-};
 
 // Programmatic dependent launch: let the next kernel of the stream be scheduled early, then
 // wait until the kernels before this one have finished and their writes are visible.  Both
@@ -690,7 +675,12 @@ apply_mask_kernel(ApplyArgs a, CtxDev ctx, unsigned long long *argkey) {
     const int span_begin = blockIdx.x * a.spans_per_block;
     const int span_end = min(span_begin + a.spans_per_block, n_spans);
     const int full_chunks = a.V / EPC;  // chunks that lie wholly inside the row
-    LaneBest best{__uint_as_float(0x7FC00000u), -1};
+    // Per-lane running maximum: a strict float compare keeps the first of equal values and
+    // treats -0.0 and +0.0 as equal; !(m <= best_v) also takes the very first candidate chunk,
+    // whatever its value (best_v starts as NaN).
+    float best_v = __uint_as_float(0x7FC00000u);
+    int best_chunk = -1;
+    uint32_t best_bits = 0, best_w[4] = {0, 0, 0, 0};
 
     // The mask words of every span this warp will handle are fetched first, so their L2
     // latency is paid once and not once per span (the spans themselves are store streams).
@@ -804,21 +794,33 @@ apply_mask_kernel(ApplyArgs a, CtxDev ctx, unsigned long long *argkey) {
                         m = fmaxf(fmaxf(__uint_as_float(w[0]), __uint_as_float(w[1])),
                                   fmaxf(__uint_as_float(w[2]), __uint_as_float(w[3])));
                     }
-                    if (!(m <= best.v)) {
-                        const int t0 = chunk * EPC;
+                    // Only the chunk and its words are noted here (selects, no divergence: with a few
+                    // chunks per lane nearly every warp would otherwise take the slow branch);
+                    // the element is looked up once, after the loop.
+                    const bool better = !(m <= best_v);
+                    best_v = better ? m : best_v;
+                    best_chunk = better ? chunk : best_chunk;
+                    best_bits = better ? bits[q] : best_bits;
 #pragma unroll
-                        for (int i = EPC - 1; i >= 0; --i) {  // descending: the lowest id stays
-                            const uint32_t e = sizeof(E) == 2
-                                ? ((i & 1) ? (w[i >> 1] & 0xFFFF0000u) : (w[i >> 1] << 16)) : w[i];
-                            if (((bits[q] >> i) & 1u) && __uint_as_float(e) == m) best.idx = t0 + i;
-                        }
-                        best.v = m;
-                    }
+                    for (int i = 0; i < 4; ++i) best_w[i] = better ? w[i] : best_w[i];
                 }
             }
         }
     }
-    unsigned long long packed = best.packed();
+    unsigned long long packed = 0ull;
+    if (ARGMAX && best_chunk >= 0) {
+        // the lane's winning chunk (as patched: disallowed elements are -inf there, but only
+        // allowed ones count): the lowest allowed id that holds the maximum
+        const uint32_t *w = best_w;
+        int idx = -1;
+#pragma unroll
+        for (int i = EPC - 1; i >= 0; --i) {  // descending: the lowest id stays
+            const uint32_t e = sizeof(E) == 2
+                ? ((i & 1) ? (w[i >> 1] & 0xFFFF0000u) : (w[i >> 1] << 16)) : w[i];
+            if (((best_bits >> i) & 1u) && __uint_as_float(e) == best_v) idx = best_chunk * EPC + i;
+        }
+        packed = pack_best(order_key(__float_as_uint(best_v)), idx);
+    }
     // elements after the last whole chunk (V not a multiple of the chunk size)
     if (blockIdx.x == gridDim.x - 1 && full_chunks * EPC < a.V) {
         if (GATHER && entry) {  // the row's last words were written out by this very block
