@@ -35,7 +35,7 @@ from wg_workloads import BY_NAME, flatten, has_structural_byte, make_logits, mak
 BUILD_WARP_INSTR_PER_TOKEN = 0.65  # mean of the two launches under profiles/build_masks_kernel_cold_templates*.md
 
 NCU_TRAFFIC_BYTES = {
-    "json_warm": 222.2e6,       # profiles/apply_mask_kernel_json_warm.md
+    "json_warm": 221.1e6,       # profiles/apply_mask_kernel_json_warm.md
 }
 
 METRIC = "masked logit rows/s (mask build+apply)"
