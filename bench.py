@@ -62,6 +62,10 @@ def parse_args():
                    help="steer every structural character (rows then dwell in free-text slots)")
     p.add_argument("--cache-mode", default="dense", choices=["dense", "compact"],
                    help="storage of cached masks: packed rows, or allows / denies entries")
+    p.add_argument("--split", default="rows", choices=["rows", "vocab"],
+                   help="with N > 1 ranks: every rank its own batch (weak scaling, no collective), "
+                        "or every rank all rows and one slice of the vocabulary, with a MAX "
+                        "all-reduce of the packed (logit, token) pairs each step (strong scaling)")
     p.add_argument("--no-cpu-baseline", action="store_true")
     p.add_argument("--no-e2e", action="store_true")
     p.add_argument("--cpu-seconds", type=float, default=12.0)
@@ -249,6 +253,13 @@ def run_ours(args, w, steer: float) -> None:
     dv = wg.Vocab(vocab.offsets, vocab.data, vocab.eos_id)
     W = dv.W
 
+    by_vocab = args.split == "vocab"
+    if by_vocab and (args.graph or args.separate):
+        raise SystemExit("--split vocab goes through wg_decode_step_shard only")
+    from paper_2507_16768_b200.sharding import reduce_best_keys, vocab_slices
+    v_begin, v_end = vocab_slices(V, world)[rank] if by_vocab else (0, V)
+    Vs = max(v_end - v_begin, 1)          # logits columns this rank holds
+
     grammar_ids = sorted({w.grammar_of_row(r) for r in range(B)})
     compiled = {g: wg.Grammar(flatten(w.grammar(g))) for g in grammar_ids}
     n_states = sum(c.n_states for c in compiled.values())
@@ -272,10 +283,10 @@ def run_ours(args, w, steer: float) -> None:
     flags = (wg.WG_USE_CACHE if w.use_cache else wg.WG_NO_CACHE) | wg.WG_RESTART_ON_DONE
 
     # ring of pristine logits, generated on the device (seeded); at most ~40 GB in all
-    row_bytes = V * esize
+    row_bytes = Vs * esize
     ring = args.ring or int(max(4, min(64, args.steps + args.warmup, (20 << 30) // (B * row_bytes))))
     gen = torch.Generator(device="cuda")
-    gen.manual_seed(1234 + 7919 * rank)
+    gen.manual_seed(1234 + (0 if by_vocab else 7919 * rank))   # one batch for all vocabulary slices
     steer_bytes = b"" if args.steer_all else w.steer_bytes
     bonus = torch.from_numpy(has_structural_byte(vocab, steer_bytes)).cuda().to(torch.float32) * steer
     pristine = []
@@ -283,7 +294,7 @@ def run_ours(args, w, steer: float) -> None:
         x = torch.randn((B, V), generator=gen, device="cuda", dtype=torch.float32) * 2.0
         if steer:
             x += bonus
-        pristine.append(x.to(tdtype))
+        pristine.append(x[:, v_begin:v_begin + Vs].to(tdtype).contiguous())
         del x
     late = [r for r in range(B) if w.row_delay(r)]
     if late:
@@ -309,8 +320,19 @@ def run_ours(args, w, steer: float) -> None:
 
     ws = torch.empty(wg.wg_apply_workspace_bytes(B), dtype=torch.uint8, device="cuda")
 
+    d_keys = torch.zeros(B, dtype=torch.int64, device="cuda")
+
     def step(i):
-        if args.separate:
+        if by_vocab:
+            if v_end > v_begin:
+                wg.wg_decode_step_shard(ctx, d_gid, d_sid, work[i % ring], d_mask, v_begin, v_end,
+                                        d_keys, flags & wg.WG_NO_CACHE)
+            else:
+                d_keys.fill_(-(1 << 63))
+            reduce_best_keys(d_keys)
+            wg.wg_advance_keys(ctx, d_gid, d_sid, d_keys, d_tok, d_status,
+                               flags & wg.WG_RESTART_ON_DONE)
+        elif args.separate:
             # the same step through the individual entry points (7 launches instead of 4)
             wg.wg_build_masks(ctx, d_gid, d_sid, d_mask, flags & wg.WG_NO_CACHE)
             wg.wg_apply_mask(work[i % ring], d_mask, V, d_tok, ws)
@@ -359,12 +381,12 @@ def run_ours(args, w, steer: float) -> None:
     clocks = sampler.stop() if sampler else {}
 
     ms = max_over_ranks(ms, device="cuda")
-    rows_total = B * args.steps * world
+    rows_total = B * args.steps * (1 if by_vocab else world)
     value = rows_total / (ms * 1e-3)
 
     # ---- end to end through the host-buffer entry point: pinned host logits in, tokens out
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and not by_vocab:
         n_e2e = max(1, min(args.steps, 16))
         host_ring = [torch.empty((B, V), dtype=tdtype).pin_memory() for _ in range(2)]
         for h, p in zip(host_ring, pristine):
@@ -391,7 +413,7 @@ def run_ours(args, w, steer: float) -> None:
         return
 
     peak, peak_kind = measured_peak()
-    algo_bytes = B * (row_bytes + 2 * (V // 8))
+    algo_bytes = B * (row_bytes + 2 * (Vs // 8))
     apply_ms = kt["apply_ms"] / max(1, kt["steps"])
     build_ms = kt["build_ms"] / max(1, kt["steps"])
     built = stats["masks_built"]
@@ -412,7 +434,7 @@ def run_ours(args, w, steer: float) -> None:
         # tokens, early and late in a run: 0.65 per token on average).
         sm_mhz = clocks.get("sm_mhz") or 1965.0
         peak_tok = 148 * 4 * sm_mhz * 1e6 / BUILD_WARP_INSTR_PER_TOKEN
-        tok_per_s = built_timed * V / (kt["build_ms"] * 1e-3) if kt["build_ms"] > 0 else 0.0
+        tok_per_s = built_timed * Vs / (kt["build_ms"] * 1e-3) if kt["build_ms"] > 0 else 0.0
         roofline = {"kernel": "build_masks_kernel (+ row reset)", "bound": "alu",
                     "achieved": tok_per_s / 1e9, "peak": peak_tok / 1e9,
                     "unit": "G tokens checked/s", "frac": tok_per_s / peak_tok,
@@ -422,8 +444,10 @@ def run_ours(args, w, steer: float) -> None:
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
+        "scaling": "strong" if by_vocab else "weak", "vs_baseline": None, "dtype": w.dtype,
+        "data": "synthetic",
         "config": {"workload": w.name, "V": V, "batch_per_gpu": B, "logits": w.dtype,
+                   "split": args.split, "vocab_slice": [v_begin, v_end],
                    "states": n_states, "launch": "separate calls" if args.separate else
                    ("cuda graph" if args.graph else "stream"), "cache": "prewarmed" if w.prewarm else
                    ("on" if w.use_cache else "off"), "cache_mode": args.cache_mode, "steer": steer,
@@ -434,7 +458,7 @@ def run_ours(args, w, steer: float) -> None:
                              "chunks outside the timed region"},
         "roofline": roofline,
         "kernel_ms": {"lookup_and_build": build_ms, "apply": apply_ms},
-        "tokens_checked_per_s": (built * V) / (ms * 1e-3) if built else 0.0,
+        "tokens_checked_per_s": (built * Vs) / (ms * 1e-3) if built else 0.0,
         "cache": {k: stats[k] for k in ("cache_hits", "cache_misses", "masks_built",
                                          "rows_uncached", "cache_entries", "cache_bytes")},
         "rows_with_error_status": bad,

@@ -410,6 +410,40 @@ int32_t wg_decode_step(wg_ctx *ctx, const int32_t *gid, int32_t *sid, int32_t B,
                        int64_t mask_stride_words, int32_t *token_out, int32_t *status,
                        uint32_t flags, void *stream);
 
+/* The decode step for a vocabulary that is sharded over several GPUs (a tensor-parallel LM
+ * head leaves each GPU with logits[:, v_begin:v_end)).  Each GPU runs the step on its own
+ * slice -- cache lookup, build of the missing masks for the slice's tokens only, mask words
+ * out, apply -- and returns, per row, its best allowed logit and token id packed into one
+ * signed 64-bit integer whose signed order is (value, then lower token id first).  The caller
+ * takes the maximum over the GPUs (one 8-byte MAX all-reduce per row, e.g. NCCL over NVLink) and
+ * hands the result to wg_advance_keys on every GPU, which unpacks the token and advances the
+ * states.  The paper has a single mask per request (Section 1); the split follows from rows and
+ * tokens being independent and is exact: tokens, states and every masked logit equal those of
+ * wg_decode_step on the whole vocabulary.
+ *   logits_shard      device, B rows of (v_end - v_begin) elements: element 0 of a row is token
+ *                     v_begin; 16-byte aligned rows take the fast kernel
+ *   bitmask           device, B rows of W words (the WHOLE vocabulary's width); only the words
+ *                     of the slice's tokens are written
+ *   v_begin, v_end    0 <= v_begin < v_end <= V; v_begin a multiple of WG_SHARD_ALIGN, v_end a
+ *                     multiple of it or V
+ *   best_keys         device, B entries, written by this call (smallest value = no allowed token)
+ *   flags             WG_USE_CACHE or WG_NO_CACHE
+ * With the cache on, a context must always be called with the same slice: cached masks then
+ * hold the slice's words only, and calls that would read other words (another slice,
+ * wg_decode_step, wg_build_masks with the cache, wg_cache_entry_read) return WG_ERR_ARG until
+ * wg_cache_clear.  Masks cached before the first sharded call (wg_cache_prewarm) are complete
+ * and stay usable.
+ * wg_advance_keys: token_out[r] = the token packed in best_keys[r] (-1: none, status
+ * WG_ERR_EMPTY_MASK), then as wg_advance. */
+#define WG_SHARD_ALIGN 8192
+int32_t wg_decode_step_shard(wg_ctx *ctx, const int32_t *gid, const int32_t *sid, int32_t B,
+                             void *logits_shard, int32_t dtype, int64_t row_stride_elems,
+                             uint32_t *bitmask, int64_t mask_stride_words, int32_t v_begin,
+                             int32_t v_end, int64_t *best_keys, uint32_t flags, void *stream);
+int32_t wg_advance_keys(wg_ctx *ctx, const int32_t *gid, int32_t *sid, const int64_t *best_keys,
+                        int32_t B, int32_t *token_out, int32_t *status, uint32_t flags,
+                        void *stream);
+
 /* A decode step recorded once as a CUDA graph and replayed: for small batches the four kernel
  * launches of wg_decode_step cost more host time than the kernels take on the GPU, and a
  * graph launch replaces them with one call.  All arguments are those of wg_decode_step and

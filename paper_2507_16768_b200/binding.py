@@ -94,6 +94,9 @@ _SIGNATURES = {
     "wg_apply_mask_noalloc": (_i32, [_vp, _i32, _i64, _vp, _i64, _i32, _i32, _vp, _vp]),
     "wg_advance": (_i32, [_vp, _vp, _vp, _vp, _i32, _vp, _u32, _vp]),
     "wg_decode_step": (_i32, [_vp, _vp, _vp, _i32, _vp, _i32, _i64, _vp, _i64, _vp, _vp, _u32, _vp]),
+    "wg_decode_step_shard": (_i32, [_vp, _vp, _vp, _i32, _vp, _i32, _i64, _vp, _i64, _i32, _i32, _vp,
+                                    _u32, _vp]),
+    "wg_advance_keys": (_i32, [_vp, _vp, _vp, _vp, _i32, _vp, _vp, _u32, _vp]),
     "wg_step_graph_create": (_i32, [_vp, _vp, _vp, _i32, _vp, _i32, _i64, _vp, _i64, _vp, _vp, _u32,
                                     C.POINTER(_vp)]),
     "wg_step_graph_launch": (_i32, [_vp, _vp]),
@@ -493,6 +496,36 @@ def wg_decode_step(ctx: Context, gid, sid, logits, bitmask, token_out, status=No
                                _dev_ptr(token_out, torch.int32, "token_out"),
                                _dev_ptr(status, torch.int32, "status"), int(flags),
                                _stream_ptr(stream)), "wg_decode_step")
+
+
+WG_SHARD_ALIGN = 8192
+
+
+def wg_decode_step_shard(ctx: Context, gid, sid, logits_shard, bitmask, v_begin: int, v_end: int,
+                         best_keys, flags: int = WG_USE_CACHE, stream=None) -> None:
+    """The decode step on the vocabulary slice [v_begin, v_end); ``best_keys`` (int64, B) gets
+    the packed per-row maxima to be MAX-reduced over the GPUs that hold the other slices."""
+    import torch
+    B, stride = _rows(logits_shard, "logits_shard")
+    _, mstride = _rows(bitmask, "bitmask")
+    _check(_lib.wg_decode_step_shard(
+        ctx.handle, _dev_ptr(gid, torch.int32, "gid"), _dev_ptr(sid, torch.int32, "sid"), B,
+        _dev_ptr(logits_shard, None, "logits_shard"), _logits_dtype(logits_shard), stride,
+        _dev_ptr(bitmask, (torch.int32, torch.uint32), "bitmask"), mstride, int(v_begin), int(v_end),
+        _dev_ptr(best_keys, torch.int64, "best_keys"), int(flags), _stream_ptr(stream)),
+        "wg_decode_step_shard")
+
+
+def wg_advance_keys(ctx: Context, gid, sid, best_keys, token_out, status=None, flags: int = 0,
+                    stream=None) -> None:
+    import torch
+    B = gid.shape[0]
+    _check(_lib.wg_advance_keys(ctx.handle, _dev_ptr(gid, torch.int32, "gid"),
+                                _dev_ptr(sid, torch.int32, "sid"),
+                                _dev_ptr(best_keys, torch.int64, "best_keys"), B,
+                                _dev_ptr(token_out, torch.int32, "token_out"),
+                                _dev_ptr(status, torch.int32, "status"), int(flags),
+                                _stream_ptr(stream)), "wg_advance_keys")
 
 
 class StepPlan:

@@ -108,6 +108,9 @@ struct wg_ctx {
     GrammarDev *d_grammars = nullptr;
     int32_t grammar_cap = 0;
     int32_t max_batch = 0;
+    // vocabulary-sharded steps fill cached masks only inside their token range; the range they
+    // used is remembered so that no call reads cached words that were never built
+    int32_t part_begin = 0, part_end = 0;  // both 0: every cached mask is complete
     int32_t *d_stage_gid = nullptr, *d_stage_sid = nullptr;  // prewarm staging
     std::vector<void *> owned;  // every other device allocation
     std::mutex mu;
@@ -661,6 +664,7 @@ int32_t wg_ctx_add_grammar(wg_ctx *c, const wg_grammar *g, int32_t *grammar_id) 
 
 int32_t wg_cache_clear(wg_ctx *c, void *stream) {
     if (!c) return WG_ERR_ARG;
+    c->part_begin = c->part_end = 0;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int n = c->dev.hash_size > 0 ? c->dev.hash_size : 1;
     cache_clear_kernel<<<(n + 255) / 256, 256, 0, st>>>(c->dev);
@@ -713,7 +717,8 @@ int32_t launch_build(wg_ctx *c, const BuildWork &work, int max_entries, cudaStre
     // few masks: small chunks so that one mask still spreads over many blocks
     BuildWork w = work;
     w.chunk = max_entries <= 32 ? 2048 : BUILD_CHUNK_MAX;
-    const long long n_chunks = ((long long)v.W * 32 + w.chunk - 1) / w.chunk;
+    if (w.t_last == 0) { w.t_first = 0; w.t_last = v.W * 32; }  // the whole vocabulary
+    const long long n_chunks = ((long long)(w.t_last - w.t_first) + w.chunk - 1) / w.chunk;
     long long items = (long long)max_entries * n_chunks;
     long long grid = (long long)sm_count() * 8;  // 8 resident blocks of 256 threads per SM
     if (items < grid) grid = items;
@@ -735,7 +740,7 @@ bool rows_aligned(const void *p, int64_t stride_elems, size_t elem) {
 // warp of a block takes 1, 2 or 4 spans of 1024 tokens; the smaller counts are used while the
 // grid would otherwise hold fewer than about four waves of blocks (a short last wave costs).
 dim3 apply_grid(ApplyArgs &a) {
-    const int n_spans = (a.W + 31) / 32;
+    const int n_spans = (a.W + 31) / 32 - a.span_first;
     int per_warp = APPLY_SPANS_PER_WARP;
     while (per_warp > 1 &&
            (long long)a.B * ((n_spans + APPLY_WARPS * per_warp - 1) / (APPLY_WARPS * per_warp)) <
@@ -802,12 +807,13 @@ int32_t wg_build_masks(wg_ctx *c, const int32_t *gid, const int32_t *sid, int32_
     if (row_stride_words < W || (flags & ~(uint32_t)WG_NO_CACHE)) return WG_ERR_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (flags & WG_NO_CACHE) {
-        BuildWork work{gid, sid, nullptr, bitmask, row_stride_words, nullptr, B, 0};
+        BuildWork work{gid, sid, nullptr, bitmask, row_stride_words, nullptr, B, 0, 0, 0};
         return launch_build(c, work, B, st);
     }
+    if (c->part_end != 0) return WG_ERR_ARG;  // cached masks are partial: see wg_decode_step_shard
     cache_lookup_insert_kernel<<<1, 1024, 0, st>>>(c->dev, gid, sid, B, bitmask, row_stride_words);
     WG_LAUNCHED();
-    BuildWork work{c->dev.bl_gid, c->dev.bl_sid, c->dev.bl_dst, nullptr, 0, c->dev.bl_count, 0, 0};
+    BuildWork work{c->dev.bl_gid, c->dev.bl_sid, c->dev.bl_dst, nullptr, 0, c->dev.bl_count, 0, 0, 0, 0};
     int32_t rc = launch_build(c, work, B, st);
     if (rc != WG_OK) return rc;
     dim3 grid((unsigned)((W + 1023) / 1024), (unsigned)B);
@@ -832,7 +838,7 @@ int32_t wg_apply_mask(void *logits, int32_t dtype, int64_t row_stride_elems,
     if (row_stride_elems < V || mask_stride_words < W) return WG_ERR_ARG;
     if (argmax_out && (!workspace || (uintptr_t)workspace % 8 != 0)) return WG_ERR_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    ApplyArgs a{logits, row_stride_elems, bitmask, nullptr, mask_stride_words, B, V, W, 0};
+    ApplyArgs a{logits, row_stride_elems, bitmask, nullptr, mask_stride_words, B, V, W, 0, 0};
     CtxDev none{};
     if (!argmax_out) return launch_apply<false, false>(dtype, a, none, nullptr, st);
     unsigned long long *keys = static_cast<unsigned long long *>(workspace);
@@ -890,7 +896,7 @@ int32_t wg_apply_mask_noalloc(void *logits, int32_t dtype, int64_t row_stride_el
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     // the array still holds the previous call's maxima: the rows in use must start at zero
     WG_CUDA(cudaMemsetAsync(keys, 0, sizeof(unsigned long long) * (size_t)B, st));
-    ApplyArgs a{logits, row_stride_elems, bitmask, nullptr, mask_stride_words, B, V, W, 0};
+    ApplyArgs a{logits, row_stride_elems, bitmask, nullptr, mask_stride_words, B, V, W, 0, 0};
     CtxDev none{};
     rc = launch_apply<true, false>(dtype, a, none, keys, st);
     if (rc != WG_OK) return rc;
@@ -905,10 +911,79 @@ int32_t wg_advance(wg_ctx *c, const int32_t *gid, int32_t *sid, const int32_t *t
     if (!batch_ok(c, B) || !gid || !sid || !token) return WG_ERR_ARG;
     if (flags & ~(uint32_t)WG_RESTART_ON_DONE) return WG_ERR_ARG;
     advance_kernel<<<(B + 127) / 128, 128, 0, static_cast<cudaStream_t>(stream)>>>(
-        c->vocab->dev, c->dev, gid, sid, token, nullptr, B, status, flags, 0);
+        c->vocab->dev, c->dev, gid, sid, token, nullptr, B, status, flags, 0,
+        (const long long *)nullptr);
     WG_LAUNCHED();
     return WG_OK;
 }
+
+}  // extern "C"
+
+namespace {
+// One decode step over the tokens [v_begin, v_end) of the vocabulary.  `logits` holds those
+// tokens only (element 0 of a row is token v_begin).  With best_keys the step ends by handing
+// the packed maxima to the caller instead of advancing the states.
+int32_t decode_step_impl(wg_ctx *c, const int32_t *gid, int32_t *sid, int32_t B, void *logits,
+                         int32_t dtype, int64_t row_stride_elems, uint32_t *bitmask,
+                         int64_t mask_stride_words, int32_t v_begin, int32_t v_end,
+                         int32_t *token_out, long long *best_keys, int32_t *status, uint32_t flags,
+                         cudaStream_t st) {
+    const VocabDev &v = c->vocab->dev;
+    const bool no_cache = (flags & WG_NO_CACHE) != 0;
+    const bool whole = v_begin == 0 && v_end == v.V;
+    if (!no_cache) {
+        // cached masks hold the words of one token range only once a partial step has run
+        if (c->part_end != 0 && (c->part_begin != v_begin || c->part_end != v_end)) return WG_ERR_ARG;
+        if (!whole) { c->part_begin = v_begin; c->part_end = v_end; }
+    }
+    const size_t esize = dtype == WG_DTYPE_BF16 ? 2 : 4;
+    // token t of the vocabulary is element t of the (virtual) row that starts v_begin earlier
+    void *row0 = static_cast<char *>(logits) - (size_t)v_begin * esize;
+    const int W_end = (v_end + 31) / 32;
+    ApplyArgs a{row0, row_stride_elems, bitmask, bitmask, mask_stride_words, B, v_end, W_end, 0,
+                v_begin / 1024};
+    const int32_t t_last = v_end == v.V ? v.W * 32 : v_end;
+    // Every kernel of the step is launched with programmatic stream serialization and starts
+    // with griddepcontrol.wait, so launch latency and block scheduling of a kernel overlap the
+    // tail of the one before it (also across consecutive steps on one stream).
+    int32_t rc;
+    if ((rc = timing_mark(c, 0, st)) != WG_OK) return rc;
+    if (no_cache) {
+        // rows have no pool row; the packed maxima were left at zero by the last advance
+        WG_CUDA(launch_pdl(reset_rows_kernel, dim3((B + 255) / 256), dim3(256), st, c->dev, B));
+        WG_LAUNCHED();
+        BuildWork work{gid, sid, nullptr, bitmask, mask_stride_words, nullptr, B, 0, v_begin, t_last};
+        rc = launch_build(c, work, B, st, true);
+    } else {
+        WG_CUDA(launch_pdl(cache_lookup_insert_kernel, dim3(1), dim3(1024), st, c->dev, gid, sid, B,
+                           bitmask, mask_stride_words));
+        WG_LAUNCHED();
+        BuildWork work{c->dev.bl_gid, c->dev.bl_sid, c->dev.bl_dst, nullptr, 0, c->dev.bl_count, 0, 0,
+                       v_begin, t_last};
+        rc = launch_build(c, work, B, st, true);
+    }
+    if (rc != WG_OK) return rc;
+    if ((rc = timing_mark(c, 1, st)) != WG_OK) return rc;
+    if ((rc = timing_mark(c, 2, st)) != WG_OK) return rc;
+    rc = no_cache ? launch_apply<true, false>(dtype, a, c->dev, c->dev.argkey, st, true)
+                  : launch_apply<true, true>(dtype, a, c->dev, c->dev.argkey, st, true);
+    if (rc != WG_OK) return rc;
+    if ((rc = timing_mark(c, 3, st)) != WG_OK) return rc;
+    if (best_keys) {
+        WG_CUDA(launch_pdl(export_keys_kernel, dim3((B + 127) / 128), dim3(128), st, c->dev,
+                           best_keys, B));
+        WG_LAUNCHED();
+        return WG_OK;
+    }
+    WG_CUDA(launch_pdl(advance_kernel, dim3((B + 127) / 128), dim3(128), st, v, c->dev, gid, sid,
+                       (const int32_t *)nullptr, token_out, B, status,
+                       (uint32_t)(flags & WG_RESTART_ON_DONE), 1, (const long long *)nullptr));
+    WG_LAUNCHED();
+    return WG_OK;
+}
+}  // namespace
+
+extern "C" {
 
 int32_t wg_decode_step(wg_ctx *c, const int32_t *gid, int32_t *sid, int32_t B, void *logits,
                        int32_t dtype, int64_t row_stride_elems, uint32_t *bitmask,
@@ -920,37 +995,40 @@ int32_t wg_decode_step(wg_ctx *c, const int32_t *gid, int32_t *sid, int32_t B, v
     if (flags & ~(uint32_t)(WG_NO_CACHE | WG_RESTART_ON_DONE)) return WG_ERR_ARG;
     const VocabDev &v = c->vocab->dev;
     if (row_stride_elems < v.V || mask_stride_words < v.W) return WG_ERR_ARG;
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    ApplyArgs a{logits, row_stride_elems, bitmask, bitmask, mask_stride_words, B, v.V, v.W, 0};
-    const bool no_cache = (flags & WG_NO_CACHE) != 0;
-    // Every kernel of the step is launched with programmatic stream serialization and starts
-    // with griddepcontrol.wait, so launch latency and block scheduling of a kernel overlap the
-    // tail of the one before it (also across consecutive steps on one stream).
-    int32_t rc;
-    if ((rc = timing_mark(c, 0, st)) != WG_OK) return rc;
-    if (no_cache) {
-        // rows have no pool row; the packed maxima were left at zero by the last advance
-        WG_CUDA(launch_pdl(reset_rows_kernel, dim3((B + 255) / 256), dim3(256), st, c->dev, B));
-        WG_LAUNCHED();
-        BuildWork work{gid, sid, nullptr, bitmask, mask_stride_words, nullptr, B, 0};
-        rc = launch_build(c, work, B, st, true);
-    } else {
-        WG_CUDA(launch_pdl(cache_lookup_insert_kernel, dim3(1), dim3(1024), st, c->dev, gid, sid, B,
-                           bitmask, mask_stride_words));
-        WG_LAUNCHED();
-        BuildWork work{c->dev.bl_gid, c->dev.bl_sid, c->dev.bl_dst, nullptr, 0, c->dev.bl_count, 0, 0};
-        rc = launch_build(c, work, B, st, true);
-    }
-    if (rc != WG_OK) return rc;
-    if ((rc = timing_mark(c, 1, st)) != WG_OK) return rc;
-    if ((rc = timing_mark(c, 2, st)) != WG_OK) return rc;
-    rc = no_cache ? launch_apply<true, false>(dtype, a, c->dev, c->dev.argkey, st, true)
-                  : launch_apply<true, true>(dtype, a, c->dev, c->dev.argkey, st, true);
-    if (rc != WG_OK) return rc;
-    if ((rc = timing_mark(c, 3, st)) != WG_OK) return rc;
-    WG_CUDA(launch_pdl(advance_kernel, dim3((B + 127) / 128), dim3(128), st, v, c->dev, gid, sid,
-                       (const int32_t *)nullptr, token_out, B, status,
-                       (uint32_t)(flags & WG_RESTART_ON_DONE), 1));
+    return decode_step_impl(c, gid, sid, B, logits, dtype, row_stride_elems, bitmask,
+                            mask_stride_words, 0, v.V, token_out, nullptr, status, flags,
+                            static_cast<cudaStream_t>(stream));
+}
+
+int32_t wg_decode_step_shard(wg_ctx *c, const int32_t *gid, const int32_t *sid, int32_t B,
+                             void *logits_shard, int32_t dtype, int64_t row_stride_elems,
+                             uint32_t *bitmask, int64_t mask_stride_words, int32_t v_begin,
+                             int32_t v_end, int64_t *best_keys, uint32_t flags, void *stream) {
+    NvtxRange nvtx_range("wg_decode_step_shard");
+    if (!batch_ok(c, B) || !gid || !sid || !logits_shard || !bitmask || !best_keys) return WG_ERR_ARG;
+    if (dtype != WG_DTYPE_BF16 && dtype != WG_DTYPE_FP32) return WG_ERR_ARG;
+    if (flags & ~(uint32_t)WG_NO_CACHE) return WG_ERR_ARG;
+    const VocabDev &v = c->vocab->dev;
+    if (v_begin < 0 || v_begin >= v_end || v_end > v.V || v_begin % WG_SHARD_ALIGN != 0 ||
+        (v_end != v.V && v_end % WG_SHARD_ALIGN != 0))
+        return WG_ERR_ARG;
+    if (row_stride_elems < v_end - v_begin || mask_stride_words < v.W) return WG_ERR_ARG;
+    static_assert(sizeof(long long) == sizeof(int64_t), "packed maxima are 64-bit");
+    return decode_step_impl(c, gid, const_cast<int32_t *>(sid), B, logits_shard, dtype,
+                            row_stride_elems, bitmask, mask_stride_words, v_begin, v_end, nullptr,
+                            reinterpret_cast<long long *>(best_keys), nullptr, flags,
+                            static_cast<cudaStream_t>(stream));
+}
+
+int32_t wg_advance_keys(wg_ctx *c, const int32_t *gid, int32_t *sid, const int64_t *best_keys,
+                        int32_t B, int32_t *token_out, int32_t *status, uint32_t flags,
+                        void *stream) {
+    NvtxRange nvtx_range("wg_advance_keys");
+    if (!batch_ok(c, B) || !gid || !sid || !best_keys || !token_out) return WG_ERR_ARG;
+    if (flags & ~(uint32_t)WG_RESTART_ON_DONE) return WG_ERR_ARG;
+    advance_kernel<<<(B + 127) / 128, 128, 0, static_cast<cudaStream_t>(stream)>>>(
+        c->vocab->dev, c->dev, gid, sid, nullptr, token_out, B, status, flags, 2,
+        reinterpret_cast<const long long *>(best_keys));
     WG_LAUNCHED();
     return WG_OK;
 }
@@ -1073,6 +1151,7 @@ int32_t wg_cache_entry_read(wg_ctx *c, int32_t grammar_id, int32_t state, int32_
                             int32_t *n_listed, int32_t *ids_host, int32_t ids_capacity,
                             int64_t *entry_bytes, void *stream) {
     if (!c || !c->dev.compact || ids_capacity < 0 || (ids_capacity > 0 && !ids_host)) return WG_ERR_ARG;
+    if (c->part_end != 0) return WG_ERR_ARG;  // cached masks hold one vocabulary slice only
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const VocabDev &v = c->vocab->dev;
     if (kind) *kind = -1;
@@ -1138,7 +1217,7 @@ int32_t wg_cache_prewarm(wg_ctx *c, int32_t grammar_id, void *stream) {
         cache_lookup_insert_kernel<<<1, 1024, 0, st>>>(c->dev, c->d_stage_gid, c->d_stage_sid, n,
                                                        nullptr, 0);
         WG_LAUNCHED();
-        BuildWork work{c->dev.bl_gid, c->dev.bl_sid, c->dev.bl_dst, nullptr, 0, c->dev.bl_count, 0, 0};
+        BuildWork work{c->dev.bl_gid, c->dev.bl_sid, c->dev.bl_dst, nullptr, 0, c->dev.bl_count, 0, 0, 0, 0};
         rc = launch_build(c, work, n, st);
         if (rc != WG_OK) return rc;
     }

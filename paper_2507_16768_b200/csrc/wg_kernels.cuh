@@ -234,6 +234,7 @@ struct BuildWork {
     const int32_t *count_ptr;   // number of entries on the device, or NULL: use count
     int32_t count;
     int32_t chunk;              // tokens per work item: a multiple of 32, <= BUILD_CHUNK_MAX
+    int32_t t_first, t_last;    // tokens [t_first, t_last) are built: whole chunks, or up to W * 32
 };
 
 // COMPACT: the cache keeps allows / denies entries; finished chunks are also stored as spans.
@@ -253,13 +254,12 @@ build_masks_kernel(VocabDev v, CtxDev ctx, BuildWork work) {
     __syncthreads();
     const int lane = threadIdx.x & 31;
     const int n_entries = work.count_ptr ? *work.count_ptr : work.count;
-    const int n_tok = v.W * 32;
-    const int n_chunks = (n_tok + work.chunk - 1) / work.chunk;
+    const int n_chunks = (work.t_last - work.t_first + work.chunk - 1) / work.chunk;
     const long long n_items = (long long)n_entries * n_chunks;
     for (long long item = blockIdx.x; item < n_items; item += gridDim.x) {
         const int m = (int)(item / n_chunks);
-        const int t_begin = (int)(item % n_chunks) * work.chunk;
-        const int t_end = min(t_begin + work.chunk, n_tok);
+        const int t_begin = work.t_first + (int)(item % n_chunks) * work.chunk;
+        const int t_end = min(t_begin + work.chunk, work.t_last);
         const int gid = work.gid[m];
         uint32_t s0 = (uint32_t)work.sid[m];
         uint32_t *dst = work.dst_list ? work.dst_list[m] : work.dst_base + (int64_t)m * work.dst_stride;
@@ -267,7 +267,7 @@ build_masks_kernel(VocabDev v, CtxDev ctx, BuildWork work) {
         GrammarDev g = {};
         if (known) g = ctx.grammars[gid];
         if (!known || s0 >= (uint32_t)g.n_states) s0 = 0;  // unknown state: an all-zero row
-        if (t_begin == 0 && threadIdx.x == 0) {
+        if (t_begin == work.t_first && threadIdx.x == 0) {
             atomicAdd(&ctx.stats[ST_BUILT], 1ull);
             if (s0 == 0 && work.sid[m] != 0) atomicAdd(&ctx.stats[ST_BAD_STATE], 1ull);
         }
@@ -589,6 +589,10 @@ struct ApplyArgs {
     int64_t mask_stride;      // words
     int32_t B, V, W;
     int32_t spans_per_block;  // spans (32 mask words) each block handles
+    int32_t span_first;       // vocabulary shard: the first span that is handled.  `logits` then
+                              // points v_begin elements BEFORE the shard's first element, so that
+                              // token t of the whole vocabulary is element t of a row, and V is
+                              // the shard's end
 };
 
 // element-wise masking of [begin, end) of one row; any alignment
@@ -642,7 +646,8 @@ __device__ __forceinline__ void pdl_enter() {
 
 // grid = (blocks per row, B).  Requires 16-byte aligned rows (pointer and stride).
 template <typename E, bool ARGMAX, bool GATHER>
-__global__ void __launch_bounds__(APPLY_THREADS)
+// (every variant fits 64 registers, four blocks per SM; one of them has to be told)
+__global__ void __launch_bounds__(APPLY_THREADS, (sizeof(E) == 4 && ARGMAX && !GATHER) ? 4 : 0)
 apply_mask_kernel(ApplyArgs a, CtxDev ctx, unsigned long long *argkey) {
     constexpr int EPC = ElemTraits<E>::PER_CHUNK;  // elements per chunk: bits per lane
     constexpr int CHUNKS_PER_WORD = 32 / EPC;      // 4 (bf16) or 8 (fp32)
@@ -672,7 +677,7 @@ apply_mask_kernel(ApplyArgs a, CtxDev ctx, unsigned long long *argkey) {
     const bool copy_out = GATHER && mrow != own;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int n_spans = (a.W + 31) / 32;
-    const int span_begin = blockIdx.x * a.spans_per_block;
+    const int span_begin = a.span_first + blockIdx.x * a.spans_per_block;
     const int span_end = min(span_begin + a.spans_per_block, n_spans);
     const int full_chunks = a.V / EPC;  // chunks that lie wholly inside the row
     // Per-lane running maximum: a strict float compare keeps the first of equal values and
@@ -841,8 +846,9 @@ apply_mask_unaligned_kernel(ApplyArgs a, CtxDev ctx, unsigned long long *argkey)
     E *row = static_cast<E *>(a.logits) + (int64_t)r * a.row_stride;
     const uint32_t *own = a.bitmask + (int64_t)r * a.mask_stride;
     const uint32_t *mrow = own;
-    const int per_block = ((a.V + gridDim.x - 1) / gridDim.x + 31) & ~31;
-    const int begin = blockIdx.x * per_block, end = min(begin + per_block, a.V);
+    const int t_first = a.span_first * 1024;
+    const int per_block = ((a.V - t_first + gridDim.x - 1) / gridDim.x + 31) & ~31;
+    const int begin = t_first + blockIdx.x * per_block, end = min(begin + per_block, a.V);
     if (GATHER) {
         const int32_t slot = ctx.slot[r];
         if (slot >= 0 && !ctx.compact) {
@@ -882,14 +888,38 @@ __global__ void argmax_finish_kernel(const unsigned long long *argkey, int B, in
 // K6: advance.  One thread per row; at most a handful of dependent lookups.
 // from_keys: the token comes from the packed maxima of the fused step and is written out.
 // ---------------------------------------------------------------------------------------
+// Packed maxima leave the library as signed 64-bit integers whose signed order is the order of
+// the packed keys (top bit flipped), so that an all-reduce with MAX over ranks picks the winner.
+__device__ __forceinline__ long long key_to_signed(unsigned long long k) {
+    return (long long)(k ^ 0x8000000000000000ull);
+}
+__device__ __forceinline__ unsigned long long key_from_signed(long long k) {
+    return (unsigned long long)k ^ 0x8000000000000000ull;
+}
+
+// The fused step's packed maxima out to the caller, and zeroed for the next step.
+__global__ void export_keys_kernel(CtxDev ctx, long long *out, int B) {
+    pdl_enter();
+    const int r = blockIdx.x * blockDim.x + threadIdx.x;
+    if (r >= B) return;
+    out[r] = key_to_signed(ctx.argkey[r]);
+    ctx.argkey[r] = 0ull;
+}
+
+// from_keys: 0 = the tokens come in token_in; 1 = from the fused step's packed maxima; 2 = from
+// ext_keys (signed packed maxima, e.g. after an all-reduce over vocabulary shards).
 __global__ void advance_kernel(VocabDev v, CtxDev ctx, const int32_t *gid, int32_t *sid,
                                const int32_t *token_in, int32_t *token_out, int B,
-                               int32_t *status, uint32_t flags, int from_keys) {
+                               int32_t *status, uint32_t flags, int from_keys,
+                               const long long *ext_keys) {
     pdl_enter();
     const int r = blockIdx.x * blockDim.x + threadIdx.x;
     if (r >= B) return;
     int t;
-    if (from_keys) {
+    if (from_keys == 2) {
+        t = unpack_best(key_from_signed(ext_keys[r]));
+        token_out[r] = t;
+    } else if (from_keys) {
         t = unpack_best(ctx.argkey[r]);
         ctx.argkey[r] = 0ull;  // ready for the next step
         token_out[r] = t;

@@ -1,9 +1,16 @@
-"""Multi-GPU host logic: rows of a batch are independent, so a job is split by rows.
+"""Multi-GPU host logic.
 
-Every rank holds the whole vocabulary, its own grammar tables and its own mask cache, and
-decodes its slice of the batch; no collective sits on the data path.  The only exchanges are
-the ones a benchmark or an engine needs around it: the slowest rank's time, and the chosen
-tokens if somebody wants them in one place.
+Rows of a batch are independent, so the default split is by rows: every rank holds the whole
+vocabulary, its own grammar tables and its own mask cache, and decodes its slice of the batch;
+no collective sits on the data path.  The only exchanges are the ones a benchmark or an engine
+needs around it: the slowest rank's time, and the chosen tokens if somebody wants them in one
+place.
+
+The second split is by vocabulary, for engines whose LM head is tensor-parallel: every rank
+holds all rows but only logits[:, v_begin:v_end).  Then the path has one real exchange step:
+the per-row (best logit, token id) pairs, packed into one int64 each by
+``wg_decode_step_shard``, are MAX-reduced over the ranks (``reduce_best_keys``) before
+``wg_advance_keys`` advances the states on every rank.
 """
 from __future__ import annotations
 
@@ -47,3 +54,25 @@ def gather_tokens(tokens, n_rows: int) -> List[int]:
     for (b, e), part in zip(sizes, parts):
         out.extend(int(x) for x in part[:e - b].tolist())
     return out
+
+
+def vocab_slices(V: int, world: int, align: int = 8192) -> List[Tuple[int, int]]:
+    """[begin, end) of every rank's vocabulary slice: contiguous, every boundary but the last a
+    multiple of ``align`` (what ``wg_decode_step_shard`` asks for), sizes as equal as that
+    allows.  A rank whose slice would be empty (more ranks than aligned pieces) gets (V, V)."""
+    if world < 1 or V < 1 or align < 1:
+        raise ValueError("bad slice request")
+    pieces = (V + align - 1) // align
+    out = []
+    for r in range(world):
+        b, e = shard_rows(pieces, world, r)
+        out.append((min(b * align, V), min(e * align, V)))
+    return out
+
+
+def reduce_best_keys(keys) -> None:
+    """In place: the per-row maximum of the packed (value, token) keys over all ranks.  One
+    8-byte element per row; NCCL runs it over NVLink / NVSwitch, gloo on CPU."""
+    import torch.distributed as dist
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(keys, op=dist.ReduceOp.MAX)
