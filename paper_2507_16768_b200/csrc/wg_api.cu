@@ -506,6 +506,7 @@ int32_t wg_ctx_create_ex(const wg_vocab *vocab, int32_t cache_capacity, int32_t 
     take(&d.bl_sid, (size_t)max_batch);
     take(&d.bl_dst, (size_t)max_batch);
     take(&d.bl_count, 1);
+    take(&d.build_next, 2);
     take(&d.argkey, (size_t)max_batch);
     take(&d.stats, (size_t)ST_COUNT);
     take(&c->d_stage_gid, (size_t)max_batch);
@@ -513,12 +514,14 @@ int32_t wg_ctx_create_ex(const wg_vocab *vocab, int32_t cache_capacity, int32_t 
     c->grammar_cap = 64;
     take(&c->d_grammars, (size_t)c->grammar_cap);
     if (rc == WG_OK) {
+        d.build_done = d.build_next + 1;
         d.grammars = c->d_grammars;
         d.n_grammars = 0;
         if (cudaMemset(d.keys, 0, sizeof(unsigned long long) * (size_t)(d.hash_size ? d.hash_size : 1)) != cudaSuccess ||
             cudaMemset(d.vals, 0xFF, sizeof(int32_t) * (size_t)(d.hash_size ? d.hash_size : 1)) != cudaSuccess ||
             cudaMemset(d.n_slots, 0, sizeof(int32_t)) != cudaSuccess ||
             cudaMemset(d.bl_count, 0, sizeof(int32_t)) != cudaSuccess ||
+            cudaMemset(d.build_next, 0, 2 * sizeof(int32_t)) != cudaSuccess ||
             cudaMemset(d.argkey, 0, sizeof(unsigned long long) * (size_t)max_batch) != cudaSuccess ||
             cudaMemset(d.stats, 0, sizeof(unsigned long long) * ST_COUNT) != cudaSuccess)
             rc = WG_ERR_CUDA;
@@ -720,10 +723,20 @@ int32_t launch_build(wg_ctx *c, const BuildWork &work, int max_entries, cudaStre
     if (w.t_last == 0) { w.t_first = 0; w.t_last = v.W * 32; }  // the whole vocabulary
     const long long n_chunks = ((long long)(w.t_last - w.t_first) + w.chunk - 1) / w.chunk;
     long long items = (long long)max_entries * n_chunks;
-    long long grid = (long long)sm_count() * 8;  // 8 resident blocks of 256 threads per SM
+    auto kernel = c->dev.compact ? build_masks_kernel<true> : build_masks_kernel<false>;
+    // One block per resident slot: the blocks stride over the items, so blocks that had to wait
+    // for a slot would start their equal share late and stretch the launch.
+    static int resident[2] = {0, 0};
+    int &per_sm = resident[c->dev.compact ? 1 : 0];
+    if (per_sm == 0) {
+        int n = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, BUILD_THREADS, 0) != cudaSuccess || n < 1)
+            n = 4;
+        per_sm = n;
+    }
+    long long grid = (long long)sm_count() * per_sm;
     if (items < grid) grid = items;
     if (grid < 1) grid = 1;
-    auto kernel = c->dev.compact ? build_masks_kernel<true> : build_masks_kernel<false>;
     if (pdl)
         WG_CUDA(launch_pdl(kernel, dim3((unsigned)grid), dim3(BUILD_THREADS), st, v, c->dev, w));
     else

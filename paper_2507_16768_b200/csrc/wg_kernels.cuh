@@ -58,6 +58,8 @@ struct CtxDev {
     int32_t *bl_gid, *bl_sid;  // [max_batch] build list
     uint32_t **bl_dst;         // [max_batch] where each listed mask goes
     int32_t *bl_count;
+    int32_t *build_next, *build_done;  // work counter of the build kernel and blocks finished;
+                                       // both zero between launches
     unsigned long long *argkey;  // [max_batch] packed (value key, ~id) maxima
     unsigned long long *stats;   // [ST_COUNT]
     // compact cache (allows / denies storage instead of dense pool rows); pool is NULL then
@@ -256,7 +258,11 @@ build_masks_kernel(VocabDev v, CtxDev ctx, BuildWork work) {
     const int n_entries = work.count_ptr ? *work.count_ptr : work.count;
     const int n_chunks = (work.t_last - work.t_first + work.chunk - 1) / work.chunk;
     const long long n_items = (long long)n_entries * n_chunks;
-    for (long long item = blockIdx.x; item < n_items; item += gridDim.x) {
+    // Items differ a lot in cost (a literal state decides nearly everything word-wise, a
+    // free-text state walks thousands of tokens), so after its first item a block takes the next
+    // one from a device counter instead of a fixed stride.
+    __shared__ long long next_item;
+    for (long long item = blockIdx.x; item < n_items; item = next_item) {
         const int m = (int)(item / n_chunks);
         const int t_begin = work.t_first + (int)(item % n_chunks) * work.chunk;
         const int t_end = min(t_begin + work.chunk, work.t_last);
@@ -358,6 +364,17 @@ build_masks_kernel(VocabDev v, CtxDev ctx, BuildWork work) {
                 store_chunk_spans(ctx.ent_hdr + (int64_t)row * ctx.hdr_stride, ctx.arena, ctx.arena_top,
                                   ctx.arena_words, ctx.ent_fail + row, ctx.stats + ST_UNCACHED,
                                   t_begin >> 10, n_words, words, v.V, v.W);
+        }
+        __syncthreads();  // (also: nobody reads next_item any more before it is rewritten)
+        if (threadIdx.x == 0) next_item = (long long)gridDim.x + atomicAdd(ctx.build_next, 1);
+        __syncthreads();
+    }
+    // the last block to leave puts the counters back to zero for the next launch
+    if (threadIdx.x == 0) {
+        __threadfence();
+        if (atomicAdd(ctx.build_done, 1) == (int)gridDim.x - 1) {
+            *ctx.build_next = 0;
+            *ctx.build_done = 0;
         }
     }
 }
