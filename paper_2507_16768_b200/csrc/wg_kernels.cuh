@@ -241,7 +241,7 @@ struct BuildWork {
 
 // COMPACT: the cache keeps allows / denies entries; finished chunks are also stored as spans.
 template <bool COMPACT>
-__global__ void __launch_bounds__(BUILD_THREADS, COMPACT ? 5 : 6)
+__global__ void __launch_bounds__(BUILD_THREADS, COMPACT ? 5 : 8)
 build_masks_kernel(VocabDev v, CtxDev ctx, BuildWork work) {
     __shared__ uint8_t cls[256];
     __shared__ int cls_gid;
