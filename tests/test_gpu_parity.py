@@ -433,8 +433,9 @@ def test_host_buffer_step_and_step_plan_equal_the_plain_step(wg, torch):
     dv = wg.Vocab(vocab.offsets, vocab.data, vocab.eos_id)
     B, V = 6, vocab.size
     results = []
-    for mode in ("plain", "plan", "host", "graph"):
-        ctx = wg.Context(dv, 256, B)
+    for mode, cache_mode in (("plain", 0), ("plan", 0), ("host", 0), ("graph", 0), ("plain", 1),
+                             ("graph", 1), ("host", 1)):
+        ctx = wg.Context(dv, 256, B, cache_mode)
         gid = torch.full((B,), ctx.add_grammar(g), dtype=torch.int32, device="cuda")
         sid = torch.full((B,), g.start_state, dtype=torch.int32, device="cuda")
         mask = torch.zeros((B, dv.W), dtype=torch.int32, device="cuda")
