@@ -312,7 +312,8 @@ int32_t wg_cache_entry_read(wg_ctx *ctx, int32_t grammar_id, int32_t state, int3
 /* Uploads a compiled grammar's table and returns its id in this context.  A grammar whose
  * content_hash and tables equal one already added gets that grammar's id, so requests
  * instantiated with the same arguments share cache entries.  Synchronous (small copies).
- * Errors: WG_ERR_ARG, WG_ERR_CAPACITY (more than 65535 grammars), WG_ERR_CUDA. */
+ * Errors: WG_ERR_ARG, WG_ERR_CAPACITY (more than 65535 grammars, or a table of 2^32 cells or
+ * more), WG_ERR_CUDA. */
 int32_t wg_ctx_add_grammar(wg_ctx *ctx, const wg_grammar *grammar, int32_t *grammar_id);
 
 /* Builds and caches the mask of every state of grammar `grammar_id` (states 1..n_states-1).

@@ -567,6 +567,8 @@ int32_t wg_ctx_add_grammar(wg_ctx *c, const wg_grammar *g, int32_t *grammar_id) 
         }
     }
     if (c->slots.size() >= 65535) return WG_ERR_CAPACITY;
+    // the kernels index table cells with 32 bits
+    if ((uint64_t)g->n_states * (uint64_t)g->n_classes >= (1ull << 32)) return WG_ERR_CAPACITY;
     const bool wide = g->n_states > 65535;
     GrammarSlot slot{g->hash, g->table, g->forced_tok, g->forced_next, g->n_states, g->n_classes,
                      nullptr, nullptr, nullptr, nullptr, nullptr};
