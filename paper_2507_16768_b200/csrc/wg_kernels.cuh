@@ -111,10 +111,10 @@ __device__ __forceinline__ uint32_t walk_token_classes(const VocabDev &v, const 
     if (n == 0) return 0;
     const uint4 rec = __ldg(&rec_class[t]);
     const uint32_t w[4] = {rec.x, rec.y, rec.z, rec.w};
-#pragma unroll
     // (the index stays in 32 bits: a table has fewer than 2^32 cells, and the address then takes
     // one wide multiply-add instead of a 64-bit multiply, add and shift)
     const uint32_t Cu = (uint32_t)C;
+#pragma unroll
     for (int j = 0; j < WG_REC_BYTES; ++j) {
         if (j >= n || s == 0) break;
         s = tab[s * Cu + ((w[j >> 2] >> (8 * (j & 3))) & 0xFFu)];
