@@ -111,6 +111,7 @@ struct wg_ctx {
     // vocabulary-sharded steps fill cached masks only inside their token range; the range they
     // used is remembered so that no call reads cached words that were never built
     int32_t part_begin = 0, part_end = 0;  // both 0: every cached mask is complete
+    int build_blocks_per_sm = 0;           // resident blocks of the build kernel (0: not asked yet)
     int32_t *d_stage_gid = nullptr, *d_stage_sid = nullptr;  // prewarm staging
     std::vector<void *> owned;  // every other device allocation
     std::mutex mu;
@@ -728,8 +729,7 @@ int32_t launch_build(wg_ctx *c, const BuildWork &work, int max_entries, cudaStre
     auto kernel = c->dev.compact ? build_masks_kernel<true> : build_masks_kernel<false>;
     // One block per resident slot: the blocks stride over the items, so blocks that had to wait
     // for a slot would start their equal share late and stretch the launch.
-    static int resident[2] = {0, 0};
-    int &per_sm = resident[c->dev.compact ? 1 : 0];
+    int &per_sm = c->build_blocks_per_sm;
     if (per_sm == 0) {
         int n = 0;
         if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, BUILD_THREADS, 0) != cudaSuccess || n < 1)
