@@ -82,7 +82,6 @@ struct wg_vocab {
     VocabDev dev{};
     void *d_rec = nullptr, *d_len = nullptr, *d_offsets = nullptr, *d_bytes = nullptr;
     void *d_first_mask = nullptr, *d_fold_mask = nullptr, *d_valid_mask = nullptr;
-    std::vector<uint8_t> host_rec;  // the 16-byte records, kept for per-grammar class mapping
     int device = 0;
 };
 
@@ -219,7 +218,6 @@ int32_t wg_load_vocab(const uint32_t *offsets, const uint8_t *bytes, int32_t V, 
     v->dev.valid_mask = static_cast<const uint32_t *>(v->d_valid_mask);
     v->dev.offsets = static_cast<const uint32_t *>(v->d_offsets);
     v->dev.bytes = static_cast<const uint8_t *>(v->d_bytes);
-    v->host_rec = std::move(rec);
     v->dev.V = V;
     v->dev.W = (V + 31) / 32;
     v->dev.eos_id = eos_id;
@@ -603,22 +601,17 @@ int32_t wg_ctx_add_grammar(wg_ctx *c, const wg_grammar *g, int32_t *grammar_id) 
     // per state: the bytes that keep it alive, and (folded mod 64) the bytes that leave it
     {
         const int32_t S = g->n_states, C = g->n_classes;
-        std::vector<uint32_t> first_ok((size_t)S * 8, 0u);
-        std::vector<unsigned long long> leaves(S, 0ull);
-        for (int32_t st = 1; st < S; ++st) {
-            const int32_t *row = &g->table[(size_t)st * C];
-            for (int b = 0; b < 256; ++b) {
-                const int32_t to = row[g->byte_class[b]];
-                if (to != 0) first_ok[(size_t)st * 8 + (b >> 5)] |= 1u << (b & 31);
-                if (to != st) leaves[st] |= 1ull << (b & 63);
-            }
-        }
-        WG_CUDA(cudaMalloc(&slot.d_first_ok, first_ok.size() * sizeof(uint32_t)));
-        WG_CUDA(cudaMemcpy(slot.d_first_ok, first_ok.data(), first_ok.size() * sizeof(uint32_t),
-                           cudaMemcpyHostToDevice));
-        WG_CUDA(cudaMalloc(&slot.d_leaves, leaves.size() * sizeof(unsigned long long)));
-        WG_CUDA(cudaMemcpy(slot.d_leaves, leaves.data(), leaves.size() * sizeof(unsigned long long),
-                           cudaMemcpyHostToDevice));
+        WG_CUDA(cudaMalloc(&slot.d_first_ok, (size_t)S * 8 * sizeof(uint32_t)));
+        WG_CUDA(cudaMalloc(&slot.d_leaves, (size_t)S * sizeof(unsigned long long)));
+        if (wide)
+            grammar_state_info_kernel<uint32_t><<<(unsigned)S, 256, 0, cudaStreamLegacy>>>(
+                static_cast<const uint32_t *>(slot.d_table), static_cast<const uint8_t *>(slot.d_cls), S, C,
+                static_cast<uint32_t *>(slot.d_first_ok), static_cast<unsigned long long *>(slot.d_leaves));
+        else
+            grammar_state_info_kernel<uint16_t><<<(unsigned)S, 256, 0, cudaStreamLegacy>>>(
+                static_cast<const uint16_t *>(slot.d_table), static_cast<const uint8_t *>(slot.d_cls), S, C,
+                static_cast<uint32_t *>(slot.d_first_ok), static_cast<unsigned long long *>(slot.d_leaves));
+        WG_LAUNCHED();
     }
     // the vocabulary's records with bytes replaced by this grammar's classes (shared between
     // grammars whose class maps are equal)
@@ -626,20 +619,23 @@ int32_t wg_ctx_add_grammar(wg_ctx *c, const wg_grammar *g, int32_t *grammar_id) 
     for (const ClassMappedRecords &r : c->class_records)
         if (memcmp(r.byte_class, g->byte_class, 256) == 0) d_rec_class = r.d_rec;
     if (!d_rec_class) {
-        const std::vector<uint8_t> &src = c->vocab->host_rec;
-        std::vector<uint8_t> mapped(src.size());
-        for (size_t i = 0; i < src.size(); ++i) mapped[i] = g->byte_class[src[i]];
+        const int V = c->vocab->dev.V;
         ClassMappedRecords r;
         memcpy(r.byte_class, g->byte_class, 256);
         r.d_rec = nullptr;
-        WG_CUDA(cudaMalloc(&r.d_rec, mapped.size() ? mapped.size() : 1));
-        if (cudaMemcpy(r.d_rec, mapped.data(), mapped.size(), cudaMemcpyHostToDevice) != cudaSuccess) {
+        WG_CUDA(cudaMalloc(&r.d_rec, (size_t)V * WG_REC_BYTES));
+        map_records_kernel<<<(unsigned)((V + 255) / 256), 256, 0, cudaStreamLegacy>>>(
+            c->vocab->dev.rec, static_cast<const uint8_t *>(slot.d_cls), static_cast<uint4 *>(r.d_rec), V);
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+        if (cudaGetLastError() != cudaSuccess) {
             cudaFree(r.d_rec);
             return WG_ERR_CUDA;
         }
         c->class_records.push_back(r);
         d_rec_class = r.d_rec;
     }
+    // both kernels have finished before the grammar is used, on whatever stream that will be
+    WG_CUDA(cudaStreamSynchronize(cudaStreamLegacy));
     GrammarDev gd{slot.d_table, static_cast<const uint8_t *>(slot.d_cls),
                   static_cast<const uint32_t *>(slot.d_first_ok),
                   static_cast<const unsigned long long *>(slot.d_leaves),

@@ -383,6 +383,55 @@ build_masks_kernel(VocabDev v, CtxDev ctx, BuildWork work) {
 }
 
 // ---------------------------------------------------------------------------------------
+// Set-up kernels of wg_ctx_add_grammar (a grammar that is instantiated per request is added on
+// the request's critical path, so its derived arrays are made here rather than on the host).
+// ---------------------------------------------------------------------------------------
+
+// Per state: first_ok (256 bits: bytes that do not lead to DEAD) and leaves (64 bits: folds
+// b & 63 of the bytes that lead anywhere but back to the state).  One block of 256 threads per
+// state, thread b looks at byte b; state 0 (DEAD) gets zeros.
+template <typename T>
+__global__ void __launch_bounds__(256)
+grammar_state_info_kernel(const T *__restrict__ table, const uint8_t *__restrict__ byte_class,
+                          int n_states, int n_classes, uint32_t *first_ok,
+                          unsigned long long *leaves) {
+    __shared__ uint32_t out_bits[8];
+    const int st = blockIdx.x;
+    if (st >= n_states) return;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t to = st == 0 ? 0u : (uint32_t)table[(size_t)st * n_classes + byte_class[threadIdx.x]];
+    const uint32_t ok = __ballot_sync(0xFFFFFFFFu, to != 0u);
+    const uint32_t out = __ballot_sync(0xFFFFFFFFu, st != 0 && to != (uint32_t)st);
+    if (lane == 0) {
+        first_ok[(size_t)st * 8 + warp] = ok;
+        out_bits[warp] = out;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {  // byte b = 32 * warp + lane folds to 32 * (warp & 1) + lane
+        const uint32_t lo = out_bits[0] | out_bits[2] | out_bits[4] | out_bits[6];
+        const uint32_t hi = out_bits[1] | out_bits[3] | out_bits[5] | out_bits[7];
+        leaves[st] = ((unsigned long long)hi << 32) | lo;
+    }
+}
+
+// The vocabulary's 16-byte records with every byte replaced by its class.
+__global__ void map_records_kernel(const uint4 *__restrict__ rec, const uint8_t *__restrict__ byte_class,
+                                   uint4 *out, int V) {
+    __shared__ uint8_t cls[256];
+    for (int i = threadIdx.x; i < 256; i += blockDim.x) cls[i] = byte_class[i];
+    __syncthreads();
+    const int t = blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= V) return;
+    const uint4 r = rec[t];
+    uint32_t w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+        w[i] = (uint32_t)cls[w[i] & 0xFFu] | ((uint32_t)cls[(w[i] >> 8) & 0xFFu] << 8) |
+               ((uint32_t)cls[(w[i] >> 16) & 0xFFu] << 16) | ((uint32_t)cls[w[i] >> 24] << 24);
+    out[t] = make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+// ---------------------------------------------------------------------------------------
 // K2: mask cache.  Open addressing with linear probing over 64-bit keys.
 // ---------------------------------------------------------------------------------------
 __device__ __forceinline__ unsigned long long cache_key(int gid, int sid) {
