@@ -34,11 +34,12 @@ def sample_rows(B, step, n):
     return sorted(rows)
 
 
-def test_json_warm_batch_1024_prewarmed(wg, torch):
+@pytest.mark.parametrize("cache_mode", [0, 1])        # dense rows, allows / denies entries
+def test_json_warm_batch_1024_prewarmed(wg, torch, cache_mode):
     w = BY_NAME["json_warm"]
     vocab = make_vocab(w.V, w.vocab_seed)
     sim = Sim(wg, torch, vocab, [w.grammar(0)], [0] * w.batch, w.dtype,
-              cache_capacity=sim_capacity(wg, w), steer=0.0, seed=4)
+              cache_capacity=sim_capacity(wg, w), steer=0.0, seed=4, cache_mode=cache_mode)
     sim.ctx.cache_prewarm(sim.gids[0])
     built = sim.ctx.stats()["masks_built"]
     assert built == sim.grams[0].n_states - 1
@@ -67,7 +68,8 @@ def test_cold_templates_batch_256_no_cache(wg, torch):
     assert len({g for g, _ in sim.visited}) == w.n_grammars
 
 
-def test_dynamic_snippets_batch_128_pairs_share_an_instantiation(wg, torch):
+@pytest.mark.parametrize("cache_mode", [0, 1])
+def test_dynamic_snippets_batch_128_pairs_share_an_instantiation(wg, torch, cache_mode):
     w = BY_NAME["dynamic_snippets"]
     vocab = make_vocab(w.V, w.vocab_seed)
     n_inst = w.batch // 2
@@ -75,7 +77,7 @@ def test_dynamic_snippets_batch_128_pairs_share_an_instantiation(wg, torch):
     rows = [w.grammar_of_row(r) for r in range(w.batch)]
     delays = [w.row_delay(r) for r in range(w.batch)]
     sim = Sim(wg, torch, vocab, ops, rows, w.dtype, cache_capacity=4096, seed=5, steer=6.0,
-              delays=delays)
+              delays=delays, cache_mode=cache_mode)
     assert max(g.n_states for g in sim.grams) > 15000
     for step in range(6):
         sim.step(check_rows=sample_rows(w.batch, step, 8))
