@@ -1,9 +1,9 @@
 """Parity at the full sizes of the workloads, in the launch configuration the benchmark times.
 
-The checker cannot redo 1024 rows x 128256 tokens per step in reasonable time, so every step
-compares a sample of rows in full (mask words, masked logits as raw bits, chosen token) and
-ALL rows through what is cheap: the token must be allowed by the checker in the row's
-cursor, and the device state must equal the host table walk of that token.
+The first and the last step compare EVERY row in full (mask words, masked logits as raw bits,
+chosen token); the steps between compare a sample of rows in full and all rows through what
+is cheap: the token must be allowed by the checker in the row's cursor, and the device state
+must equal the host table walk of that token.
 """
 import numpy as np
 import pytest
@@ -45,7 +45,7 @@ def test_json_warm_batch_1024_prewarmed(wg, torch, cache_mode):
     assert built == sim.grams[0].n_states - 1
     sim.ctx.reset_stats()
     for step in range(5):
-        sim.step(check_rows=sample_rows(w.batch, step, 10))
+        sim.step(check_rows=None if step in (0, 4) else sample_rows(w.batch, step, 10))
     st = sim.ctx.stats()
     assert st["masks_built"] == 0, "a prewarmed cache must serve every row"
     assert st["cache_hits"] == 5 * w.batch and st["cache_misses"] == 0
@@ -63,7 +63,7 @@ def test_cold_templates_batch_256_no_cache(wg, torch):
     rows = [w.grammar_of_row(r) for r in range(w.batch)]
     sim = Sim(wg, torch, vocab, ops, rows, w.dtype, cache_capacity=0, use_cache=False, seed=3)
     for step in range(4):
-        sim.step(check_rows=sample_rows(w.batch, step, 14))
+        sim.step(check_rows=None if step in (0, 3) else sample_rows(w.batch, step, 14))
     assert sim.ctx.stats()["masks_built"] == 4 * w.batch
     assert len({g for g, _ in sim.visited}) == w.n_grammars
 
@@ -80,7 +80,7 @@ def test_dynamic_snippets_batch_128_pairs_share_an_instantiation(wg, torch, cach
               delays=delays, cache_mode=cache_mode)
     assert max(g.n_states for g in sim.grams) > 15000
     for step in range(6):
-        sim.step(check_rows=sample_rows(w.batch, step, 8))
+        sim.step(check_rows=None if step in (0, 5) else sample_rows(w.batch, step, 8))
     st = sim.ctx.stats()
     # from the second step on a follower finds what its leader built one step before
     assert st["cache_hits"] >= 5 * n_inst - n_inst
