@@ -170,3 +170,66 @@ def test_instantiation_is_cheaper_than_lowering_when_the_static_part_dominates(w
     g = T.instantiate([wg.Grammar(f) for f in flat_args])
     assert g.n_states == wg.Grammar(whole).n_states > 20000
     assert t_inst < t_full, (t_inst, t_full)
+
+
+def _random_op(rng, depth, hole_args=0):
+    """A random operator tree over a small alphabet; with hole_args > 0 some leaves are holes."""
+    alphabet = b"abcd,;"
+
+    def pick_sets(k):
+        syms = list(alphabet)
+        rng.shuffle(syms)
+        cases = [SymSet([syms.pop()]) for _ in range(k)]
+        stay = SymSet([s for s in syms if rng.random() < 0.5])
+        return cases, stay
+
+    def node(d):
+        if hole_args and rng.random() < 0.25:
+            return Hole(int(rng.integers(0, hole_args)))
+        kind = rng.integers(0, 6) if d > 0 else rng.integers(0, 2)
+        if kind == 0:
+            return Write(bytes(rng.choice(list(alphabet), size=int(rng.integers(1, 4))).tolist()))
+        if kind == 1:
+            (w,), stay = pick_sets(1)
+            return Wait(allow=stay | w, wait=w, body=node(d - 1) if d > 0 and rng.random() < 0.3 else None)
+        if kind == 2:
+            k = int(rng.integers(2, 4))
+            cases, stay = pick_sets(k)
+            union = stay
+            for c in cases:
+                union = union | c
+            return Switch(allow=union, cases=cases,
+                          bodies=[node(d - 1) if rng.random() < 0.7 else None for _ in range(k)])
+        if kind == 3:
+            (t, f), stay = pick_sets(2)
+            return DoWhile(node(d - 1) if rng.random() < 0.85 else None,
+                           Cond(allow=stay | t | f, true_waits=t, false_waits=f))
+        if kind == 4:
+            return WaitUntil(SymSet(b"ab,"), bytes(rng.choice(list(b"ab"), size=int(rng.integers(1, 4))).tolist()))
+        return Sequence([node(d - 1) for _ in range(int(rng.integers(0, 4)))])
+
+    return Sequence(node(depth), node(depth - 1))
+
+
+def test_random_templates_and_arguments(wg):
+    rng = np.random.default_rng(77)
+    symbols = list(b"abcd,;x") + [EOS]
+    checked = holes = 0
+    for _ in range(80):
+        n_args = int(rng.integers(1, 4))
+        template = _random_op(rng, 3, hole_args=n_args)
+        args = [_random_op(rng, 2) for _ in range(n_args)]
+        whole = flatten(substitute(template, args))
+        tree = oracle.Tree(whole)
+        T = wg.Template(flatten(template))
+        assert T.n_args <= n_args                   # 1 + the largest argument index that occurs
+        g = T.instantiate([wg.Grammar(flatten(a)) for a in args[:T.n_args]])
+        cursor_of = co_reachable(tree, g, symbols)
+        # every reachable cursor has one state; the spliced table has no fewer states than a
+        # fresh lowering reaches (copies of an argument that no path enters may be left over)
+        full = wg.Grammar(whole)
+        assert len(cursor_of) == full.n_states - 1 <= g.n_states - 1
+        assert g.minimized().n_states == full.minimized().n_states
+        checked += 1
+        holes += T.n_holes
+    assert checked == 80 and holes > 60
