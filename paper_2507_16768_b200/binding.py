@@ -173,7 +173,7 @@ class Vocab:
         self.handle = h
 
     def close(self):
-        if getattr(self, "handle", None):
+        if getattr(self, "handle", None) and _lib is not None:
             _lib.wg_vocab_free(self.handle)
             self.handle = None
 
@@ -289,7 +289,7 @@ class Grammar:
         return state
 
     def close(self):
-        if getattr(self, "handle", None):
+        if getattr(self, "handle", None) and _lib is not None:
             _lib.wg_grammar_free(self.handle)
             self.handle = None
 
@@ -325,7 +325,7 @@ class Template:
         return Grammar(_handle=h)
 
     def close(self):
-        if getattr(self, "handle", None):
+        if getattr(self, "handle", None) and _lib is not None:
             _lib.wg_template_free(self.handle)
             self.handle = None
 
@@ -363,7 +363,7 @@ class Context:
         return kind.value, ids[:n.value].copy(), int(nbytes.value)
 
     def close(self):
-        if getattr(self, "handle", None):
+        if getattr(self, "handle", None) and _lib is not None:
             _lib.wg_ctx_free(self.handle)
             self.handle = None
 
@@ -590,7 +590,7 @@ class StepGraph:
             raise WgError(rc, "wg_step_graph_launch")
 
     def close(self):
-        if getattr(self, "handle", None):
+        if getattr(self, "handle", None) and _lib is not None:
             _lib.wg_step_graph_free(self.handle)
             self.handle = None
 
