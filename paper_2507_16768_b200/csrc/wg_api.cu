@@ -90,7 +90,7 @@ struct GrammarSlot {
     std::vector<int32_t> table;  // host copy, for exact comparison on hash equality
     std::vector<int32_t> forced_tok, forced_next;
     int32_t n_states, n_classes;
-    void *d_table, *d_cls, *d_first_ok, *d_leaves, *d_forced;
+    void *d_table, *d_cls, *d_first_ok, *d_leaves, *d_forced, *d_leave1, *d_leave_fold;
 };
 
 struct ClassMappedRecords {
@@ -111,6 +111,12 @@ struct wg_ctx {
     // used is remembered so that no call reads cached words that were never built
     int32_t part_begin = 0, part_end = 0;  // both 0: every cached mask is complete
     int build_blocks_per_sm = 0;           // resident blocks of the build kernel (0: not asked yet)
+    // "what follows byte b" masks (see after_masks_kernel): made on demand, at most AFTER_SLOTS bytes
+    uint32_t *d_after_masks = nullptr;
+    int8_t *d_after_slot = nullptr;
+    uint32_t *d_leave_bits = nullptr;      // 8 words of scratch for wg_ctx_add_grammar
+    int8_t after_slot[256];
+    int n_after = 0;
     int32_t *d_stage_gid = nullptr, *d_stage_sid = nullptr;  // prewarm staging
     std::vector<void *> owned;  // every other device allocation
     std::mutex mu;
@@ -462,6 +468,7 @@ int32_t wg_ctx_create_ex(const wg_vocab *vocab, int32_t cache_capacity, int32_t 
     if (!c) return WG_ERR_ARG;
     c->vocab = vocab;
     c->max_batch = max_batch;
+    memset(c->after_slot, 0xFF, sizeof(c->after_slot));
     CtxDev &d = c->dev;
     d.capacity = cache_capacity;
     d.pool_stride = ((int64_t)vocab->dev.W + 31) / 32 * 32;  // rows start on 128-byte lines
@@ -541,6 +548,9 @@ void wg_ctx_free(wg_ctx *c) {
     if (!c) return;
     cudaDeviceSynchronize();
     for (void *p : c->owned) cudaFree(p);
+    cudaFree(c->d_after_masks);
+    cudaFree(c->d_after_slot);
+    cudaFree(c->d_leave_bits);
     for (ClassMappedRecords &r : c->class_records) cudaFree(r.d_rec);
     for (cudaEvent_t e : c->events) cudaEventDestroy(e);
     for (GrammarSlot &s : c->slots) {
@@ -549,6 +559,8 @@ void wg_ctx_free(wg_ctx *c) {
         cudaFree(s.d_first_ok);
         cudaFree(s.d_leaves);
         cudaFree(s.d_forced);
+        cudaFree(s.d_leave1);
+        cudaFree(s.d_leave_fold);
     }
     delete c;
 }
@@ -570,13 +582,13 @@ int32_t wg_ctx_add_grammar(wg_ctx *c, const wg_grammar *g, int32_t *grammar_id) 
     if ((uint64_t)g->n_states * (uint64_t)g->n_classes >= (1ull << 32)) return WG_ERR_CAPACITY;
     const bool wide = g->n_states > 65535;
     GrammarSlot slot{g->hash, g->table, g->forced_tok, g->forced_next, g->n_states, g->n_classes,
-                     nullptr, nullptr, nullptr, nullptr, nullptr};
+                     nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
     struct Guard {  // frees the uploads again if any later step fails
         GrammarSlot *s;
         ~Guard() {
             if (!s) return;
             cudaFree(s->d_table); cudaFree(s->d_cls); cudaFree(s->d_first_ok);
-            cudaFree(s->d_leaves); cudaFree(s->d_forced);
+            cudaFree(s->d_leaves); cudaFree(s->d_forced); cudaFree(s->d_leave1); cudaFree(s->d_leave_fold);
         }
     } guard{&slot};
     if (!g->forced_tok.empty()) {
@@ -603,15 +615,56 @@ int32_t wg_ctx_add_grammar(wg_ctx *c, const wg_grammar *g, int32_t *grammar_id) 
         const int32_t S = g->n_states, C = g->n_classes;
         WG_CUDA(cudaMalloc(&slot.d_first_ok, (size_t)S * 8 * sizeof(uint32_t)));
         WG_CUDA(cudaMalloc(&slot.d_leaves, (size_t)S * sizeof(unsigned long long)));
-        if (wide)
+        WG_CUDA(cudaMalloc(&slot.d_leave1, (size_t)S * sizeof(int16_t)));
+        WG_CUDA(cudaMalloc(&slot.d_leave_fold, (size_t)S * sizeof(unsigned long long)));
+        if (!c->d_leave_bits) WG_CUDA(cudaMalloc((void **)&c->d_leave_bits, 8 * sizeof(uint32_t)));
+        WG_CUDA(cudaMemsetAsync(c->d_leave_bits, 0, 8 * sizeof(uint32_t), cudaStreamLegacy));
+        const uint8_t *d_cls = static_cast<const uint8_t *>(slot.d_cls);
+        uint32_t *d_ok = static_cast<uint32_t *>(slot.d_first_ok);
+        int16_t *d_l1 = static_cast<int16_t *>(slot.d_leave1);
+        unsigned long long *d_lf = static_cast<unsigned long long *>(slot.d_leave_fold);
+        if (wide) {
+            const uint32_t *tab = static_cast<const uint32_t *>(slot.d_table);
             grammar_state_info_kernel<uint32_t><<<(unsigned)S, 256, 0, cudaStreamLegacy>>>(
-                static_cast<const uint32_t *>(slot.d_table), static_cast<const uint8_t *>(slot.d_cls), S, C,
-                static_cast<uint32_t *>(slot.d_first_ok), static_cast<unsigned long long *>(slot.d_leaves));
-        else
+                tab, d_cls, S, C, d_ok, static_cast<unsigned long long *>(slot.d_leaves), d_l1);
+            WG_LAUNCHED();
+            leave_info_kernel<uint32_t><<<(unsigned)((S + 255) / 256), 256, 0, cudaStreamLegacy>>>(
+                tab, d_cls, d_ok, d_l1, S, C, d_lf, c->d_leave_bits);
+        } else {
+            const uint16_t *tab = static_cast<const uint16_t *>(slot.d_table);
             grammar_state_info_kernel<uint16_t><<<(unsigned)S, 256, 0, cudaStreamLegacy>>>(
-                static_cast<const uint16_t *>(slot.d_table), static_cast<const uint8_t *>(slot.d_cls), S, C,
-                static_cast<uint32_t *>(slot.d_first_ok), static_cast<unsigned long long *>(slot.d_leaves));
+                tab, d_cls, S, C, d_ok, static_cast<unsigned long long *>(slot.d_leaves), d_l1);
+            WG_LAUNCHED();
+            leave_info_kernel<uint16_t><<<(unsigned)((S + 255) / 256), 256, 0, cudaStreamLegacy>>>(
+                tab, d_cls, d_ok, d_l1, S, C, d_lf, c->d_leave_bits);
+        }
         WG_LAUNCHED();
+        // the bytes that close a free-text slot of this grammar get their vocabulary masks now
+        uint32_t leave_bits[8];
+        WG_CUDA(cudaMemcpy(leave_bits, c->d_leave_bits, sizeof(leave_bits), cudaMemcpyDeviceToHost));
+        const VocabDev &v = c->vocab->dev;
+        const size_t slot_words = (size_t)AFTER_ROWS * (size_t)v.W;
+        bool table_changed = false;
+        for (int b = 0; b < 256; ++b) {
+            if (!((leave_bits[b >> 5] >> (b & 31)) & 1u) || c->after_slot[b] >= 0) continue;
+            if (c->n_after >= AFTER_SLOTS) break;  // the rest goes without (results are the same)
+            if (!c->d_after_masks) {
+                WG_CUDA(cudaMalloc((void **)&c->d_after_masks, AFTER_SLOTS * slot_words * sizeof(uint32_t)));
+                WG_CUDA(cudaMalloc((void **)&c->d_after_slot, 256));
+            }
+            uint32_t *rows = c->d_after_masks + (size_t)c->n_after * slot_words;
+            WG_CUDA(cudaMemsetAsync(rows, 0, slot_words * sizeof(uint32_t), cudaStreamLegacy));
+            after_masks_kernel<<<(unsigned)((v.W * 32 + 255) / 256), 256, 0, cudaStreamLegacy>>>(v, b, rows);
+            WG_LAUNCHED();
+            c->after_slot[b] = (int8_t)c->n_after++;
+            table_changed = true;
+        }
+        if (table_changed) {
+            WG_CUDA(cudaMemcpyAsync(c->d_after_slot, c->after_slot, 256, cudaMemcpyHostToDevice,
+                                    cudaStreamLegacy));
+            c->dev.after_masks = c->d_after_masks;
+            c->dev.after_slot = c->d_after_slot;
+        }
     }
     // the vocabulary's records with bytes replaced by this grammar's classes (shared between
     // grammars whose class maps are equal)
@@ -640,7 +693,9 @@ int32_t wg_ctx_add_grammar(wg_ctx *c, const wg_grammar *g, int32_t *grammar_id) 
                   static_cast<const uint32_t *>(slot.d_first_ok),
                   static_cast<const unsigned long long *>(slot.d_leaves),
                   static_cast<const int2 *>(slot.d_forced),
-                  static_cast<const uint4 *>(d_rec_class), g->n_states,
+                  static_cast<const uint4 *>(d_rec_class),
+                  static_cast<const int16_t *>(slot.d_leave1),
+                  static_cast<const unsigned long long *>(slot.d_leave_fold), g->n_states,
                   g->n_classes, g->start, g->done, g->eos_class, wide ? 1 : 0};
     const int32_t id = (int32_t)c->slots.size();
     if (id >= c->grammar_cap) {  // grow the registry; queued kernels still read the old one

@@ -23,6 +23,12 @@ struct GrammarDev {
     const uint4 *rec_class;     // [V] the vocabulary's 16-byte records with every byte replaced by
                                 // its class under THIS grammar's byte_class (shared by grammars
                                 // with equal class maps): saves the class look-up in the walk
+    const int16_t *leave1;      // [n_states] the byte, if exactly ONE byte leads from the state to a
+                                // live state other than itself (a free-text slot's closing byte),
+                                // else -1
+    const unsigned long long *leave_fold;  // [n_states] for such a state, if it accepts most bytes
+                                // and few survive after the leaving byte: the folded set of
+                                // bytes that survive in the state after that byte; else 0
     int32_t n_states, n_classes, start, done, eos_class, wide;
 };
 
@@ -62,6 +68,10 @@ struct CtxDev {
                                        // both zero between launches
     unsigned long long *argkey;  // [max_batch] packed (value key, ~id) maxima
     unsigned long long *stats;   // [ST_COUNT]
+    // "what follows byte b" masks of the vocabulary, made for the bytes that close a free-text
+    // slot of some added grammar (see after_masks_kernel); slot k holds AFTER_ROWS rows of W words
+    const uint32_t *after_masks; // [AFTER_SLOTS][AFTER_ROWS][W], or NULL while no byte needed them
+    const int8_t *after_slot;    // [256] slot of byte b, or -1
     // compact cache (allows / denies storage instead of dense pool rows); pool is NULL then
     int32_t compact;
     uint2 *ent_hdr;                  // [capacity][hdr_stride] per cache row and span of 32 mask
@@ -80,6 +90,11 @@ struct CtxDev {
 };
 
 
+constexpr int BUILD_AFTER_MAX_FOLDS = 8;  // larger sets after the leaving byte: no filtering
+constexpr int AFTER_SLOTS = 8;   // bytes that can have "what follows" masks
+constexpr int AFTER_ROWS = 66;   // row 0: token contains b; row 1: worth a walk whatever follows
+                                 // (b is the last byte, or the record ends before the answer is
+                                 // known); rows 2 + c: the byte after the first b folds to c
 constexpr uint32_t NEG_INF_F32 = 0xFF800000u;
 constexpr uint32_t NEG_INF_BF16X2 = 0xFF80FF80u;
 
@@ -297,6 +312,18 @@ build_masks_kernel(VocabDev v, CtxDev ctx, BuildWork work) {
         if (s0) eos_next = g.wide ? static_cast<const uint32_t *>(g.table)[(size_t)s0 * g.n_classes + g.eos_class]
                                   : static_cast<const uint16_t *>(g.table)[(size_t)s0 * g.n_classes + g.eos_class];
         const int forced_tok = (s0 && g.forced) ? g.forced[s0].x : -1;  // token-level Write state
+        // A free-text slot has ONE byte that leads on (its closing byte); a token that holds it is
+        // dead unless that byte ends the token or the byte after its first occurrence survives
+        // in the next state.  The vocabulary masks for that byte turn this into word-wise work.
+        int after_k = -1;
+        unsigned long long after_fold = 0ull;
+        if (s0 && ctx.after_masks) {
+            const int lv = g.leave1[s0];
+            if (lv >= 0) {
+                after_fold = g.leave_fold[s0];  // 0: not a state the masks were made for
+                if (after_fold != 0ull) after_k = ctx.after_slot[lv];
+            }
+        }
         __syncthreads();
         if (threadIdx.x == 0 && known) cls_gid = gid;  // read again only after the next barrier
         {
@@ -322,6 +349,23 @@ build_masks_kernel(VocabDev v, CtxDev ctx, BuildWork work) {
                 for (int i = 0; i < nq; ++i) q |= __ldg(&v.fold_mask[(size_t)fold_list[i] * v.W + w]);
                 alive = p & ~q;
                 queue = p & q;
+                if (after_k >= 0 && queue != 0) {
+                    const uint32_t *rows = ctx.after_masks + (size_t)after_k * AFTER_ROWS * v.W;
+                    const uint32_t has = __ldg(&rows[w]);
+                    if (n_ok == 256) {
+                        // no byte kills the state and only the closing byte leaves it: a token
+                        // without that byte is allowed without a walk (the folded sets also
+                        // catch the other bytes of the closing byte's fold, e.g. 'b' for '"')
+                        alive |= queue & ~has;
+                        queue &= has;
+                    }
+                    if (queue & has) {
+                        uint32_t worth = __ldg(&rows[(size_t)v.W + w]);
+                        for (unsigned long long f = after_fold; f; f &= f - 1)
+                            worth |= __ldg(&rows[(size_t)(2 + __ffsll((long long)f) - 1) * v.W + w]);
+                        queue &= ~has | worth;
+                    }
+                }
                 if ((v.eos_id >> 5) == w && eos_next != 0) alive |= 1u << (v.eos_id & 31);
             }
             if (wl < n_words) words[wl] = alive;
@@ -394,7 +438,7 @@ template <typename T>
 __global__ void __launch_bounds__(256)
 grammar_state_info_kernel(const T *__restrict__ table, const uint8_t *__restrict__ byte_class,
                           int n_states, int n_classes, uint32_t *first_ok,
-                          unsigned long long *leaves) {
+                          unsigned long long *leaves, int16_t *leave1) {
     __shared__ uint32_t out_bits[8];
     const int st = blockIdx.x;
     if (st >= n_states) return;
@@ -412,6 +456,83 @@ grammar_state_info_kernel(const T *__restrict__ table, const uint8_t *__restrict
         const uint32_t hi = out_bits[1] | out_bits[3] | out_bits[5] | out_bits[7];
         leaves[st] = ((unsigned long long)hi << 32) | lo;
     }
+    // bytes that lead to a LIVE state other than the state itself: exactly one?
+    const uint32_t away = __ballot_sync(0xFFFFFFFFu, st != 0 && to != 0u && to != (uint32_t)st);
+    __syncthreads();
+    if (lane == 0) out_bits[warp] = away;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int n = 0, byte = -1;
+        for (int w = 0; w < 8; ++w) {
+            n += __popc(out_bits[w]);
+            if (out_bits[w]) byte = w * 32 + __ffs(out_bits[w]) - 1;
+        }
+        leave1[st] = (int16_t)(n == 1 ? byte : -1);
+    }
+}
+
+// Second pass, one thread per state: for a state with a single leaving byte, the folded set of
+// bytes that survive right after it; and one bit per byte value that is such a leaving byte with
+// a small set after it (bits: 8 words, zeroed before) -- those bytes get "what follows" masks.
+template <typename T>
+__global__ void leave_info_kernel(const T *__restrict__ table, const uint8_t *__restrict__ byte_class,
+                                  const uint32_t *__restrict__ first_ok, const int16_t *leave1,
+                                  int n_states, int n_classes, unsigned long long *leave_fold,
+                                  uint32_t *bits) {
+    const int s = blockIdx.x * blockDim.x + threadIdx.x;
+    if (s >= n_states) return;
+    const int b = leave1[s];
+    unsigned long long fold = 0ull;
+    if (b >= 0) {
+        const uint32_t s1 = (uint32_t)table[(size_t)s * n_classes + byte_class[b]];
+        const uint32_t *ok1 = first_ok + (size_t)s1 * 8;
+        fold = (unsigned long long)(ok1[0] | ok1[2] | ok1[4] | ok1[6]) |
+               ((unsigned long long)(ok1[1] | ok1[3] | ok1[5] | ok1[7]) << 32);
+        // masks are only worth making for states that accept most bytes (free-text slots): a
+        // state inside a literal queues few tokens anyway
+        int n_ok = 0;
+        for (int i = 0; i < 8; ++i) n_ok += __popc(first_ok[(size_t)s * 8 + i]);
+        if (n_ok > 128 && __popcll(fold) <= BUILD_AFTER_MAX_FOLDS) atomicOr(&bits[b >> 5], 1u << (b & 31));
+        else fold = 0ull;
+    }
+    leave_fold[s] = fold;
+}
+
+// The "what follows byte b" masks of one byte (AFTER_ROWS rows of W words, zeroed before).
+// One thread per token, a warp per mask word.  Only the first 16 bytes of a token are looked at;
+// where they do not settle the question the token is marked as worth a walk.
+__global__ void after_masks_kernel(VocabDev v, int b, uint32_t *rows) {
+    const int t = blockIdx.x * blockDim.x + threadIdx.x;  // grid covers W * 32 tokens
+    const int w = t >> 5;
+    if (w >= v.W) return;
+    int fold = -1;            // fold of the byte after the first b, if the record shows it
+    bool has = false, always = false;
+    if (t < v.V) {
+        const int n = v.len[t];
+        const uint4 r = v.rec[t];
+        const uint32_t word[4] = {r.x, r.y, r.z, r.w};
+        const int seen = n < WG_REC_BYTES ? n : WG_REC_BYTES;
+        int pos = -1;
+        for (int j = seen - 1; j >= 0; --j)
+            if (((word[j >> 2] >> (8 * (j & 3))) & 0xFFu) == (uint32_t)b) pos = j;
+        if (pos >= 0) {
+            has = true;
+            if (pos + 1 < seen) fold = (int)((word[(pos + 1) >> 2] >> (8 * ((pos + 1) & 3))) & 63u);
+            else always = true;  // b ends the token, or what follows lies beyond the record
+        } else if (n > WG_REC_BYTES) {
+            has = true;          // b may occur further on
+            always = true;
+        }
+    }
+    const uint32_t m_has = __ballot_sync(0xFFFFFFFFu, has);
+    const uint32_t m_always = __ballot_sync(0xFFFFFFFFu, always);
+    const uint32_t peers = __match_any_sync(0xFFFFFFFFu, fold);
+    const int lane = threadIdx.x & 31;
+    if (lane == 0) {
+        rows[w] = m_has;
+        rows[(size_t)v.W + w] = m_always;
+    }
+    if (fold >= 0 && lane == __ffs(peers) - 1) rows[(size_t)(2 + fold) * v.W + w] = peers;
 }
 
 // The vocabulary's 16-byte records with every byte replaced by its class.
