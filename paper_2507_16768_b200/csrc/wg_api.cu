@@ -777,6 +777,7 @@ int32_t launch_build(wg_ctx *c, const BuildWork &work, int max_entries, cudaStre
     if (w.t_last == 0) { w.t_first = 0; w.t_last = v.W * 32; }  // the whole vocabulary
     const long long n_chunks = ((long long)(w.t_last - w.t_first) + w.chunk - 1) / w.chunk;
     long long items = (long long)max_entries * n_chunks;
+    if (items >= (1LL << 31)) return WG_ERR_CAPACITY;  // the kernel numbers its items with 32 bits
     auto kernel = c->dev.compact ? build_masks_kernel<true> : build_masks_kernel<false>;
     // One block per resident slot: the blocks stride over the items, so blocks that had to wait
     // for a slot would start their equal share late and stretch the launch.

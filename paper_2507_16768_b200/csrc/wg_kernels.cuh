@@ -275,14 +275,16 @@ build_masks_kernel(VocabDev v, CtxDev ctx, BuildWork work) {
     const int lane = threadIdx.x & 31;
     const int n_entries = work.count_ptr ? *work.count_ptr : work.count;
     const int n_chunks = (work.t_last - work.t_first + work.chunk - 1) / work.chunk;
-    const long long n_items = (long long)n_entries * n_chunks;
+    // (item numbers stay in 32 bits: the launch refuses more than 2^31 of them; the division by
+    // the chunk count below would otherwise be a 64-bit one, a hundred instructions per item)
+    const uint32_t n_items = (uint32_t)n_entries * (uint32_t)n_chunks;
     // Items differ a lot in cost (a literal state decides nearly everything word-wise, a
     // free-text state walks thousands of tokens), so after its first item a block takes the next
     // one from a device counter instead of a fixed stride.
-    __shared__ long long next_item;
-    for (long long item = blockIdx.x; item < n_items; item = next_item) {
-        const int m = (int)(item / n_chunks);
-        const int t_begin = work.t_first + (int)(item % n_chunks) * work.chunk;
+    __shared__ uint32_t next_item;
+    for (uint32_t item = blockIdx.x; item < n_items; item = next_item) {
+        const int m = (int)(item / (uint32_t)n_chunks);
+        const int t_begin = work.t_first + (int)(item - (uint32_t)m * (uint32_t)n_chunks) * work.chunk;
         const int t_end = min(t_begin + work.chunk, work.t_last);
         const int gid = work.gid[m];
         uint32_t s0 = (uint32_t)work.sid[m];
@@ -413,7 +415,7 @@ build_masks_kernel(VocabDev v, CtxDev ctx, BuildWork work) {
                                   t_begin >> 10, n_words, words, v.V, v.W);
         }
         __syncthreads();  // (also: nobody reads next_item any more before it is rewritten)
-        if (threadIdx.x == 0) next_item = (long long)gridDim.x + atomicAdd(ctx.build_next, 1);
+        if (threadIdx.x == 0) next_item = gridDim.x + (uint32_t)atomicAdd(ctx.build_next, 1);
         __syncthreads();
     }
     // the last block to leave puts the counters back to zero for the next launch
