@@ -266,6 +266,16 @@ build_masks_kernel(VocabDev v, CtxDev ctx, BuildWork work) {
     __shared__ uint8_t first_list[128];  // first bytes to OR (or to exclude, when complemented)
     __shared__ uint8_t fold_list[64];
     __shared__ int n_first, n_fold;
+    __shared__ struct {
+        const void *table;
+        const uint8_t *byte_class;
+        const uint4 *rec_class;
+        uint32_t *dst;
+        unsigned long long leaves, after_fold;
+        uint32_t first_ok[8];
+        uint32_t s0, eos_next;
+        int32_t gid, n_classes, wide, n_ok, forced_tok, after_k;
+    } info;
     __shared__ uint32_t words[BUILD_CHUNK_MAX / 32];
     __shared__ uint16_t todo[BUILD_CHUNK_MAX];
     __shared__ int n_todo;
@@ -286,48 +296,76 @@ build_masks_kernel(VocabDev v, CtxDev ctx, BuildWork work) {
         const int m = (int)(item / (uint32_t)n_chunks);
         const int t_begin = work.t_first + (int)(item - (uint32_t)m * (uint32_t)n_chunks) * work.chunk;
         const int t_end = min(t_begin + work.chunk, work.t_last);
-        const int gid = work.gid[m];
-        uint32_t s0 = (uint32_t)work.sid[m];
-        uint32_t *dst = work.dst_list ? work.dst_list[m] : work.dst_base + (int64_t)m * work.dst_stride;
-        const bool known = gid >= 0 && gid < ctx.n_grammars;
-        GrammarDev g = {};
-        if (known) g = ctx.grammars[gid];
-        if (!known || s0 >= (uint32_t)g.n_states) s0 = 0;  // unknown state: an all-zero row
-        if (t_begin == work.t_first && threadIdx.x == 0) {
-            atomicAdd(&ctx.stats[ST_BUILT], 1ull);
-            if (s0 == 0 && work.sid[m] != 0) atomicAdd(&ctx.stats[ST_BAD_STATE], 1ull);
-        }
         __syncthreads();  // the previous item is done with the shared arrays
-        if (known && cls_gid != gid) cls[threadIdx.x] = g.byte_class[threadIdx.x];
-        if (threadIdx.x == 0) { n_todo = 0; n_first = 0; n_fold = 0; }
-        // the state's first-byte set; complemented when more than half of the bytes are fine
-        const uint32_t ok_word = s0 ? g.first_ok[(size_t)s0 * 8 + (threadIdx.x >> 5)] : 0u;
-        int n_ok = 0;
-        if (s0) {
+        // Warp 0 gathers the facts about the item's mask (grammar record, the state's sets) and
+        // leaves them in shared memory; the other warps wait at the barrier instead of each
+        // repeating the same two hundred instructions.
+        if (threadIdx.x < 32) {
+            const int gid_ = work.gid[m];
+            uint32_t s_ = (uint32_t)work.sid[m];
+            const bool known_ = gid_ >= 0 && gid_ < ctx.n_grammars;
+            GrammarDev g = {};
+            if (known_) g = ctx.grammars[gid_];
+            if (!known_ || s_ >= (uint32_t)g.n_states) s_ = 0;  // unknown state: an all-zero row
+            const uint32_t ok_word_ = (s_ && lane < 8) ? g.first_ok[(size_t)s_ * 8 + lane] : 0u;
+            int n_ok_ = __popc(ok_word_);
 #pragma unroll
-            for (int i = 0; i < 8; ++i) n_ok += __popc(g.first_ok[(size_t)s0 * 8 + i]);
-        }
-        const bool complement = n_ok > 128;
-        const unsigned long long leaves = s0 ? g.leaves[s0] : 0ull;
-        const bool queue_all = __popcll(leaves) > BUILD_MAX_FOLDS;
-        uint32_t eos_next = 0;
-        if (s0) eos_next = g.wide ? static_cast<const uint32_t *>(g.table)[(size_t)s0 * g.n_classes + g.eos_class]
-                                  : static_cast<const uint16_t *>(g.table)[(size_t)s0 * g.n_classes + g.eos_class];
-        const int forced_tok = (s0 && g.forced) ? g.forced[s0].x : -1;  // token-level Write state
-        // A free-text slot has ONE byte that leads on (its closing byte); a token that holds it is
-        // dead unless that byte ends the token or the byte after its first occurrence survives
-        // in the next state.  The vocabulary masks for that byte turn this into word-wise work.
-        int after_k = -1;
-        unsigned long long after_fold = 0ull;
-        if (s0 && ctx.after_masks) {
-            const int lv = g.leave1[s0];
-            if (lv >= 0) {
-                after_fold = g.leave_fold[s0];  // 0: not a state the masks were made for
-                if (after_fold != 0ull) after_k = ctx.after_slot[lv];
+            for (int o = 4; o > 0; o >>= 1) n_ok_ += __shfl_xor_sync(0xFFFFFFFFu, n_ok_, o);
+            if (lane < 8) info.first_ok[lane] = ok_word_;
+            if (lane == 0) {
+                info.gid = known_ ? gid_ : -1;
+                info.s0 = s_;
+                info.dst = work.dst_list ? work.dst_list[m] : work.dst_base + (int64_t)m * work.dst_stride;
+                info.table = g.table;
+                info.byte_class = g.byte_class;
+                info.rec_class = g.rec_class;
+                info.n_classes = g.n_classes;
+                info.wide = g.wide;
+                info.n_ok = n_ok_;
+                info.leaves = s_ ? g.leaves[s_] : 0ull;
+                uint32_t eos_ = 0;
+                if (s_) eos_ = g.wide ? static_cast<const uint32_t *>(g.table)[(size_t)s_ * g.n_classes + g.eos_class]
+                                     : static_cast<const uint16_t *>(g.table)[(size_t)s_ * g.n_classes + g.eos_class];
+                info.eos_next = eos_;
+                info.forced_tok = (s_ && g.forced) ? g.forced[s_].x : -1;  // token-level Write state
+                // A free-text slot has ONE byte that leads on (its closing byte); a token that
+                // holds it is dead unless that byte ends the token or the byte after its first
+                // occurrence survives in the next state.  The vocabulary masks for that byte turn
+                // this into word-wise work.
+                int k_ = -1;
+                unsigned long long fold_ = 0ull;
+                if (s_ && ctx.after_masks) {
+                    const int lv = g.leave1[s_];
+                    if (lv >= 0) {
+                        fold_ = g.leave_fold[s_];  // 0: not a state the masks were made for
+                        if (fold_ != 0ull) k_ = ctx.after_slot[lv];
+                    }
+                }
+                info.after_k = k_;
+                info.after_fold = fold_;
+                n_todo = 0; n_first = 0; n_fold = 0;
+                if (t_begin == work.t_first) {
+                    atomicAdd(&ctx.stats[ST_BUILT], 1ull);
+                    if (s_ == 0 && work.sid[m] != 0) atomicAdd(&ctx.stats[ST_BAD_STATE], 1ull);
+                }
             }
         }
         __syncthreads();
-        if (threadIdx.x == 0 && known) cls_gid = gid;  // read again only after the next barrier
+        const int gid = info.gid;
+        const bool known = gid >= 0;
+        const uint32_t s0 = info.s0;
+        uint32_t *dst = info.dst;
+        if (known && cls_gid != gid) cls[threadIdx.x] = info.byte_class[threadIdx.x];
+        // the state's first-byte set; complemented when more than half of the bytes are fine
+        const uint32_t ok_word = info.first_ok[threadIdx.x >> 5];
+        const int n_ok = info.n_ok;
+        const bool complement = n_ok > 128;
+        const unsigned long long leaves = info.leaves;
+        const bool queue_all = __popcll(leaves) > BUILD_MAX_FOLDS;
+        const uint32_t eos_next = info.eos_next;
+        const int forced_tok = info.forced_tok;
+        const int after_k = info.after_k;
+        const unsigned long long after_fold = info.after_fold;
         {
             const bool is_ok = (ok_word >> lane) & 1u;   // thread b looks at byte b
             if (is_ok != complement) first_list[atomicAdd(&n_first, 1)] = (uint8_t)threadIdx.x;
@@ -335,6 +373,7 @@ build_masks_kernel(VocabDev v, CtxDev ctx, BuildWork work) {
                 fold_list[atomicAdd(&n_fold, 1)] = (uint8_t)threadIdx.x;
         }
         __syncthreads();
+        if (threadIdx.x == 0 && known) cls_gid = gid;  // read again only after the next barrier
         // phase 1: one word of 32 tokens per thread
         const int n_words = (t_end - t_begin) >> 5;
         const int nf = n_first, nq = n_fold;
@@ -394,11 +433,11 @@ build_masks_kernel(VocabDev v, CtxDev ctx, BuildWork work) {
         for (int i = threadIdx.x; i < n; i += BUILD_THREADS) {
             const int rel = todo[i];
             // (the EOS token is never queued: it has no bytes)
-            const uint32_t end = g.wide
-                ? walk_token_classes<uint32_t>(v, g.rec_class, static_cast<const uint32_t *>(g.table),
-                                               g.n_classes, cls, s0, t_begin + rel)
-                : walk_token_classes<uint16_t>(v, g.rec_class, static_cast<const uint16_t *>(g.table),
-                                               g.n_classes, cls, s0, t_begin + rel);
+            const uint32_t end = info.wide
+                ? walk_token_classes<uint32_t>(v, info.rec_class, static_cast<const uint32_t *>(info.table),
+                                               info.n_classes, cls, s0, t_begin + rel)
+                : walk_token_classes<uint16_t>(v, info.rec_class, static_cast<const uint16_t *>(info.table),
+                                               info.n_classes, cls, s0, t_begin + rel);
             if (end != 0) atomicOr(&words[rel >> 5], 1u << (rel & 31));
         }
         __syncthreads();
