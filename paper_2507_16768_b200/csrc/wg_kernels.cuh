@@ -261,12 +261,9 @@ struct BuildWork {
 template <bool COMPACT>
 __global__ void __launch_bounds__(BUILD_THREADS, COMPACT ? 5 : 8)
 build_masks_kernel(VocabDev v, CtxDev ctx, BuildWork work) {
-    __shared__ uint8_t cls[256];
-    __shared__ int cls_gid;
-    __shared__ uint8_t first_list[128];  // first bytes to OR (or to exclude, when complemented)
-    __shared__ uint8_t fold_list[64];
-    __shared__ int n_first, n_fold;
-    __shared__ struct {
+    // the facts about one work item's mask, gathered by warp 0 (two copies: the next item's are
+    // gathered while the other warps walk the current item's tokens)
+    struct ItemFacts {
         const void *table;
         const uint8_t *byte_class;
         const uint4 *rec_class;
@@ -275,82 +272,91 @@ build_masks_kernel(VocabDev v, CtxDev ctx, BuildWork work) {
         uint32_t first_ok[8];
         uint32_t s0, eos_next;
         int32_t gid, n_classes, wide, n_ok, forced_tok, after_k;
-    } info;
+    };
+    __shared__ ItemFacts facts[2];
+    __shared__ uint8_t cls[256];
+    __shared__ int cls_gid;
+    __shared__ uint8_t first_list[128];  // first bytes to OR (or to exclude, when complemented)
+    __shared__ uint8_t fold_list[64];
+    __shared__ int n_first, n_fold;
     __shared__ uint32_t words[BUILD_CHUNK_MAX / 32];
     __shared__ uint16_t todo[BUILD_CHUNK_MAX];
     __shared__ int n_todo;
+    __shared__ uint32_t next_item;
     pdl_enter();
-    if (threadIdx.x == 0) cls_gid = -1;
-    __syncthreads();
     const int lane = threadIdx.x & 31;
     const int n_entries = work.count_ptr ? *work.count_ptr : work.count;
     const int n_chunks = (work.t_last - work.t_first + work.chunk - 1) / work.chunk;
     // (item numbers stay in 32 bits: the launch refuses more than 2^31 of them; the division by
     // the chunk count below would otherwise be a 64-bit one, a hundred instructions per item)
     const uint32_t n_items = (uint32_t)n_entries * (uint32_t)n_chunks;
+
+    // Called by warp 0: the grammar record and the state's sets of item `it` into fx.
+    auto gather = [&](uint32_t it, ItemFacts &fx) {
+        const int m = (int)(it / (uint32_t)n_chunks);
+        const int t_begin_ = work.t_first + (int)(it - (uint32_t)m * (uint32_t)n_chunks) * work.chunk;
+        const int gid_ = work.gid[m];
+        uint32_t s_ = (uint32_t)work.sid[m];
+        const bool known_ = gid_ >= 0 && gid_ < ctx.n_grammars;
+        GrammarDev g = {};
+        if (known_) g = ctx.grammars[gid_];
+        if (!known_ || s_ >= (uint32_t)g.n_states) s_ = 0;  // unknown state: an all-zero row
+        const uint32_t ok_word_ = (s_ && lane < 8) ? g.first_ok[(size_t)s_ * 8 + lane] : 0u;
+        int n_ok_ = __popc(ok_word_);
+#pragma unroll
+        for (int o = 4; o > 0; o >>= 1) n_ok_ += __shfl_xor_sync(0xFFFFFFFFu, n_ok_, o);
+        if (lane < 8) fx.first_ok[lane] = ok_word_;
+        if (lane == 0) {
+            fx.gid = known_ ? gid_ : -1;
+            fx.s0 = s_;
+            fx.dst = work.dst_list ? work.dst_list[m] : work.dst_base + (int64_t)m * work.dst_stride;
+            fx.table = g.table;
+            fx.byte_class = g.byte_class;
+            fx.rec_class = g.rec_class;
+            fx.n_classes = g.n_classes;
+            fx.wide = g.wide;
+            fx.n_ok = n_ok_;
+            fx.leaves = s_ ? g.leaves[s_] : 0ull;
+            uint32_t eos_ = 0;
+            if (s_) eos_ = g.wide ? static_cast<const uint32_t *>(g.table)[(size_t)s_ * g.n_classes + g.eos_class]
+                                 : static_cast<const uint16_t *>(g.table)[(size_t)s_ * g.n_classes + g.eos_class];
+            fx.eos_next = eos_;
+            fx.forced_tok = (s_ && g.forced) ? g.forced[s_].x : -1;  // token-level Write state
+            // A free-text slot has ONE byte that leads on (its closing byte); a token that
+            // holds it is dead unless that byte ends the token or the byte after its first
+            // occurrence survives in the next state.  The vocabulary masks for that byte turn
+            // this into word-wise work.
+            int k_ = -1;
+            unsigned long long fold_ = 0ull;
+            if (s_ && ctx.after_masks) {
+                const int lv = g.leave1[s_];
+                if (lv >= 0) {
+                    fold_ = g.leave_fold[s_];  // 0: not a state the masks were made for
+                    if (fold_ != 0ull) k_ = ctx.after_slot[lv];
+                }
+            }
+            fx.after_k = k_;
+            fx.after_fold = fold_;
+                if (t_begin_ == work.t_first) {
+                atomicAdd(&ctx.stats[ST_BUILT], 1ull);
+                if (s_ == 0 && work.sid[m] != 0) atomicAdd(&ctx.stats[ST_BAD_STATE], 1ull);
+            }
+        }
+    };
+
+    if (threadIdx.x == 0) { cls_gid = -1; n_todo = 0; n_first = 0; n_fold = 0; }
+    if (threadIdx.x < 32 && blockIdx.x < n_items) gather(blockIdx.x, facts[0]);
+    __syncthreads();
     // Items differ a lot in cost (a literal state decides nearly everything word-wise, a
     // free-text state walks thousands of tokens), so after its first item a block takes the next
-    // one from a device counter instead of a fixed stride.
-    __shared__ uint32_t next_item;
-    for (uint32_t item = blockIdx.x; item < n_items; item = next_item) {
+    // one from a device counter instead of a fixed stride.  Warp 0 does that, and gathers the
+    // next item's facts, while the other seven warps walk the current item's queued tokens.
+    int cur = 0;
+    for (uint32_t item = blockIdx.x; item < n_items; item = next_item, cur ^= 1) {
+        const ItemFacts &info = facts[cur];
         const int m = (int)(item / (uint32_t)n_chunks);
         const int t_begin = work.t_first + (int)(item - (uint32_t)m * (uint32_t)n_chunks) * work.chunk;
         const int t_end = min(t_begin + work.chunk, work.t_last);
-        __syncthreads();  // the previous item is done with the shared arrays
-        // Warp 0 gathers the facts about the item's mask (grammar record, the state's sets) and
-        // leaves them in shared memory; the other warps wait at the barrier instead of each
-        // repeating the same two hundred instructions.
-        if (threadIdx.x < 32) {
-            const int gid_ = work.gid[m];
-            uint32_t s_ = (uint32_t)work.sid[m];
-            const bool known_ = gid_ >= 0 && gid_ < ctx.n_grammars;
-            GrammarDev g = {};
-            if (known_) g = ctx.grammars[gid_];
-            if (!known_ || s_ >= (uint32_t)g.n_states) s_ = 0;  // unknown state: an all-zero row
-            const uint32_t ok_word_ = (s_ && lane < 8) ? g.first_ok[(size_t)s_ * 8 + lane] : 0u;
-            int n_ok_ = __popc(ok_word_);
-#pragma unroll
-            for (int o = 4; o > 0; o >>= 1) n_ok_ += __shfl_xor_sync(0xFFFFFFFFu, n_ok_, o);
-            if (lane < 8) info.first_ok[lane] = ok_word_;
-            if (lane == 0) {
-                info.gid = known_ ? gid_ : -1;
-                info.s0 = s_;
-                info.dst = work.dst_list ? work.dst_list[m] : work.dst_base + (int64_t)m * work.dst_stride;
-                info.table = g.table;
-                info.byte_class = g.byte_class;
-                info.rec_class = g.rec_class;
-                info.n_classes = g.n_classes;
-                info.wide = g.wide;
-                info.n_ok = n_ok_;
-                info.leaves = s_ ? g.leaves[s_] : 0ull;
-                uint32_t eos_ = 0;
-                if (s_) eos_ = g.wide ? static_cast<const uint32_t *>(g.table)[(size_t)s_ * g.n_classes + g.eos_class]
-                                     : static_cast<const uint16_t *>(g.table)[(size_t)s_ * g.n_classes + g.eos_class];
-                info.eos_next = eos_;
-                info.forced_tok = (s_ && g.forced) ? g.forced[s_].x : -1;  // token-level Write state
-                // A free-text slot has ONE byte that leads on (its closing byte); a token that
-                // holds it is dead unless that byte ends the token or the byte after its first
-                // occurrence survives in the next state.  The vocabulary masks for that byte turn
-                // this into word-wise work.
-                int k_ = -1;
-                unsigned long long fold_ = 0ull;
-                if (s_ && ctx.after_masks) {
-                    const int lv = g.leave1[s_];
-                    if (lv >= 0) {
-                        fold_ = g.leave_fold[s_];  // 0: not a state the masks were made for
-                        if (fold_ != 0ull) k_ = ctx.after_slot[lv];
-                    }
-                }
-                info.after_k = k_;
-                info.after_fold = fold_;
-                n_todo = 0; n_first = 0; n_fold = 0;
-                if (t_begin == work.t_first) {
-                    atomicAdd(&ctx.stats[ST_BUILT], 1ull);
-                    if (s_ == 0 && work.sid[m] != 0) atomicAdd(&ctx.stats[ST_BAD_STATE], 1ull);
-                }
-            }
-        }
-        __syncthreads();
         const int gid = info.gid;
         const bool known = gid >= 0;
         const uint32_t s0 = info.s0;
@@ -428,19 +434,29 @@ build_masks_kernel(VocabDev v, CtxDev ctx, BuildWork work) {
             }
         }
         __syncthreads();
-        // phase 2: walk the queued tokens, one per thread
+        if (threadIdx.x == 0) { n_first = 0; n_fold = 0; }  // everybody has read them
+        // phase 2: warp 0 takes the block's next item and gathers its facts; the other warps
+        // walk the queued tokens, one per thread (the EOS token is never queued: it has no bytes)
         const int n = n_todo;
-        for (int i = threadIdx.x; i < n; i += BUILD_THREADS) {
-            const int rel = todo[i];
-            // (the EOS token is never queued: it has no bytes)
-            const uint32_t end = info.wide
-                ? walk_token_classes<uint32_t>(v, info.rec_class, static_cast<const uint32_t *>(info.table),
-                                               info.n_classes, cls, s0, t_begin + rel)
-                : walk_token_classes<uint16_t>(v, info.rec_class, static_cast<const uint16_t *>(info.table),
-                                               info.n_classes, cls, s0, t_begin + rel);
-            if (end != 0) atomicOr(&words[rel >> 5], 1u << (rel & 31));
+        if (threadIdx.x < 32) {
+            uint32_t nxt = 0;
+            if (lane == 0) nxt = gridDim.x + (uint32_t)atomicAdd(ctx.build_next, 1);
+            nxt = __shfl_sync(0xFFFFFFFFu, nxt, 0);
+            if (lane == 0) next_item = nxt;
+            if (nxt < n_items) gather(nxt, facts[cur ^ 1]);
+        } else {
+            for (int i = threadIdx.x - 32; i < n; i += BUILD_THREADS - 32) {
+                const int rel = todo[i];
+                const uint32_t end = info.wide
+                    ? walk_token_classes<uint32_t>(v, info.rec_class, static_cast<const uint32_t *>(info.table),
+                                                   info.n_classes, cls, s0, t_begin + rel)
+                    : walk_token_classes<uint16_t>(v, info.rec_class, static_cast<const uint16_t *>(info.table),
+                                                   info.n_classes, cls, s0, t_begin + rel);
+                if (end != 0) atomicOr(&words[rel >> 5], 1u << (rel & 31));
+            }
         }
         __syncthreads();
+        if (threadIdx.x == 0) n_todo = 0;  // everybody has read it
         // phase 3: whole words out
         for (int wl = threadIdx.x; wl < n_words; wl += BUILD_THREADS)
             dst[(t_begin >> 5) + wl] = words[wl];
@@ -453,9 +469,7 @@ build_masks_kernel(VocabDev v, CtxDev ctx, BuildWork work) {
                                   ctx.arena_words, ctx.ent_fail + row, ctx.stats + ST_UNCACHED,
                                   t_begin >> 10, n_words, words, v.V, v.W);
         }
-        __syncthreads();  // (also: nobody reads next_item any more before it is rewritten)
-        if (threadIdx.x == 0) next_item = gridDim.x + (uint32_t)atomicAdd(ctx.build_next, 1);
-        __syncthreads();
+        __syncthreads();  // the shared arrays are free for the next item
     }
     // the last block to leave puts the counters back to zero for the next launch
     if (threadIdx.x == 0) {
