@@ -337,7 +337,7 @@ build_masks_kernel(VocabDev v, CtxDev ctx, BuildWork work) {
             }
             fx.after_k = k_;
             fx.after_fold = fold_;
-                if (t_begin_ == work.t_first) {
+            if (t_begin_ == work.t_first) {
                 atomicAdd(&ctx.stats[ST_BUILT], 1ull);
                 if (s_ == 0 && work.sid[m] != 0) atomicAdd(&ctx.stats[ST_BAD_STATE], 1ull);
             }
