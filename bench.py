@@ -32,7 +32,7 @@ from wg_workloads import BY_NAME, flatten, has_structural_byte, make_logits, mak
 # dram__bytes_read.sum + dram__bytes_write.sum of ONE launch of the dominant kernel, from the ncu
 # capture summarised under profiles/ (same launch shape as the timed run).  Set an entry to None
 # when its kernel changes and the capture has not been redone.
-BUILD_WARP_INSTR_PER_TOKEN = 0.42  # mean of the two launches under profiles/build_masks_kernel_cold_templates*.md
+BUILD_WARP_INSTR_PER_TOKEN = 0.44  # mean of the two launches under profiles/build_masks_kernel_cold_templates*.md
 
 NCU_TRAFFIC_BYTES = {
     "json_warm": 221.1e6,       # profiles/apply_mask_kernel_json_warm.md
@@ -430,8 +430,8 @@ def run_ours(args, w, steer: float) -> None:
     else:
         # Issue-slot bound of the build kernel: 148 SMs x 4 schedulers x 1 warp instruction per
         # clock at the sampled SM clock, divided by the warp instructions the kernel spends per
-        # token checked (ncu: 13.1 M and 19.3 M instructions for two launches of 256 x 151 936
-        # tokens, early and late in a run: 0.42 per token on average).
+        # token checked (ncu: 13.8 M and 20.2 M instructions for two launches of 256 x 151 936
+        # tokens, early and late in a run: 0.44 per token on average).
         sm_mhz = clocks.get("sm_mhz") or 1965.0
         peak_tok = 148 * 4 * sm_mhz * 1e6 / BUILD_WARP_INSTR_PER_TOKEN
         tok_per_s = built_timed * Vs / (kt["build_ms"] * 1e-3) if kt["build_ms"] > 0 else 0.0
