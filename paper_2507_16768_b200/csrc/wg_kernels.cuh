@@ -103,21 +103,9 @@ __device__ __forceinline__ void pdl_enter();
 // ---------------------------------------------------------------------------------------
 // table walk
 // ---------------------------------------------------------------------------------------
-template <typename T>
-__device__ __forceinline__ uint32_t walk_record(const T *__restrict__ tab, int C,
-                                                const uint8_t *cls, uint32_t s, uint4 rec, int n) {
-    const uint32_t w[4] = {rec.x, rec.y, rec.z, rec.w};
-#pragma unroll
-    for (int j = 0; j < WG_REC_BYTES; ++j) {
-        if (j >= n || s == 0) break;
-        const uint32_t b = (w[j >> 2] >> (8 * (j & 3))) & 0xFFu;
-        s = tab[(size_t)s * C + cls[b]];
-    }
-    return s;
-}
-
-// The walk of the build kernel: the first 16 bytes come as classes straight from the
-// grammar's class-mapped record, so every step is one dependent table look-up.
+// The token walk (build and advance kernels): state after token t from state s (0 = DEAD).
+// The first 16 bytes come as classes straight from the grammar's class-mapped record, so every
+// step is one dependent table look-up; longer tokens continue from the CSR bytes.
 template <typename T>
 __device__ __forceinline__ uint32_t walk_token_classes(const VocabDev &v, const uint4 *rec_class,
                                                        const T *__restrict__ tab, int C,
@@ -137,23 +125,6 @@ __device__ __forceinline__ uint32_t walk_token_classes(const VocabDev &v, const 
     if (n > WG_REC_BYTES && s != 0) {
         const uint32_t b = v.offsets[t] + WG_REC_BYTES, e = v.offsets[t + 1];
         for (uint32_t i = b; i < e && s != 0; ++i) s = tab[s * Cu + cls[v.bytes[i]]];
-    }
-    return s;
-}
-
-// State after token t from state s (0 = DEAD).  cls: the grammar's byte classes (shared or
-// global memory).  Tokens longer than the record continue from the CSR bytes.
-template <typename T>
-__device__ __forceinline__ uint32_t walk_token(const VocabDev &v, const T *__restrict__ tab,
-                                               int C, int eos_class, const uint8_t *cls,
-                                               uint32_t s, int t) {
-    if (t == v.eos_id) return tab[(size_t)s * C + eos_class];
-    const int n = v.len[t];
-    if (n == 0) return 0;
-    s = walk_record(tab, C, cls, s, __ldg(&v.rec[t]), n);
-    if (n > WG_REC_BYTES && s != 0) {
-        const uint32_t b = v.offsets[t] + WG_REC_BYTES, e = v.offsets[t + 1];
-        for (uint32_t i = b; i < e && s != 0; ++i) s = tab[(size_t)s * C + cls[v.bytes[i]]];
     }
     return s;
 }
@@ -1187,10 +1158,17 @@ __global__ void advance_kernel(VocabDev v, CtxDev ctx, const int32_t *gid, int32
             const int2 f = gr.forced[s];
             if (t == f.x && t < v.V) next = (uint32_t)f.y;
         } else if (t >= 0 && t < v.V && s != 0) {
-            next = gr.wide ? walk_token<uint32_t>(v, static_cast<const uint32_t *>(gr.table),
-                                                  gr.n_classes, gr.eos_class, gr.byte_class, s, t)
-                           : walk_token<uint16_t>(v, static_cast<const uint16_t *>(gr.table),
-                                                  gr.n_classes, gr.eos_class, gr.byte_class, s, t);
+            // the class-mapped record of the token: one dependent look-up per byte instead of
+            // two (this kernel is a chain of dependent loads at the very end of every step)
+            if (t == v.eos_id)
+                next = gr.wide ? static_cast<const uint32_t *>(gr.table)[(size_t)s * gr.n_classes + gr.eos_class]
+                               : static_cast<const uint16_t *>(gr.table)[(size_t)s * gr.n_classes + gr.eos_class];
+            else
+                next = gr.wide
+                    ? walk_token_classes<uint32_t>(v, gr.rec_class, static_cast<const uint32_t *>(gr.table),
+                                                   gr.n_classes, gr.byte_class, s, t)
+                    : walk_token_classes<uint16_t>(v, gr.rec_class, static_cast<const uint16_t *>(gr.table),
+                                                   gr.n_classes, gr.byte_class, s, t);
         }
         if (next == 0) {
             st = WG_ERR_TOKEN_REJECTED;
