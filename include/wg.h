@@ -285,17 +285,19 @@ void wg_ctx_free(wg_ctx *ctx);
  * WG_CACHE_DENSE is wg_ctx_create.  WG_CACHE_COMPACT stores every cached mask the way the
  * paper's Wait operator keeps its token sets (Section 3.3: a few refused tokens in `denies`
  * when most of the vocabulary is accepted, the accepted ones in `allows` when most is
- * refused): the side with fewer tokens is kept -- allows when at most half of the V tokens
- * are allowed, denies otherwise.  On the device an entry holds its listed tokens grouped by
- * 32-token mask word (only the words that contain a listed token are stored, behind a small
- * per-span index), so an entry never takes more room than the id list and a row is masked
- * straight from it.  Masks of literal states and of free-text slots shrink from V/8 bytes to
- * a few hundred bytes, which is what lets grammars with hundreds of thousands of states stay
- * cached.  Results of every call are identical in both modes.
- *   arena_bytes  device memory for the entries; 0 = a quarter of what cache_capacity dense
- *                rows would take.  When the arena is full, further new states are built on
+ * refused): the side with fewer tokens is kept.  On the device the choice is made for every
+ * span of 1024 tokens by itself (never worse than one choice per mask), and a span holds its
+ * listed tokens grouped by 32-token mask word: only the words that contain a listed token are
+ * stored, behind an 8-byte header per span, so a mask never takes more room than its id list
+ * plus the headers, and a row is masked straight from it.  Masks of literal states and of
+ * free-text slots shrink from V/8 bytes to about a kilobyte, which is what lets grammars with
+ * hundreds of thousands of states stay cached.  Results of every call are identical in both
+ * modes; wg_cache_entry_read reports an entry as the paper's per-mask allows / denies set.
+ *   arena_bytes  device memory for the stored words; 0 = a quarter of what cache_capacity
+ *                dense rows would take (the span headers, capacity x ceil(W/32) x 8 bytes,
+ *                come on top).  When the arena is full, further new states are built on
  *                every step (counted as rows_uncached), as with a full dense pool.
- * Errors: WG_ERR_ARG (also: unknown cache_mode, V above 1 048 576 in compact mode), WG_ERR_CUDA. */
+ * Errors: WG_ERR_ARG (also: unknown cache_mode), WG_ERR_CUDA. */
 int32_t wg_ctx_create_ex(const wg_vocab *vocab, int32_t cache_capacity, int32_t max_batch,
                          int32_t cache_mode, size_t arena_bytes, wg_ctx **out);
 
