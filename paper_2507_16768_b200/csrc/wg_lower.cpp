@@ -15,6 +15,7 @@
 #include <cstring>
 #include <queue>
 #include <unordered_map>
+#include <utility>
 
 #include "wg_internal.h"
 
@@ -461,6 +462,7 @@ int32_t wg_minimize_grammar(const wg_grammar &in, wg_grammar *out) {
     const int width = C + 2;
     std::vector<int32_t> sig((size_t)S * width);
     std::vector<int32_t> order(S), next_block(S);
+    std::vector<std::pair<uint64_t, int32_t>> keyed(S);
     for (;;) {
         for (int32_t s = 0; s < S; ++s) {
             int32_t *row = &sig[(size_t)s * width];
@@ -468,11 +470,32 @@ int32_t wg_minimize_grammar(const wg_grammar &in, wg_grammar *out) {
             for (int32_t c = 0; c < C; ++c) row[1 + c] = block[in.table[(size_t)s * C + c]];
             row[1 + C] = (forced && in.forced_tok[s] >= 0) ? block[in.forced_next[s]] : -1;
         }
-        for (int32_t s = 0; s < S; ++s) order[s] = s;
-        std::sort(order.begin(), order.end(), [&](int32_t a, int32_t b) {
+        // states with equal signatures next to each other: sort by a hash of the row (sorting
+        // the wide rows themselves took most of the time), then by the rows inside the rare runs
+        // where different rows share a hash
+        auto row_less = [&](int32_t a, int32_t b) {
             const int cmp = memcmp(&sig[(size_t)a * width], &sig[(size_t)b * width], sizeof(int32_t) * width);
             return cmp != 0 ? cmp < 0 : a < b;
-        });
+        };
+        for (int32_t s = 0; s < S; ++s) {
+            uint64_t h = 0xCBF29CE484222325ull;
+            const int32_t *row = &sig[(size_t)s * width];
+            for (int i = 0; i < width; ++i) { h = (h ^ (uint32_t)row[i]) * 0x100000001B3ull; h ^= h >> 32; }
+            keyed[s] = {h, s};
+        }
+        std::sort(keyed.begin(), keyed.end());
+        for (int32_t s = 0; s < S; ++s) order[s] = keyed[s].second;
+        for (int32_t i = 0; i < S;) {
+            int32_t j = i + 1;
+            bool mixed = false;
+            while (j < S && keyed[j].first == keyed[i].first) {
+                mixed |= memcmp(&sig[(size_t)order[j] * width], &sig[(size_t)order[i] * width],
+                                sizeof(int32_t) * width) != 0;
+                ++j;
+            }
+            if (mixed) std::sort(order.begin() + i, order.begin() + j, row_less);
+            i = j;
+        }
         int32_t n_next = 0;
         for (int32_t i = 0; i < S; ++i) {
             if (i > 0 && memcmp(&sig[(size_t)order[i] * width], &sig[(size_t)order[i - 1] * width],
