@@ -363,12 +363,26 @@ int32_t wg_lower_tree(const wg_op_node *nodes, int32_t n_nodes, const int32_t *c
         };
         std::unordered_map<SymSet, int, SetHash, SetEq> seen;
         std::vector<int32_t> renum;
+        std::vector<int32_t> class_size(1, WG_N_SYMBOLS);
         for (int32_t i = 0; i < S; ++i) {
             for (const Edge &e : lw.states[order[i]]) {
                 const auto ins = seen.emplace(e.on, (int)distinct.size());
                 edge_set.push_back(ins.first->second);
                 if (!ins.second) continue;
                 distinct.push_back(e.on);
+                // a one-symbol set (a literal's byte, a branch of an enum: most sets) only takes
+                // its symbol out of the class it shares with others
+                int members = 0, only = -1;
+                for (int wi = 0; wi < WG_SET_WORDS; ++wi)
+                    if (e.on.w[wi]) { members += __builtin_popcount(e.on.w[wi]); only = wi * 32 + __builtin_ctz(e.on.w[wi]); }
+                if (members == 1) {
+                    if (class_size[cls[only]] > 1) {
+                        --class_size[cls[only]];
+                        cls[only] = n_cls++;
+                        class_size.push_back(1);
+                    }
+                    continue;
+                }
                 renum.assign((size_t)n_cls * 2, -1);
                 int32_t n_next = 0;
                 for (int sym = 0; sym < WG_N_SYMBOLS; ++sym) {
@@ -377,6 +391,8 @@ int32_t wg_lower_tree(const wg_op_node *nodes, int32_t n_nodes, const int32_t *c
                     cls[sym] = renum[key];
                 }
                 n_cls = n_next;
+                class_size.assign(n_cls, 0);
+                for (int sym = 0; sym < WG_N_SYMBOLS; ++sym) ++class_size[cls[sym]];
             }
         }
     }
