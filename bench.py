@@ -37,6 +37,11 @@ BUILD_WARP_INSTR_PER_TOKEN = 0.44  # mean of the two launches under profiles/bui
 NCU_TRAFFIC_BYTES = {
     "json_warm": 221.1e6,       # profiles/apply_mask_kernel_json_warm.md
 }
+# the build kernel reads vocabulary masks, token records and tables that sit in L2: DRAM reads of
+# one launch, mean of the early and the late step under profiles/build_masks_kernel_cold_templates*.md
+NCU_BUILD_TRAFFIC_BYTES = {
+    "cold_templates": 5.7e6,
+}
 
 METRIC = "masked logit rows/s (mask build+apply)"
 UNIT = "rows/s"
@@ -439,7 +444,8 @@ def run_ours(args, w, steer: float) -> None:
                     "achieved": tok_per_s / 1e9, "peak": peak_tok / 1e9,
                     "unit": "G tokens checked/s", "frac": tok_per_s / peak_tok,
                     "peak_kind": "issue slots at the kernel's measured instructions per token",
-                    "traffic": None, "avg_launch_ms": build_ms}
+                    "traffic": NCU_BUILD_TRAFFIC_BYTES.get(w.name) if B == w.batch else None,
+                    "avg_launch_ms": build_ms}
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
