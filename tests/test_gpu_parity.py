@@ -52,7 +52,9 @@ def odd_vocab():
     toks = base.tokens()
     extra = [b"<h1 class=\"document-title\" id=\"outline-root\">", b"section-title\" id=\"outline-",
              b"a" * 17, b"x" * 40 + b"<", b"  " * 9 + b"</p>\n<h2 class=", b"0123456789/0123456789",
-             b'{"topic": 12, "paths": ["1/2', b"q" * 300, b"", b"</h1>\n<p class=\"document-abs"]
+             b'{"topic": 12, "paths": ["1/2', b"q" * 300, b"", b"</h1>\n<p class=\"document-abs",
+             # a slot's closing byte as the last byte of the 16-byte record, and one byte before it
+             b"a" * 15 + b"</h1>\n", b"a" * 14 + b"</", b"a" * 15 + b"<", b"b" * 16 + b"</p>"]
     return vocab_from_tokens(toks + extra + toks[300:311][::-1][:0], eos_id=2)
 
 
