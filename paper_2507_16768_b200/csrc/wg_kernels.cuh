@@ -1128,8 +1128,16 @@ __global__ void advance_kernel(VocabDev v, CtxDev ctx, const int32_t *gid, int32
                                const int32_t *token_in, int32_t *token_out, int B,
                                int32_t *status, uint32_t flags, int from_keys,
                                const long long *ext_keys) {
-    pdl_enter();
+    // What never changes while steps are in flight (the row's grammar id, the grammar's record)
+    // is read BEFORE waiting for the kernel ahead, so that these two dependent loads run under
+    // its tail; states and tokens are only touched after the wait.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int r = blockIdx.x * blockDim.x + threadIdx.x;
+    const int g = r < B ? gid[r] : -1;
+    const bool known = g >= 0 && g < ctx.n_grammars;
+    GrammarDev gr = {};
+    if (known) gr = ctx.grammars[g];
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     if (r >= B) return;
     int t;
     if (from_keys == 2) {
@@ -1142,17 +1150,15 @@ __global__ void advance_kernel(VocabDev v, CtxDev ctx, const int32_t *gid, int32
     } else {
         t = token_in[r];
     }
-    const int g = gid[r];
     const uint32_t s = (uint32_t)sid[r];
     int32_t st = WG_OK;
-    if (g < 0 || g >= ctx.n_grammars || s >= (uint32_t)ctx.grammars[g].n_states) {
+    if (!known || s >= (uint32_t)gr.n_states) {
         st = WG_ERR_STATE;
         atomicAdd(&ctx.stats[ST_BAD_STATE], 1ull);
     } else if (from_keys && t < 0) {
         st = WG_ERR_EMPTY_MASK;
         atomicAdd(&ctx.stats[ST_EMPTY], 1ull);
     } else {
-        const GrammarDev gr = ctx.grammars[g];
         uint32_t next = 0;
         if (gr.forced && s != 0 && gr.forced[s].x >= 0) {  // token-level Write: that token only
             const int2 f = gr.forced[s];
