@@ -990,9 +990,11 @@ apply_mask_kernel(ApplyArgs a, CtxDev ctx, unsigned long long *argkey) {
                     if (sizeof(E) == 2) {
 #pragma unroll
                         for (int i = 0; i < 4; ++i) {
+                            // one byte permute per pair: bytes 0-3 are the pair, 4-7 the two -inf;
+                            // an allowed element takes its own bytes, a refused one those of -inf
                             const uint32_t two = (bits[q] >> (2 * i)) & 3u;
-                            const uint32_t keep = ((two & 1u) ? 0x0000FFFFu : 0u) | ((two & 2u) ? 0xFFFF0000u : 0u);
-                            w[i] = (w[i] & keep) | (NEG_INF_BF16X2 & ~keep);
+                            const uint32_t sel = 0x7654u - 0x0044u * (two & 1u) - 0x4400u * (two >> 1);
+                            w[i] = __byte_perm(w[i], NEG_INF_BF16X2, sel);
                         }
                     } else {
 #pragma unroll
