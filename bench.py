@@ -35,7 +35,7 @@ from wg_workloads import BY_NAME, flatten, has_structural_byte, make_logits, mak
 BUILD_WARP_INSTR_PER_TOKEN = 0.44  # mean of the two launches under profiles/build_masks_kernel_cold_templates*.md
 
 NCU_TRAFFIC_BYTES = {
-    "json_warm": 221.1e6,       # profiles/apply_mask_kernel_json_warm.md
+    "json_warm": 220.9e6,       # profiles/apply_mask_kernel_json_warm.md
 }
 # the build kernel reads vocabulary masks, token records and tables that sit in L2: DRAM reads of
 # one launch, mean of the early and the late step under profiles/build_masks_kernel_cold_templates*.md
