@@ -313,7 +313,9 @@ int32_t wg_cache_entry_read(wg_ctx *ctx, int32_t grammar_id, int32_t state, int3
 
 /* Uploads a compiled grammar's table and returns its id in this context.  A grammar whose
  * content_hash and tables equal one already added gets that grammar's id, so requests
- * instantiated with the same arguments share cache entries.  Synchronous (small copies).
+ * instantiated with the same arguments share cache entries.  Synchronous: the table is
+ * copied and a few set-up kernels run on the legacy default stream, which the call waits for
+ * (so it must not be made while a stream capture is under way).
  * Errors: WG_ERR_ARG, WG_ERR_CAPACITY (more than 65535 grammars, or a table of 2^32 cells or
  * more), WG_ERR_CUDA. */
 int32_t wg_ctx_add_grammar(wg_ctx *ctx, const wg_grammar *grammar, int32_t *grammar_id);
