@@ -62,6 +62,10 @@ typedef enum wg_status {
     WG_ERR_STATE = -7           /* per row: grammar id or state id out of range              */
 } wg_status;
 
+/* Most rows one call may take: the row number is the second grid dimension of the apply
+ * kernels.  wg_ctx_create refuses a larger max_batch, wg_apply_mask a larger B (WG_ERR_ARG). */
+#define WG_MAX_ROWS 65535
+
 /* Logit element types of wg_apply_mask / wg_decode_step. */
 enum { WG_DTYPE_BF16 = 0, WG_DTYPE_FP32 = 1 };
 
@@ -253,7 +257,8 @@ int32_t wg_grammar_minimize(const wg_grammar *grammar, wg_grammar **out);
  *   blob needs in *needed; returns WG_ERR_CAPACITY (nothing written) if capacity is too
  *   small, so a first call with blob = NULL, capacity = 0 asks for the size.
  * wg_grammar_load: rebuilds a grammar from such a blob after checking it (magic, version,
- *   sizes, every table entry and state id in range); a damaged blob gives WG_ERR_ARG.
+ *   sizes, every table entry and state id in range, and the stored content hash against the
+ *   hash of what was read); a damaged blob gives WG_ERR_ARG.
  * The format is little-endian and private to this library version. */
 int32_t wg_grammar_save(const wg_grammar *grammar, void *blob, size_t capacity, size_t *needed);
 int32_t wg_grammar_load(const void *blob, size_t size, wg_grammar **out);
@@ -275,7 +280,7 @@ int32_t wg_grammar_forced_token(const wg_grammar *grammar, int32_t state, int32_
 /* Creates the device context on the current device: grammar table registry, the mask cache
  * (a hash table keyed by (grammar id, state id) plus a pool of `cache_capacity` mask rows,
  * paper Section 3.3) and per-batch scratch for up to `max_batch` rows per call.
- * cache_capacity may be 0 (every WG_USE_CACHE row is then built uncached).
+ * cache_capacity may be 0 (every WG_USE_CACHE row is then built uncached).  max_batch <= WG_MAX_ROWS.
  * The vocabulary must outlive the context.  Errors: WG_ERR_ARG, WG_ERR_CUDA. */
 int32_t wg_ctx_create(const wg_vocab *vocab, int32_t cache_capacity, int32_t max_batch,
                       wg_ctx **out);
@@ -312,7 +317,8 @@ int32_t wg_cache_entry_read(wg_ctx *ctx, int32_t grammar_id, int32_t state, int3
                             int64_t *entry_bytes, void *stream);
 
 /* Uploads a compiled grammar's table and returns its id in this context.  A grammar whose
- * content_hash and tables equal one already added gets that grammar's id, so requests
+ * content_hash, tables, symbol-class map and start / DONE states all equal those of one
+ * already added gets that grammar's id, so requests
  * instantiated with the same arguments share cache entries.  Synchronous: the table is
  * copied and a few set-up kernels run on the legacy default stream, which the call waits for
  * (so it must not be made while a stream capture is under way).
@@ -320,8 +326,10 @@ int32_t wg_cache_entry_read(wg_ctx *ctx, int32_t grammar_id, int32_t state, int3
  * more), WG_ERR_CUDA. */
 int32_t wg_ctx_add_grammar(wg_ctx *ctx, const wg_grammar *grammar, int32_t *grammar_id);
 
-/* Builds and caches the mask of every state of grammar `grammar_id` (states 1..n_states-1).
- * Stops with WG_ERR_CAPACITY if the pool cannot hold them all.  Synchronises `stream`. */
+/* Builds and caches the mask of every state of grammar `grammar_id` (states 1..n_states-1),
+ * max_batch states at a time.  Returns WG_ERR_CAPACITY after the first batch that found the
+ * pool (or the arena) full; the states cached up to then stay cached.  Synchronises `stream`
+ * after every batch. */
 int32_t wg_cache_prewarm(wg_ctx *ctx, int32_t grammar_id, void *stream);
 
 /* Forgets every cached mask (enqueued on `stream`). */
@@ -348,13 +356,15 @@ int32_t wg_mask_cache_lookup(wg_ctx *ctx, const int32_t *gid, const int32_t *sid
  *                     others are built once per distinct state, inserted, then copied.  When
  *                     the pool is full the remaining rows are built straight into `bitmask`.
  *                     WG_NO_CACHE: every row is built, duplicates included.
- * Rows with an unknown grammar or state get an all-zero mask and count as bad_states. */
+ * Rows with an unknown grammar or state get an all-zero mask and count as bad_states, on every
+ * call that meets them: such a row never takes a cache entry (it also counts as rows_uncached). */
 int32_t wg_build_masks(wg_ctx *ctx, const int32_t *gid, const int32_t *sid, int32_t B,
                        uint32_t *bitmask, int64_t row_stride_words, uint32_t flags, void *stream);
 
 /* Mask application (paper Section 1: the mask acts on the logits before a token is sampled),
  * in place.
- *   logits            device, B rows of V elements, row r at logits + r * row_stride_elems
+ *   logits            device, B rows of V elements, row r at logits + r * row_stride_elems;
+ *                     1 <= B <= WG_MAX_ROWS
  *   dtype             WG_DTYPE_BF16 or WG_DTYPE_FP32
  *   bitmask           device, as written by wg_build_masks
  *   argmax_out        device, B entries, or NULL.  When given, token[r] = the lowest id among

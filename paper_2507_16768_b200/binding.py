@@ -136,7 +136,12 @@ def _np_ptr(a: Optional[np.ndarray]):
     return None if a is None else a.ctypes.data_as(C.c_void_p)
 
 
-def _dev_ptr(t, dtype=None, what: str = "tensor"):
+def _device_of(ctx):
+    """Index of the device a context (or None: any device) lives on."""
+    return None if ctx is None else getattr(ctx, "device", None)
+
+
+def _dev_ptr(t, dtype=None, what: str = "tensor", device=None):
     """Raw device pointer of a torch CUDA tensor (None passes through)."""
     if t is None:
         return None
@@ -144,7 +149,32 @@ def _dev_ptr(t, dtype=None, what: str = "tensor"):
         raise TypeError(f"{what} must be a CUDA tensor")
     if dtype is not None and t.dtype not in (dtype if isinstance(dtype, tuple) else (dtype,)):
         raise TypeError(f"{what} has dtype {t.dtype}")
+    if device is not None and t.device.index != device:
+        raise ValueError(f"{what} lives on cuda:{t.device.index}, the context on cuda:{device}")
     return C.c_void_p(t.data_ptr())
+
+
+def _vec(t, n: int, dtype, what: str, device=None):
+    """Pointer of a contiguous 1-D device array that holds at least ``n`` elements: the kernels
+    index these arrays by row number without any further check."""
+    if t is None:
+        return None
+    p = _dev_ptr(t, dtype, what, device)
+    if t.dim() != 1 or not t.is_contiguous():
+        raise ValueError(f"{what} must be a contiguous 1-D tensor")
+    if t.numel() < n:
+        raise ValueError(f"{what} holds {t.numel()} elements, the batch has {n} rows")
+    return p
+
+
+def _mat(t, rows: int, cols: int, dtype, what: str, device=None):
+    """(pointer, row stride) of a 2-D device array with unit inner stride that holds at least
+    ``rows`` rows of ``cols`` elements."""
+    p = _dev_ptr(t, dtype, what, device)
+    _, stride = _rows(t, what)
+    if t.shape[0] < rows or t.shape[1] < cols:
+        raise ValueError(f"{what} is {tuple(t.shape)}, at least ({rows}, {cols}) is needed")
+    return p, stride
 
 
 def _stream_ptr(stream):
@@ -171,6 +201,8 @@ class Vocab:
         _check(_lib.wg_load_vocab(_np_ptr(self._offsets), _np_ptr(self._data), self.V, self.eos_id,
                                   C.byref(h)), "wg_load_vocab")
         self.handle = h
+        import torch
+        self.device = torch.cuda.current_device()     # wg_load_vocab uploads to the current device
 
     def close(self):
         if getattr(self, "handle", None) and _lib is not None:
@@ -340,6 +372,7 @@ class Context:
                  cache_mode: int = WG_CACHE_DENSE, arena_bytes: int = 0):
         self.vocab = vocab
         self.max_batch = int(max_batch)
+        self.device = vocab.device
         h = _vp()
         if cache_mode == WG_CACHE_DENSE and not arena_bytes:
             _check(_lib.wg_ctx_create(vocab.handle, int(cache_capacity), int(max_batch),
@@ -419,32 +452,44 @@ def _rows(t, what: str):
 
 def wg_mask_cache_lookup(ctx: Context, gid, sid, slot, stream=None) -> None:
     import torch
-    B = gid.shape[0]
-    _check(_lib.wg_mask_cache_lookup(ctx.handle, _dev_ptr(gid, torch.int32, "gid"),
-                                     _dev_ptr(sid, torch.int32, "sid"), B,
-                                     _dev_ptr(slot, torch.int32, "slot"), _stream_ptr(stream)),
+    B, dev = gid.shape[0], _device_of(ctx)
+    _check(_lib.wg_mask_cache_lookup(ctx.handle, _vec(gid, B, torch.int32, "gid", dev),
+                                     _vec(sid, B, torch.int32, "sid", dev), B,
+                                     _vec(slot, B, torch.int32, "slot", dev), _stream_ptr(stream)),
            "wg_mask_cache_lookup")
 
 
 def wg_build_masks(ctx: Context, gid, sid, bitmask, flags: int = WG_USE_CACHE, stream=None) -> None:
     import torch
-    B, stride = _rows(bitmask, "bitmask")
-    _check(_lib.wg_build_masks(ctx.handle, _dev_ptr(gid, torch.int32, "gid"),
-                               _dev_ptr(sid, torch.int32, "sid"), B,
-                               _dev_ptr(bitmask, (torch.int32, torch.uint32), "bitmask"), stride,
+    B, dev = bitmask.shape[0], _device_of(ctx)
+    mask, stride = _mat(bitmask, B, ctx.vocab.W, (torch.int32, torch.uint32), "bitmask", dev)
+    _check(_lib.wg_build_masks(ctx.handle, _vec(gid, B, torch.int32, "gid", dev),
+                               _vec(sid, B, torch.int32, "sid", dev), B, mask, stride,
                                int(flags), _stream_ptr(stream)), "wg_build_masks")
 
 
-def wg_apply_mask(logits, bitmask, V: int, argmax_out=None, workspace=None, stream=None) -> None:
+def _apply_args(logits, bitmask, V: int, argmax_out):
+    """Checked (logits pointer, dtype, stride, mask pointer, mask stride, B, token pointer)."""
     import torch
-    B, stride = _rows(logits, "logits")
-    Bm, mstride = _rows(bitmask, "bitmask")
-    if Bm != B:
-        raise ValueError("logits and bitmask disagree on the batch size")
-    _check(_lib.wg_apply_mask(_dev_ptr(logits, None, "logits"), _logits_dtype(logits), stride,
-                              _dev_ptr(bitmask, (torch.int32, torch.uint32), "bitmask"), mstride,
-                              B, int(V), _dev_ptr(argmax_out, torch.int32, "argmax_out"),
-                              _dev_ptr(workspace, None, "workspace"), _stream_ptr(stream)),
+    if logits.dim() != 2:
+        raise ValueError("logits must be 2-D with unit inner stride")
+    B, V = logits.shape[0], int(V)
+    dev = logits.device.index if logits.is_cuda else None
+    lp, stride = _mat(logits, B, V, None, "logits", dev)
+    mp, mstride = _mat(bitmask, B, (V + 31) // 32, (torch.int32, torch.uint32), "bitmask", dev)
+    return lp, _logits_dtype(logits), stride, mp, mstride, B, V, \
+        _vec(argmax_out, B, torch.int32, "argmax_out", dev), dev
+
+
+def wg_apply_mask(logits, bitmask, V: int, argmax_out=None, workspace=None, stream=None) -> None:
+    lp, dtype, stride, mp, mstride, B, V, tok, dev = _apply_args(logits, bitmask, V, argmax_out)
+    ws = _dev_ptr(workspace, None, "workspace", dev)
+    if argmax_out is not None:
+        need = wg_apply_workspace_bytes(B)
+        if workspace is None or not workspace.is_contiguous() or \
+                workspace.numel() * workspace.element_size() < need:
+            raise ValueError(f"workspace must be a contiguous device buffer of {need} bytes")
+    _check(_lib.wg_apply_mask(lp, dtype, stride, mp, mstride, B, V, tok, ws, _stream_ptr(stream)),
            "wg_apply_mask")
 
 
@@ -458,16 +503,10 @@ def wg_apply_mask_noalloc(logits, bitmask, V: int, argmax_out, stream=None) -> N
     inside the library, so at most ``WG_NOALLOC_MAX_ROWS`` rows per call, and calls that can
     overlap on the GPU must not be issued (they share that array).
     """
-    import torch
-    B, stride = _rows(logits, "logits")
-    Bm, mstride = _rows(bitmask, "bitmask")
-    if Bm != B:
-        raise ValueError("logits and bitmask disagree on the batch size")
-    _check(_lib.wg_apply_mask_noalloc(_dev_ptr(logits, None, "logits"), _logits_dtype(logits),
-                                      stride,
-                                      _dev_ptr(bitmask, (torch.int32, torch.uint32), "bitmask"),
-                                      mstride, B, int(V),
-                                      _dev_ptr(argmax_out, torch.int32, "argmax_out"),
+    if argmax_out is None:
+        raise ValueError("argmax_out is required")
+    lp, dtype, stride, mp, mstride, B, V, tok, _ = _apply_args(logits, bitmask, V, argmax_out)
+    _check(_lib.wg_apply_mask_noalloc(lp, dtype, stride, mp, mstride, B, V, tok,
                                       _stream_ptr(stream)), "wg_apply_mask_noalloc")
 
 
@@ -477,25 +516,36 @@ def wg_apply_workspace_bytes(B: int) -> int:
 
 def wg_advance(ctx: Context, gid, sid, token, status=None, flags: int = 0, stream=None) -> None:
     import torch
-    B = gid.shape[0]
-    _check(_lib.wg_advance(ctx.handle, _dev_ptr(gid, torch.int32, "gid"),
-                           _dev_ptr(sid, torch.int32, "sid"), _dev_ptr(token, torch.int32, "token"),
-                           B, _dev_ptr(status, torch.int32, "status"), int(flags),
+    B, dev = gid.shape[0], _device_of(ctx)
+    _check(_lib.wg_advance(ctx.handle, _vec(gid, B, torch.int32, "gid", dev),
+                           _vec(sid, B, torch.int32, "sid", dev),
+                           _vec(token, B, torch.int32, "token", dev), B,
+                           _vec(status, B, torch.int32, "status", dev), int(flags),
                            _stream_ptr(stream)), "wg_advance")
+
+
+def _step_args(ctx: Context, gid, sid, logits, n_cols: int, bitmask, token_out, status):
+    """The checked arrays of one decode step over ``logits.shape[0]`` rows."""
+    import torch
+    if logits.dim() != 2:
+        raise ValueError("logits must be 2-D with unit inner stride")
+    B, dev = logits.shape[0], _device_of(ctx)
+    lp, stride = _mat(logits, B, n_cols, None, "logits", dev)
+    mp, mstride = _mat(bitmask, B, ctx.vocab.W, (torch.int32, torch.uint32), "bitmask", dev)
+    return (_vec(gid, B, torch.int32, "gid", dev), _vec(sid, B, torch.int32, "sid", dev), B, lp,
+            _logits_dtype(logits), stride, mp, mstride,
+            _vec(token_out, B, torch.int32, "token_out", dev),
+            _vec(status, B, torch.int32, "status", dev))
 
 
 def wg_decode_step(ctx: Context, gid, sid, logits, bitmask, token_out, status=None,
                    flags: int = WG_USE_CACHE, stream=None) -> None:
-    import torch
-    B, stride = _rows(logits, "logits")
-    _, mstride = _rows(bitmask, "bitmask")
-    _check(_lib.wg_decode_step(ctx.handle, _dev_ptr(gid, torch.int32, "gid"),
-                               _dev_ptr(sid, torch.int32, "sid"), B,
-                               _dev_ptr(logits, None, "logits"), _logits_dtype(logits), stride,
-                               _dev_ptr(bitmask, (torch.int32, torch.uint32), "bitmask"), mstride,
-                               _dev_ptr(token_out, torch.int32, "token_out"),
-                               _dev_ptr(status, torch.int32, "status"), int(flags),
-                               _stream_ptr(stream)), "wg_decode_step")
+    g, s, B, lp, dtype, stride, mp, mstride, tok, st = _step_args(
+        ctx, gid, sid, logits, ctx.vocab.V, bitmask, token_out, status)
+    if tok is None:
+        raise ValueError("token_out is required")
+    _check(_lib.wg_decode_step(ctx.handle, g, s, B, lp, dtype, stride, mp, mstride, tok, st,
+                               int(flags), _stream_ptr(stream)), "wg_decode_step")
 
 
 WG_SHARD_ALIGN = 8192
@@ -506,25 +556,23 @@ def wg_decode_step_shard(ctx: Context, gid, sid, logits_shard, bitmask, v_begin:
     """The decode step on the vocabulary slice [v_begin, v_end); ``best_keys`` (int64, B) gets
     the packed per-row maxima to be MAX-reduced over the GPUs that hold the other slices."""
     import torch
-    B, stride = _rows(logits_shard, "logits_shard")
-    _, mstride = _rows(bitmask, "bitmask")
+    g, s, B, lp, dtype, stride, mp, mstride, _, _ = _step_args(
+        ctx, gid, sid, logits_shard, max(int(v_end) - int(v_begin), 0), bitmask, None, None)
     _check(_lib.wg_decode_step_shard(
-        ctx.handle, _dev_ptr(gid, torch.int32, "gid"), _dev_ptr(sid, torch.int32, "sid"), B,
-        _dev_ptr(logits_shard, None, "logits_shard"), _logits_dtype(logits_shard), stride,
-        _dev_ptr(bitmask, (torch.int32, torch.uint32), "bitmask"), mstride, int(v_begin), int(v_end),
-        _dev_ptr(best_keys, torch.int64, "best_keys"), int(flags), _stream_ptr(stream)),
-        "wg_decode_step_shard")
+        ctx.handle, g, s, B, lp, dtype, stride, mp, mstride, int(v_begin), int(v_end),
+        _vec(best_keys, B, torch.int64, "best_keys", _device_of(ctx)), int(flags),
+        _stream_ptr(stream)), "wg_decode_step_shard")
 
 
 def wg_advance_keys(ctx: Context, gid, sid, best_keys, token_out, status=None, flags: int = 0,
                     stream=None) -> None:
     import torch
-    B = gid.shape[0]
-    _check(_lib.wg_advance_keys(ctx.handle, _dev_ptr(gid, torch.int32, "gid"),
-                                _dev_ptr(sid, torch.int32, "sid"),
-                                _dev_ptr(best_keys, torch.int64, "best_keys"), B,
-                                _dev_ptr(token_out, torch.int32, "token_out"),
-                                _dev_ptr(status, torch.int32, "status"), int(flags),
+    B, dev = gid.shape[0], _device_of(ctx)
+    _check(_lib.wg_advance_keys(ctx.handle, _vec(gid, B, torch.int32, "gid", dev),
+                                _vec(sid, B, torch.int32, "sid", dev),
+                                _vec(best_keys, B, torch.int64, "best_keys", dev), B,
+                                _vec(token_out, B, torch.int32, "token_out", dev),
+                                _vec(status, B, torch.int32, "status", dev), int(flags),
                                 _stream_ptr(stream)), "wg_advance_keys")
 
 
@@ -540,24 +588,28 @@ class StepPlan:
                  flags: int = WG_USE_CACHE, stream=None):
         import torch
         self._keep = (ctx, gid, sid, bitmask, token_out, status)
-        self.B, self._mstride = _rows(bitmask, "bitmask")
+        self.B, dev = bitmask.shape[0], _device_of(ctx)
         if gid.shape[0] != self.B or sid.shape[0] != self.B or token_out.shape[0] != self.B:
             raise ValueError("gid, sid, token_out and bitmask disagree on the batch size")
         self._ctx = ctx.handle
-        self._gid = _dev_ptr(gid, torch.int32, "gid")
-        self._sid = _dev_ptr(sid, torch.int32, "sid")
-        self._mask = _dev_ptr(bitmask, (torch.int32, torch.uint32), "bitmask")
-        self._tok = _dev_ptr(token_out, torch.int32, "token_out")
-        self._status = _dev_ptr(status, torch.int32, "status")
+        self._V, self._device = ctx.vocab.V, dev
+        self._gid = _vec(gid, self.B, torch.int32, "gid", dev)
+        self._sid = _vec(sid, self.B, torch.int32, "sid", dev)
+        self._mask, self._mstride = _mat(bitmask, self.B, ctx.vocab.W, (torch.int32, torch.uint32),
+                                         "bitmask", dev)
+        self._tok = _vec(token_out, self.B, torch.int32, "token_out", dev)
+        self._status = _vec(status, self.B, torch.int32, "status", dev)
         self._flags = int(flags)
         self._stream = _stream_ptr(stream)
         self._dtypes = {torch.bfloat16: WG_DTYPE_BF16, torch.float32: WG_DTYPE_FP32}
         self._fn = _lib.wg_decode_step
 
     def __call__(self, logits) -> None:
-        if logits.dim() != 2 or logits.shape[0] != self.B or logits.stride(1) != 1 \
-                or not logits.is_cuda:
-            raise ValueError("logits must be a CUDA tensor [B, V] with unit inner stride")
+        if logits.dim() != 2 or logits.shape[0] != self.B or logits.shape[1] < self._V \
+                or logits.stride(1) != 1 or not logits.is_cuda \
+                or (self._device is not None and logits.device.index != self._device):
+            raise ValueError("logits must be a tensor [B, V] with unit inner stride on the "
+                             "context's device")
         rc = self._fn(self._ctx, self._gid, self._sid, self.B, logits.data_ptr(),
                       self._dtypes[logits.dtype], logits.stride(0), self._mask, self._mstride,
                       self._tok, self._status, self._flags, self._stream)
@@ -570,17 +622,14 @@ class StepGraph:
 
     def __init__(self, ctx: Context, gid, sid, logits, bitmask, token_out, status=None,
                  flags: int = WG_USE_CACHE):
-        import torch
         self._keep = (ctx, gid, sid, logits, bitmask, token_out, status)
-        B, stride = _rows(logits, "logits")
-        _, mstride = _rows(bitmask, "bitmask")
+        g, s, B, lp, dtype, stride, mp, mstride, tok, st = _step_args(
+            ctx, gid, sid, logits, ctx.vocab.V, bitmask, token_out, status)
+        if tok is None:
+            raise ValueError("token_out is required")
         h = _vp()
-        _check(_lib.wg_step_graph_create(
-            ctx.handle, _dev_ptr(gid, torch.int32, "gid"), _dev_ptr(sid, torch.int32, "sid"), B,
-            _dev_ptr(logits, None, "logits"), _logits_dtype(logits), stride,
-            _dev_ptr(bitmask, (torch.int32, torch.uint32), "bitmask"), mstride,
-            _dev_ptr(token_out, torch.int32, "token_out"), _dev_ptr(status, torch.int32, "status"),
-            int(flags), C.byref(h)), "wg_step_graph_create")
+        _check(_lib.wg_step_graph_create(ctx.handle, g, s, B, lp, dtype, stride, mp, mstride, tok, st,
+                                         int(flags), C.byref(h)), "wg_step_graph_create")
         self.handle = h
         self._launch = _lib.wg_step_graph_launch
 
@@ -601,16 +650,19 @@ class StepGraph:
 def wg_decode_step_host(ctx: Context, gid, sid, logits_host, logits_dev, bitmask, token_dev,
                         token_host, status=None, flags: int = WG_USE_CACHE, stream=None) -> None:
     """logits_host / token_host are CPU tensors (pinned for asynchronous copies)."""
-    import torch
-    B, stride = _rows(logits_dev, "logits_dev")
-    _, mstride = _rows(bitmask, "bitmask")
-    if logits_host.is_cuda or token_host.is_cuda or not logits_host.is_contiguous():
+    g, s, B, lp, dtype, stride, mp, mstride, tok, st = _step_args(
+        ctx, gid, sid, logits_dev, ctx.vocab.V, bitmask, token_dev, status)
+    if tok is None:
+        raise ValueError("token_dev is required")
+    if logits_host.is_cuda or token_host.is_cuda or not logits_host.is_contiguous() \
+            or not token_host.is_contiguous():
         raise TypeError("logits_host and token_host must be contiguous CPU tensors")
+    if logits_host.dim() != 2 or logits_host.shape[0] < B or logits_host.shape[1] != ctx.vocab.V \
+            or logits_host.dtype != logits_dev.dtype:
+        raise ValueError("logits_host must hold B rows of V elements of the device dtype")
+    if token_host.numel() < B or token_host.element_size() != 4:
+        raise ValueError("token_host must hold B 32-bit integers")
     _check(_lib.wg_decode_step_host(
-        ctx.handle, _dev_ptr(gid, torch.int32, "gid"), _dev_ptr(sid, torch.int32, "sid"), B,
-        C.c_void_p(logits_host.data_ptr()), _dev_ptr(logits_dev, None, "logits_dev"),
-        _logits_dtype(logits_dev), stride,
-        _dev_ptr(bitmask, (torch.int32, torch.uint32), "bitmask"), mstride,
-        _dev_ptr(token_dev, torch.int32, "token_dev"), C.c_void_p(token_host.data_ptr()),
-        _dev_ptr(status, torch.int32, "status"), int(flags), _stream_ptr(stream)),
+        ctx.handle, g, s, B, C.c_void_p(logits_host.data_ptr()), lp, dtype, stride, mp, mstride,
+        tok, C.c_void_p(token_host.data_ptr()), st, int(flags), _stream_ptr(stream)),
         "wg_decode_step_host")

@@ -91,6 +91,17 @@ struct GrammarSlot {
     std::vector<int32_t> forced_tok, forced_next;
     int32_t n_states, n_classes;
     void *d_table, *d_cls, *d_first_ok, *d_leaves, *d_forced, *d_leave1, *d_leave_fold;
+    // the rest of what makes two grammars the same: equal tables over different class maps
+    // (Write("a") and Write("b")) are different grammars
+    uint8_t byte_class[256];
+    int32_t start, done, eos_class;
+
+    bool same_as(const wg_grammar &g) const {
+        return hash == g.hash && n_states == g.n_states && n_classes == g.n_classes &&
+               start == g.start && done == g.done && eos_class == g.eos_class &&
+               memcmp(byte_class, g.byte_class, 256) == 0 && table == g.table &&
+               forced_tok == g.forced_tok && forced_next == g.forced_next;
+    }
 };
 
 struct ClassMappedRecords {
@@ -415,6 +426,8 @@ int32_t wg_grammar_load(const void *blob, size_t size, wg_grammar **out) {
     } catch (const std::bad_alloc &) {
         ok = false;
     }
+    // the stored hash must be the hash of what was stored: grammars are told apart by it
+    if (ok && wg_grammar_content_hash(*g) != h.hash) ok = false;
     if (!ok) {
         delete g;
         return WG_ERR_ARG;
@@ -460,7 +473,8 @@ int32_t wg_ctx_create_ex(const wg_vocab *vocab, int32_t cache_capacity, int32_t 
                          int32_t cache_mode, size_t arena_bytes, wg_ctx **out) {
     if (!out) return WG_ERR_ARG;
     *out = nullptr;
-    if (!vocab || cache_capacity < 0 || max_batch <= 0 || cache_capacity > (1 << 28))
+    if (!vocab || cache_capacity < 0 || max_batch <= 0 || max_batch > WG_MAX_ROWS ||
+        cache_capacity > (1 << 28))
         return WG_ERR_ARG;
     if (cache_mode != WG_CACHE_DENSE && cache_mode != WG_CACHE_COMPACT) return WG_ERR_ARG;
     const bool compact = cache_mode == WG_CACHE_COMPACT && cache_capacity > 0;
@@ -570,9 +584,7 @@ int32_t wg_ctx_add_grammar(wg_ctx *c, const wg_grammar *g, int32_t *grammar_id) 
     if (!c || !g || !grammar_id) return WG_ERR_ARG;
     std::lock_guard<std::mutex> lock(c->mu);
     for (size_t i = 0; i < c->slots.size(); ++i) {
-        const GrammarSlot &s = c->slots[i];
-        if (s.hash == g->hash && s.n_states == g->n_states && s.n_classes == g->n_classes &&
-            s.table == g->table && s.forced_tok == g->forced_tok && s.forced_next == g->forced_next) {
+        if (c->slots[i].same_as(*g)) {
             *grammar_id = (int32_t)i;
             return WG_OK;
         }
@@ -582,7 +594,9 @@ int32_t wg_ctx_add_grammar(wg_ctx *c, const wg_grammar *g, int32_t *grammar_id) 
     if ((uint64_t)g->n_states * (uint64_t)g->n_classes >= (1ull << 32)) return WG_ERR_CAPACITY;
     const bool wide = g->n_states > 65535;
     GrammarSlot slot{g->hash, g->table, g->forced_tok, g->forced_next, g->n_states, g->n_classes,
-                     nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
+                     nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr,
+                     {}, g->start, g->done, g->eos_class};
+    memcpy(slot.byte_class, g->byte_class, 256);
     struct Guard {  // frees the uploads again if any later step fails
         GrammarSlot *s;
         ~Guard() {
@@ -899,7 +913,7 @@ int32_t wg_apply_mask(void *logits, int32_t dtype, int64_t row_stride_elems,
                       const uint32_t *bitmask, int64_t mask_stride_words, int32_t B, int32_t V,
                       int32_t *argmax_out, void *workspace, void *stream) {
     NvtxRange nvtx_range("wg_apply_mask");
-    if (!logits || !bitmask || B < 1 || V < 1) return WG_ERR_ARG;
+    if (!logits || !bitmask || B < 1 || B > WG_MAX_ROWS || V < 1) return WG_ERR_ARG;
     if (dtype != WG_DTYPE_BF16 && dtype != WG_DTYPE_FP32) return WG_ERR_ARG;
     const int W = (V + 31) / 32;
     if (row_stride_elems < V || mask_stride_words < W) return WG_ERR_ARG;
@@ -1287,10 +1301,13 @@ int32_t wg_cache_prewarm(wg_ctx *c, int32_t grammar_id, void *stream) {
         BuildWork work{c->dev.bl_gid, c->dev.bl_sid, c->dev.bl_dst, nullptr, 0, c->dev.bl_count, 0, 0, 0, 0};
         rc = launch_build(c, work, n, st);
         if (rc != WG_OK) return rc;
+        // a batch that found the pool (or the arena) full ends the prewarm: later batches would
+        // only be looked up and dropped
+        rc = wg_get_stats(c, &after, stream);
+        if (rc != WG_OK) return rc;
+        if (after.rows_uncached > before.rows_uncached) return WG_ERR_CAPACITY;
     }
-    rc = wg_get_stats(c, &after, stream);
-    if (rc != WG_OK) return rc;
-    return after.rows_uncached > before.rows_uncached ? WG_ERR_CAPACITY : WG_OK;
+    return WG_OK;
 }
 
 }  // extern "C"

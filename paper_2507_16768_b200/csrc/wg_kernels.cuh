@@ -629,7 +629,10 @@ cache_lookup_insert_kernel(CtxDev ctx, const int32_t *gid, const int32_t *sid, i
         const int g = gid[r], s = sid[r];
         int32_t entry = -1;
         bool inserted = false;
-        if (ctx.hash_size > 0 && g >= 0 && g < ctx.n_grammars) {
+        // a state id that the grammar does not have (or DEAD) gets no cache entry: the row is
+        // built uncached, as a row of zeros, and counted as a bad state on every step
+        if (ctx.hash_size > 0 && g >= 0 && g < ctx.n_grammars && s > 0 &&
+            s < ctx.grammars[g].n_states) {
             const unsigned long long key = cache_key(g, s);
             uint32_t h = cache_hash(key) & mask;
             for (int probe = 0; probe < ctx.hash_size; ++probe, h = (h + 1) & mask) {
@@ -673,7 +676,6 @@ cache_lookup_insert_kernel(CtxDev ctx, const int32_t *gid, const int32_t *sid, i
     for (int r = threadIdx.x; r < B; r += blockDim.x) {
         const int32_t e = ctx.ent[r];
         int32_t row = e >= 0 ? ctx.vals[e & ~ENT_NEW] : -1;
-        // a state whose entry found no room in the arena is rebuilt on every step
         // a state whose entry found no room in the arena is rebuilt on every step (a row
         // inserted by this very call still has the flag clear here)
         if (ctx.compact && row >= 0 && ctx.ent_fail[row]) row = -1;

@@ -26,6 +26,28 @@ def mentioned_symbols(flat) -> List[int]:
     return sorted(syms)
 
 
+def symbol_representatives(flat) -> List[int]:
+    """One symbol of every group of symbols that the tree cannot tell apart.
+
+    Two symbols are told apart when some set of the tree holds one and not the other, or when
+    one of them is a byte of a literal.  This is a property of the input arrays alone."""
+    member = np.zeros((flat.sets.shape[0] + 1, 257), np.uint8)
+    for s in range(257):
+        member[:-1, s] = (flat.sets[:, s >> 5] >> np.uint32(s & 31)) & 1
+    member[-1, :] = 0
+    literal = np.unique(np.asarray(flat.data, np.uint8))
+    seen, reps = set(), []
+    sig = np.packbits(member, axis=0)
+    in_literal = np.zeros(257, bool)
+    in_literal[literal] = True
+    for s in range(257):
+        key = (bytes(sig[:, s]), s if (in_literal[s] or s == EOS) else -1)   # end-of-sequence stands alone
+        if key not in seen:
+            seen.add(key)
+            reps.append(s)
+    return reps
+
+
 def co_reachable(tree: oracle.Tree, grammar, symbols: Iterable[int], max_states: int = 10 ** 9
                  ) -> Dict[int, Tuple[int, int]]:
     """Breadth-first walk of both automata with the same symbols.
@@ -59,3 +81,30 @@ def co_reachable(tree: oracle.Tree, grammar, symbols: Iterable[int], max_states:
 
 def token_symbols(vocab, t: int) -> List[int]:
     return [EOS] if t == vocab.eos_id else list(vocab.token(t))
+
+
+def random_walk_states(tree: oracle.Tree, grammar, symbols: Iterable[int], rng, n_walks: int,
+                       max_steps: int) -> Dict[int, Tuple[int, int]]:
+    """States met on random walks of both automata from the start (for grammars too large to
+    enumerate).  At each step one of the symbols that keeps both sides alive is taken, so a walk
+    runs deep into the grammar; a finished walk starts again.  Returns {library state: cursor}."""
+    symbols = list(symbols)
+    cursor_of = {grammar.start_state: tree.start()}
+    for _ in range(n_walks):
+        cur, sid = tree.start(), grammar.start_state
+        for _ in range(max_steps):
+            live = []
+            for s in symbols:
+                nsid = grammar.step(sid, s)
+                if nsid != 0:
+                    live.append((s, nsid))
+            if not live:
+                break
+            s, nsid = live[int(rng.integers(0, len(live)))]
+            cur = tree.step(cur, s)
+            assert not oracle.is_dead(cur), (sid, s)
+            if cur == oracle.DONE:
+                break
+            sid = nsid
+            cursor_of.setdefault(sid, cur)
+    return cursor_of

@@ -226,6 +226,18 @@ def test_saved_grammar_loads_back_identical_and_damage_is_refused(wg):
         bad[off:off + 4] = (g.n_states + 5).to_bytes(4, "little")
         with pytest.raises(wg.WgError):
             wg.Grammar.load(bytes(bad))
+        # damage that keeps every field in range is caught by the content hash: a stored hash
+        # that is not the hash of the contents, and a changed symbol-class map (the header is 48
+        # bytes with the hash in its last 8; the class map follows)
+        wrong_hash = bytearray(blob)
+        wrong_hash[40] ^= 1
+        swapped = bytearray(blob)
+        swapped[48 + ord("a")], swapped[48 + ord("b")] = swapped[48 + ord("b")], swapped[48 + ord("a")]
+        assert bytes(swapped) != blob
+        for damaged in (wrong_hash, swapped):
+            with pytest.raises(wg.WgError) as e:
+                wg.Grammar.load(bytes(damaged))
+            assert e.value.status == wg.binding.WG_ERR_ARG
 
 
 def test_random_trees_lower_to_tables_that_match_the_checker(wg):

@@ -55,7 +55,7 @@ def odd_vocab():
              b'{"topic": 12, "paths": ["1/2', b"q" * 300, b"", b"</h1>\n<p class=\"document-abs",
              # a slot's closing byte as the last byte of the 16-byte record, and one byte before it
              b"a" * 15 + b"</h1>\n", b"a" * 14 + b"</", b"a" * 15 + b"<", b"b" * 16 + b"</p>"]
-    return vocab_from_tokens(toks + extra + toks[300:311][::-1][:0], eos_id=2)
+    return vocab_from_tokens(toks + extra, eos_id=2)
 
 
 SMALL = {
@@ -163,7 +163,7 @@ class Sim:
 
     def __init__(self, wg, torch, vocab, ops, row_grammar, dtype, cache_capacity, use_cache=True,
                  seed=0, steer=6.0, delays=None, minimize=False, cache_mode=0, arena_bytes=0,
-                 grams=None):
+                 grams=None, starts=None):
         self.wg, self.torch, self.vocab, self.dtype = wg, torch, vocab, dtype
         self.flats = [op if hasattr(op, "nodes") else flatten(op) for op in ops]
         self.trees = [oracle.Tree(f) for f in self.flats]
@@ -190,6 +190,10 @@ class Sim:
         self.d_sid = to_dev(torch, np.array(
             [self.grams[g].done_state if late[r] else self.grams[g].start_state
              for r, g in enumerate(self.row_grammar)], np.int32))
+        if starts is not None:
+            # rows that begin in the middle of a run: (library state, checker cursor) per row
+            self.cursors = [c for _, c in starts]
+            self.d_sid = to_dev(torch, np.array([s for s, _ in starts], np.int32))
         self.h_sid = self.d_sid.cpu().numpy().copy()
         self.W = self.dv.W
         self.d_mask = torch.zeros((self.B, self.W), dtype=torch.int32, device="cuda")
@@ -202,13 +206,17 @@ class Sim:
         x = make_logits(self.B, self.vocab.size, self.dtype, [self.seed, self.B], self.step_no,
                         self.bonus, self.steer)
         if any(self.delays) and self.step_no > 0:
-            # a late row sees what the row before it saw one step earlier
-            prev = make_logits(self.B, self.vocab.size, self.dtype, [self.seed, self.B],
-                               self.step_no - 1, self.bonus, self.steer)
-            for r, d in enumerate(self.delays):
-                if d > 0:
-                    x[r] = prev[r - 1]
+            # a late row sees what the row before it saw one step earlier (kept on the device,
+            # untouched by any kernel: a copy of the previous step's inputs)
+            late = [r for r, d in enumerate(self.delays) if d > 0]
+            idx = self.torch.tensor([r - 1 for r in late], device="cuda")
+            bits = x.view(np.uint32) if self.dtype == "fp32" else x
+            bits[late] = raw_bits(self.torch, self._prev_inputs[idx])
         return x
+
+    def _remember_inputs(self, dl):
+        if any(self.delays):
+            self._prev_inputs = dl.clone()
 
     def step(self, check_rows=None, fused=True):
         wg, torch, vocab = self.wg, self.torch, self.vocab
@@ -216,13 +224,15 @@ class Sim:
         host = self.logits()
         # ---- checker: mask -> apply -> argmax -> advance on the checked rows
         trees = [self.trees[self.row_grammar[r]] for r in rows]
-        want_mask = oracle.masks(trees, vocab, [self.cursors[r] for r in rows], n_threads=8)
+        want_mask = oracle.masks(trees, vocab, [self.cursors[r] for r in rows],
+                                 n_threads=oracle.max_threads())
         sub = np.ascontiguousarray(host[list(rows)])
         want_tok = oracle.argmax(sub, want_mask, vocab.size)
         want_logits = sub.copy()
         oracle.apply_mask(want_logits, want_mask, vocab.size)
         # ---- library
         dl = dev_logits(torch, host, self.dtype)
+        self._remember_inputs(dl)
         if fused:
             wg.wg_decode_step(self.ctx, self.d_gid, self.d_sid, dl, self.d_mask, self.d_tok,
                               self.d_status, self.flags)
@@ -238,11 +248,14 @@ class Sim:
         got_sid = self.d_sid.cpu().numpy()
         status = self.d_status.cpu().numpy()
         raw_want = want_logits.view(np.uint32) if self.dtype == "fp32" else want_logits
-        for i, r in enumerate(rows):
-            assert (got_mask[r] == want_mask[i]).all(), (self.step_no, r)
-            assert got_tok[r] == want_tok[i], (self.step_no, r)
-            assert (got_logits[r] == raw_want[i]).all(), (self.step_no, r)
-            assert status[r] == 0
+        sel = list(rows)
+        if not ((got_mask[sel] == want_mask).all() and (got_tok[sel] == want_tok).all()
+                and (got_logits[sel] == raw_want).all() and (status[sel] == 0).all()):
+            for i, r in enumerate(rows):          # name the first row that differs
+                assert (got_mask[r] == want_mask[i]).all(), (self.step_no, r)
+                assert got_tok[r] == want_tok[i], (self.step_no, r)
+                assert (got_logits[r] == raw_want[i]).all(), (self.step_no, r)
+                assert status[r] == 0
         # ---- advance the checker with the LIBRARY's tokens on every row (checked rows were
         # just shown to agree); unchecked rows are verified through the state mapping below
         for r in range(self.B):
@@ -257,6 +270,49 @@ class Sim:
             self.cursors[r] = cur
             assert got_sid[r] == host_sid, (self.step_no, r)
             self.visited.add((gi, host_sid))
+        self.h_sid = got_sid.copy()
+        self.step_no += 1
+
+    def step_unchecked(self):
+        """A step whose masks and logits are NOT compared: the logits are drawn on the device
+        (seeded by the step number), so a long run between compared steps costs no host
+        generation.  Every row is still checked through what is cheap: the library's token must
+        be accepted by the checker in the row's cursor, and the device state must equal the host
+        table walk of that token."""
+        wg, torch, vocab = self.wg, self.torch, self.vocab
+        if not hasattr(self, "_memo"):
+            self._memo = {}
+            self._bonus_dev = torch.from_numpy(self.bonus.astype(np.float32)).cuda() * self.steer
+        gen = torch.Generator(device="cuda")
+        gen.manual_seed(977 * self.seed + self.step_no)
+        x = torch.randn((self.B, vocab.size), generator=gen, device="cuda") * 2.0
+        if self.steer:
+            x += self._bonus_dev
+        dl = x.to(torch.bfloat16) if self.dtype == "bf16" else x
+        if any(self.delays) and self.step_no > 0:
+            late = [r for r, d in enumerate(self.delays) if d > 0]
+            dl[late] = self._prev_inputs[torch.tensor([r - 1 for r in late], device="cuda")]
+        self._remember_inputs(dl)
+        wg.wg_decode_step(self.ctx, self.d_gid, self.d_sid, dl, self.d_mask, self.d_tok,
+                          self.d_status, self.flags)
+        got_tok = self.d_tok.cpu().numpy()
+        got_sid = self.d_sid.cpu().numpy()
+        assert (self.d_status == 0).all(), self.step_no
+        for r in range(self.B):
+            gi, t = self.row_grammar[r], int(got_tok[r])
+            key = (gi, self.cursors[r], int(self.h_sid[r]), t)
+            hit = self._memo.get(key)
+            if hit is None:
+                rc, cur = oracle.advance(self.trees[gi], vocab, self.cursors[r], t)
+                assert rc == 0, (self.step_no, r, t)
+                host_sid = self.grams[gi].step_token(int(self.h_sid[r]), t, token_symbols(vocab, t))
+                if cur == oracle.DONE:
+                    cur = self.trees[gi].start()
+                    host_sid = self.grams[gi].start_state
+                hit = self._memo[key] = (cur, host_sid)
+            self.cursors[r] = hit[0]
+            assert got_sid[r] == hit[1], (self.step_no, r)
+            self.visited.add((gi, hit[1]))
         self.h_sid = got_sid.copy()
         self.step_no += 1
 
