@@ -499,6 +499,17 @@ int32_t wg_decode_step_host(wg_ctx *ctx, const int32_t *gid, int32_t *sid, int32
 int32_t wg_ctx_set_timing(wg_ctx *ctx, int32_t enable);
 int32_t wg_ctx_get_timing(wg_ctx *ctx, double *build_ms, double *apply_ms, int64_t *steps);
 
+/* Work counters of the mask-build kernel, for the benchmark's bound on that kernel (paper
+ * Section 1: mask creation is one of the three cost stages; these say what one build costs).
+ * While enabled, wg_build_masks / wg_decode_step launch a variant of the build kernel that also
+ * counts, over all masks built: the tokens it could not decide 32 at a time and walked through
+ * the table, the table look-ups of those walks, and the words of vocabulary masks its word-wise
+ * phase read.  The variant is slower; timed runs keep it off.  wg_get_build_work reads the
+ * counters (since the last wg_reset_stats) and synchronises `stream`; any pointer may be NULL. */
+int32_t wg_ctx_count_build_work(wg_ctx *ctx, int32_t enable);
+int32_t wg_get_build_work(wg_ctx *ctx, int64_t *tokens_walked, int64_t *table_lookups,
+                          int64_t *mask_words_read, void *stream);
+
 const char *wg_strerror(int32_t status);
 /* cudaError_t of the last failed CUDA call on this thread (0 if none). */
 int32_t wg_last_cuda_error(void);

@@ -106,6 +106,8 @@ _SIGNATURES = {
     "wg_ctx_set_timing": (_i32, [_vp, _i32]),
     "wg_ctx_get_timing": (_i32, [_vp, C.POINTER(C.c_double), C.POINTER(C.c_double),
                                  C.POINTER(_i64)]),
+    "wg_ctx_count_build_work": (_i32, [_vp, _i32]),
+    "wg_get_build_work": (_i32, [_vp, C.POINTER(_i64), C.POINTER(_i64), C.POINTER(_i64), _vp]),
     "wg_strerror": (C.c_char_p, [_i32]),
     "wg_last_cuda_error": (_i32, []),
     "wg_kernel_launch_count": (_i64, []),
@@ -430,6 +432,17 @@ class Context:
         _check(_lib.wg_ctx_get_timing(self.handle, C.byref(b), C.byref(a), C.byref(n)),
                "wg_ctx_get_timing")
         return {"build_ms": b.value, "apply_ms": a.value, "steps": int(n.value)}
+
+    def count_build_work(self, enable: bool) -> None:
+        _check(_lib.wg_ctx_count_build_work(self.handle, int(bool(enable))),
+               "wg_ctx_count_build_work")
+
+    def build_work(self, stream=None) -> dict:
+        """Work counted by the build kernel's counting variant since the last reset_stats."""
+        q, l, m = _i64(), _i64(), _i64()
+        _check(_lib.wg_get_build_work(self.handle, C.byref(q), C.byref(l), C.byref(m),
+                                      _stream_ptr(stream)), "wg_get_build_work")
+        return {"tokens_walked": q.value, "table_lookups": l.value, "mask_words_read": m.value}
 
     def reset_stats(self, stream=None) -> None:
         _check(_lib.wg_reset_stats(self.handle, _stream_ptr(stream)), "wg_reset_stats")

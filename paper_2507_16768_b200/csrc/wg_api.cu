@@ -131,6 +131,7 @@ struct wg_ctx {
     int32_t *d_stage_gid = nullptr, *d_stage_sid = nullptr;  // prewarm staging
     std::vector<void *> owned;  // every other device allocation
     std::mutex mu;
+    bool count_build_work = false;  // launch the counting variant of the build kernel
     // optional per-kernel timing: events[4 * i + {0,1,2,3}] = build begin/end, apply begin/end
     bool timing = false;
     std::vector<cudaEvent_t> events;
@@ -793,9 +794,12 @@ int32_t launch_build(wg_ctx *c, const BuildWork &work, int max_entries, cudaStre
     long long items = (long long)max_entries * n_chunks;
     if (items >= (1LL << 31)) return WG_ERR_CAPACITY;  // the kernel numbers its items with 32 bits
     auto kernel = c->dev.compact ? build_masks_kernel<true> : build_masks_kernel<false>;
+    if (c->count_build_work)
+        kernel = c->dev.compact ? build_masks_kernel<true, true> : build_masks_kernel<false, true>;
     // One block per resident slot: the blocks stride over the items, so blocks that had to wait
     // for a slot would start their equal share late and stretch the launch.
-    int &per_sm = c->build_blocks_per_sm;
+    int uncached_per_sm = 0;  // the counting variant is asked every time (it is never timed)
+    int &per_sm = c->count_build_work ? uncached_per_sm : c->build_blocks_per_sm;
     if (per_sm == 0) {
         int n = 0;
         if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, BUILD_THREADS, 0) != cudaSuccess || n < 1)
@@ -1200,6 +1204,25 @@ int32_t wg_decode_step_host(wg_ctx *c, const int32_t *gid, int32_t *sid, int32_t
     WG_CUDA(cudaMemcpyAsync(token_host, token_dev, sizeof(int32_t) * (size_t)B,
                             cudaMemcpyDeviceToHost, st));
     WG_CUDA(cudaStreamSynchronize(st));
+    return WG_OK;
+}
+
+int32_t wg_ctx_count_build_work(wg_ctx *c, int32_t enable) {
+    if (!c) return WG_ERR_ARG;
+    c->count_build_work = enable != 0;
+    return WG_OK;
+}
+
+int32_t wg_get_build_work(wg_ctx *c, int64_t *tokens_walked, int64_t *table_lookups,
+                          int64_t *mask_words_read, void *stream) {
+    if (!c) return WG_ERR_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    unsigned long long h[ST_COUNT];
+    WG_CUDA(cudaMemcpyAsync(h, c->dev.stats, sizeof(h), cudaMemcpyDeviceToHost, st));
+    WG_CUDA(cudaStreamSynchronize(st));
+    if (tokens_walked) *tokens_walked = (int64_t)h[ST_QUEUED];
+    if (table_lookups) *table_lookups = (int64_t)h[ST_WALKED];
+    if (mask_words_read) *mask_words_read = (int64_t)h[ST_MASK_WORDS];
     return WG_OK;
 }
 

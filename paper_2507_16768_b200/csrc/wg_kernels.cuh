@@ -44,7 +44,12 @@ struct VocabDev {
 };
 
 enum StatSlot {
-    ST_HITS = 0, ST_MISSES, ST_BUILT, ST_UNCACHED, ST_REJECTED, ST_EMPTY, ST_BAD_STATE, ST_COUNT
+    ST_HITS = 0, ST_MISSES, ST_BUILT, ST_UNCACHED, ST_REJECTED, ST_EMPTY, ST_BAD_STATE,
+    // work counters of the build kernel, only kept by its counting variant (wg_ctx_count_build_work)
+    ST_QUEUED,      // tokens that were not decided word-wise and went through the table walk
+    ST_WALKED,      // table look-ups of those walks
+    ST_MASK_WORDS,  // words of vocabulary masks read by the word-wise phase
+    ST_COUNT
 };
 
 struct CtxDev {
@@ -109,7 +114,8 @@ __device__ __forceinline__ void pdl_enter();
 template <typename T>
 __device__ __forceinline__ uint32_t walk_token_classes(const VocabDev &v, const uint4 *rec_class,
                                                        const T *__restrict__ tab, int C,
-                                                       const uint8_t *cls, uint32_t s, int t) {
+                                                       const uint8_t *cls, uint32_t s, int t,
+                                                       int *lookups = nullptr) {
     const int n = v.len[t];
     if (n == 0) return 0;
     const uint4 rec = __ldg(&rec_class[t]);
@@ -121,10 +127,14 @@ __device__ __forceinline__ uint32_t walk_token_classes(const VocabDev &v, const 
     for (int j = 0; j < WG_REC_BYTES; ++j) {
         if (j >= n || s == 0) break;
         s = tab[s * Cu + ((w[j >> 2] >> (8 * (j & 3))) & 0xFFu)];
+        if (lookups) ++*lookups;
     }
     if (n > WG_REC_BYTES && s != 0) {
         const uint32_t b = v.offsets[t] + WG_REC_BYTES, e = v.offsets[t + 1];
-        for (uint32_t i = b; i < e && s != 0; ++i) s = tab[s * Cu + cls[v.bytes[i]]];
+        for (uint32_t i = b; i < e && s != 0; ++i) {
+            s = tab[s * Cu + cls[v.bytes[i]]];
+            if (lookups) ++*lookups;
+        }
     }
     return s;
 }
@@ -229,8 +239,10 @@ struct BuildWork {
 };
 
 // COMPACT: the cache keeps allows / denies entries; finished chunks are also stored as spans.
-template <bool COMPACT>
-__global__ void __launch_bounds__(BUILD_THREADS, COMPACT ? 5 : 8)
+// COUNT: the variant that also counts its work (queued tokens, table look-ups, vocabulary-mask
+// words read) for the benchmark's bound; never used for a timed launch.
+template <bool COMPACT, bool COUNT = false>
+__global__ void __launch_bounds__(BUILD_THREADS, (COMPACT || COUNT) ? 5 : 8)
 build_masks_kernel(VocabDev v, CtxDev ctx, BuildWork work) {
     // the facts about one work item's mask, gathered by warp 0 (two copies: the next item's are
     // gathered while the other warps walk the current item's tokens)
@@ -354,6 +366,7 @@ build_masks_kernel(VocabDev v, CtxDev ctx, BuildWork work) {
         // phase 1: one word of 32 tokens per thread
         const int n_words = (t_end - t_begin) >> 5;
         const int nf = n_first, nq = n_fold;
+        int counted_words = 0, counted_lookups = 0;
         for (int wl = threadIdx.x; wl < ((n_words + 31) & ~31); wl += BUILD_THREADS) {
             uint32_t alive = 0, queue = 0;
             const int w = (t_begin >> 5) + wl;
@@ -367,6 +380,7 @@ build_masks_kernel(VocabDev v, CtxDev ctx, BuildWork work) {
                 for (int i = 0; i < nq; ++i) q |= __ldg(&v.fold_mask[(size_t)fold_list[i] * v.W + w]);
                 alive = p & ~q;
                 queue = p & q;
+                if (COUNT) counted_words += nf + nq + (complement ? 1 : 0);
                 if (after_k >= 0 && queue != 0) {
                     const uint32_t *rows = ctx.after_masks + (size_t)after_k * AFTER_ROWS * v.W;
                     const uint32_t has = __ldg(&rows[w]);
@@ -377,11 +391,13 @@ build_masks_kernel(VocabDev v, CtxDev ctx, BuildWork work) {
                         alive |= queue & ~has;
                         queue &= has;
                     }
+                    if (COUNT) counted_words += 1;
                     if (queue & has) {
                         uint32_t worth = __ldg(&rows[(size_t)v.W + w]);
                         for (unsigned long long f = after_fold; f; f &= f - 1)
                             worth |= __ldg(&rows[(size_t)(2 + __ffsll((long long)f) - 1) * v.W + w]);
                         queue &= ~has | worth;
+                        if (COUNT) counted_words += 1 + __popcll(after_fold);
                     }
                 }
                 if ((v.eos_id >> 5) == w && eos_next != 0) alive |= 1u << (v.eos_id & 31);
@@ -418,13 +434,26 @@ build_masks_kernel(VocabDev v, CtxDev ctx, BuildWork work) {
         } else {
             for (int i = threadIdx.x - 32; i < n; i += BUILD_THREADS - 32) {
                 const int rel = todo[i];
+                int *const counter = COUNT ? &counted_lookups : nullptr;
                 const uint32_t end = info.wide
                     ? walk_token_classes<uint32_t>(v, info.rec_class, static_cast<const uint32_t *>(info.table),
-                                                   info.n_classes, cls, s0, t_begin + rel)
+                                                   info.n_classes, cls, s0, t_begin + rel, counter)
                     : walk_token_classes<uint16_t>(v, info.rec_class, static_cast<const uint16_t *>(info.table),
-                                                   info.n_classes, cls, s0, t_begin + rel);
+                                                   info.n_classes, cls, s0, t_begin + rel, counter);
                 if (end != 0) atomicOr(&words[rel >> 5], 1u << (rel & 31));
             }
+        }
+        if (COUNT) {
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                counted_words += __shfl_xor_sync(0xFFFFFFFFu, counted_words, o);
+                counted_lookups += __shfl_xor_sync(0xFFFFFFFFu, counted_lookups, o);
+            }
+            if (lane == 0) {
+                atomicAdd(&ctx.stats[ST_MASK_WORDS], (unsigned long long)counted_words);
+                atomicAdd(&ctx.stats[ST_WALKED], (unsigned long long)counted_lookups);
+            }
+            if (threadIdx.x == 32) atomicAdd(&ctx.stats[ST_QUEUED], (unsigned long long)n);
         }
         __syncthreads();
         if (threadIdx.x == 0) n_todo = 0;  // everybody has read it

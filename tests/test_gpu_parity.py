@@ -682,3 +682,39 @@ def test_masks_of_random_trees_on_a_dense_small_alphabet_vocabulary(wg, torch):
             assert (out.cpu().numpy().view(np.uint32) == want).all()
         n_states += len(sids)
     assert n_states > 150
+
+
+def test_bad_state_ids_take_no_cache_entry_and_are_counted_every_step(wg, torch):
+    vocab = make_vocab(4096, seed=4)
+    g = wg.Grammar(flatten(grammars.html_template()))
+    dv = wg.Vocab(vocab.offsets, vocab.data, vocab.eos_id)
+    ctx = wg.Context(dv, cache_capacity=64, max_batch=4)
+    gid = torch.full((3,), ctx.add_grammar(g), dtype=torch.int32, device="cuda")
+    sid = to_dev(torch, np.array([g.start_state, g.n_states + 3, -9], np.int32))
+    mask = torch.ones((3, dv.W), dtype=torch.int32, device="cuda")
+    tok = torch.zeros(3, dtype=torch.int32, device="cuda")
+    status = torch.zeros(3, dtype=torch.int32, device="cuda")
+    for step in range(2):
+        logits = torch.randn(3, vocab.size, device="cuda")
+        wg.wg_decode_step(ctx, gid, sid.clone(), logits, mask, tok, status)
+        assert (mask[1:] == 0).all() and tok.cpu().tolist()[1:] == [-1, -1]
+        assert status.cpu().tolist()[1:] == [wg.binding.WG_ERR_STATE] * 2
+    st = ctx.stats()
+    # two bad rows a step: counted when their zero masks are built and again by the advance
+    assert st["bad_states"] == 2 * 2 * 2 and st["cache_entries"] == 1
+    assert st["rows_uncached"] == 4 and st["cache_hits"] == 1
+
+
+def test_equal_tables_over_different_class_maps_are_different_grammars(wg, torch):
+    vocab = make_vocab(1024, seed=4)
+    dv = wg.Vocab(vocab.offsets, vocab.data, vocab.eos_id)
+    ctx = wg.Context(dv, 16, 2)
+    ga, gb = wg.Grammar(flatten(Write(b"a"))), wg.Grammar(flatten(Write(b"b")))
+    ida, idb = ctx.add_grammar(ga), ctx.add_grammar(gb)
+    assert ida != idb and ctx.add_grammar(wg.Grammar(flatten(Write(b"a")))) == ida
+    out = torch.zeros((2, dv.W), dtype=torch.int32, device="cuda")
+    wg.wg_build_masks(ctx, to_dev(torch, np.array([ida, idb], np.int32)),
+                      to_dev(torch, np.array([ga.start_state, gb.start_state], np.int32)), out)
+    bits = np.unpackbits(out.cpu().numpy().view(np.uint8), axis=1, bitorder="little")
+    assert np.flatnonzero(bits[0]).tolist() == [ord("a")]
+    assert np.flatnonzero(bits[1]).tolist() == [ord("b")]

@@ -50,6 +50,7 @@ _GRAMMARS: dict[str, Callable[[int], Op]] = {
     "json_lookup": lambda g: grammars.json_reference_lookup(),
     "cold_templates": lambda g: grammars.random_template(seed=g),
     "json_warm": lambda g: grammars.json_reference_lookup(),
+    "html_warm_free_text": lambda g: grammars.html_template(),
     "dynamic_snippets": lambda g: grammars.dynamic_snippet_template(seed=g),
 }
 
@@ -66,4 +67,13 @@ WORKLOADS: List[Workload] = [
              "large dynamic-snippet grammar: 64 instantiations shared by row pairs"),
 ]
 
-BY_NAME = {w.name: w for w in WORKLOADS}
+# Not one of the five configurations: the cache-warm steady state of workload 4 with every row
+# dwelling in a free-text slot (the HTML template on unsteered logits walks through its first tag
+# and then stays in the slot), so that nearly every token is allowed and the apply pass reads
+# every logit instead of overwriting it.  A diagnostic for the apply kernel's other extreme.
+EXTRA_WORKLOADS: List[Workload] = [
+    Workload("html_warm_free_text", 128256, 1024, 256, "bf16", 4, True, True, 1,
+             "cache-warm steady state with rows in free-text slots (mostly-allowed masks)"),
+]
+
+BY_NAME = {w.name: w for w in WORKLOADS + EXTRA_WORKLOADS}
