@@ -461,7 +461,7 @@ def test_host_argument_errors(wg, torch):
         wg.wg_build_masks(ctx, five, five, mask)
     assert e.value.status == wg.binding.WG_ERR_ARG
     narrow = torch.zeros((4, dv.W - 1), dtype=torch.int32, device="cuda")
-    with pytest.raises(wg.WgError):                                # rows shorter than W words
+    with pytest.raises(ValueError):                                # rows shorter than W words
         wg.wg_build_masks(ctx, five[:4], five[:4], narrow)
     with pytest.raises(wg.WgError):
         ctx.cache_prewarm(3)                                       # unknown grammar id

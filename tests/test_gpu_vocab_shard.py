@@ -112,12 +112,15 @@ def test_more_ranks_than_slices_and_what_is_refused(wg, torch):
                            steps=12, steer=8.0)
     rk = next(r for r in ranks if r["e"] - r["b"] > 0 and r["b"] > 0)
     B = 2
-    x = torch.zeros((B, rk["e"] - rk["b"]), dtype=torch.float32, device="cuda")
+    x = torch.zeros((B, vocab.size), dtype=torch.float32, device="cuda")
     for b, e in ((0, 8192), (100, vocab.size), (8192, 9000)):
         with pytest.raises(wg.WgError) as err:      # another slice / unaligned begin / unaligned end
             wg.wg_decode_step_shard(rk["ctx"], rk["gid"], rk["sid"], x[:, :max(1, e - b)], rk["mask"],
                                     b, e, rk["keys"])
         assert err.value.status == wg.WG_ERR_ARG
+    with pytest.raises(ValueError):                  # fewer logits columns than the slice has tokens
+        wg.wg_decode_step_shard(rk["ctx"], rk["gid"], rk["sid"], x[:, :50], rk["mask"], rk["b"],
+                                rk["e"], rk["keys"])
     full = torch.zeros((B, vocab.size), dtype=torch.float32, device="cuda")
     with pytest.raises(wg.WgError):                  # the cache holds one slice's words only
         wg.wg_decode_step(rk["ctx"], rk["gid"], rk["sid"], full, rk["mask"], rk["tok"])
