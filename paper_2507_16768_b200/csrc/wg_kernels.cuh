@@ -273,6 +273,10 @@ build_masks_kernel(VocabDev v, CtxDev ctx, BuildWork work) {
     // (item numbers stay in 32 bits: the launch refuses more than 2^31 of them; the division by
     // the chunk count below would otherwise be a 64-bit one, a hundred instructions per item)
     const uint32_t n_items = (uint32_t)n_entries * (uint32_t)n_chunks;
+    // Nothing to build (every row of a warm step hit the cache): leave at once.  Nobody has
+    // touched the work counters, so they need no reset either -- and the launch is then a few
+    // hundred blocks that read one word and exit, on the critical path of every warm step.
+    if (n_items == 0) return;
 
     // Called by warp 0: the grammar record and the state's sets of item `it` into fx.
     auto gather = [&](uint32_t it, ItemFacts &fx) {
