@@ -44,7 +44,7 @@ def test_strerror_and_launch_counter(wg):
 
 
 GRAMMARS = {
-    "listing": grammars.paper_listing_example,
+    "dotted_number": grammars.dotted_number,
     "html": grammars.html_template,
     "json_generic": lambda: grammars.json_reference_lookup(doc_nodes=0),
     "json_doc": lambda: grammars.json_reference_lookup(doc_nodes=120),
@@ -176,7 +176,7 @@ def test_header_compiles_as_plain_c(tmp_path):
                            str(tmp_path / "use_wg.o")])
 
 
-@pytest.mark.parametrize("name", ["listing", "html", "json_doc", "template1", "snippets",
+@pytest.mark.parametrize("name", ["dotted_number", "html", "json_doc", "template1", "snippets",
                                   "html_tags", "overlapping_until", "empty_bodies"])
 def test_minimized_grammar_keeps_the_language(wg, name):
     flat = flatten(GRAMMARS[name]())

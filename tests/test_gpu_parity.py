@@ -64,7 +64,7 @@ SMALL = {
     "json_generic": lambda: grammars.json_reference_lookup(doc_nodes=0),
     "template2": lambda: grammars.random_template(2),
     "snippets": lambda: grammars.dynamic_snippet_template(4, n_args=3, enum_size=10),
-    "listing": grammars.paper_listing_example,
+    "dotted_number": grammars.dotted_number,
     "html_tags": lambda: grammars.html_template(wait_for_tag=True),
 }
 

@@ -36,10 +36,53 @@ def unpack(words, V):
 
 
 # ---------------------------------------------------------------------------------------
-# Section 3.2 listing: said to represent \d+(\.\d+)* followed by <eos>
+# Section 3.2, worked example: an operator tree said to represent \d+(\.\d+)* followed by <eos>
 # ---------------------------------------------------------------------------------------
-def test_paper_listing_language_exhaustive():
-    tree = tree_of(grammars.paper_listing_example())
+def worked_example_tree():
+    """The example's operator tree, read from its fixture (tests/golden)."""
+    import os
+    path = os.path.join(os.path.dirname(__file__), "golden", "section_3_2_worked_example_tree.txt")
+    text = " ".join(l for l in open(path).read().splitlines() if not l.startswith("#"))
+    tokens = text.replace("(", " ( ").replace(")", " ) ").split()
+    named = {"digits": SymSet(b"0123456789"), "dot": SymSet(b"."), "eos": SymSet([EOS])}
+
+    def symset(spec):
+        out = SymSet()
+        for name in spec.split("+"):
+            out = out | named[name]
+        return out
+
+    def parse(i):
+        assert tokens[i] == "("
+        kind, i = tokens[i + 1], i + 2
+        sets, kids = {}, []
+        while tokens[i] != ")":
+            if tokens[i] == "(":
+                kid, i = parse(i)
+                kids.append(kid)
+            else:
+                key, spec = tokens[i].split("=")
+                sets[key] = symset(spec)
+                i += 1
+        if kind == "none":
+            return None, i + 1
+        if kind == "sequence":
+            return Sequence(kids), i + 1
+        if kind == "wait":
+            return Wait(allow=sets["allow"], wait=sets["wait"]), i + 1
+        cond = Cond(allow=sets["allow"], true_waits=sets["true"], false_waits=sets["false"])
+        if kind == "ifelse":
+            return IfElse(condition=cond, if_body=kids[0], else_body=kids[1]), i + 1
+        assert kind == "dowhile"
+        return DoWhile(body=kids[0], condition=cond), i + 1
+
+    return parse(0)[0]
+
+
+@pytest.mark.parametrize("which", ["worked example", "dotted_number"])
+def test_paper_listing_language_exhaustive(which):
+    # the paper's own tree, and the tree the workloads build from the stated language
+    tree = tree_of(worked_example_tree() if which == "worked example" else grammars.dotted_number())
     hand = re.compile(rb"[0-9]+(\.[0-9]+)*\x02+")
     alphabet = [ord("0"), ord("7"), ord("."), ord("x"), EOS]
     n_accept = 0
@@ -68,7 +111,7 @@ def test_paper_listing_language_exhaustive():
 
 
 def test_paper_listing_keeps_digit_runs_and_needs_a_digit_after_the_dot():
-    tree = tree_of(grammars.paper_listing_example())
+    tree = tree_of(worked_example_tree())
     ok = lambda s: tree.accepts([ord(c) for c in s] + [EOS])  # noqa: E731
     assert ok("7") and ok("2025") and ok("3.14") and ok("10.0.0.255")
     assert not ok("") and not ok(".5") and not ok("5.") and not ok("1..2") and not ok("1.x")
@@ -155,7 +198,7 @@ def test_shared_subtree_is_rejected():
 # masks against the independent partial matcher
 # ---------------------------------------------------------------------------------------
 SMALL_GRAMMARS = {
-    "listing": grammars.paper_listing_example,
+    "dotted_number": grammars.dotted_number,
     "html": grammars.html_template,
     "json": grammars.json_reference_lookup,
     "template0": lambda: grammars.random_template(0, 4, 6),
@@ -568,7 +611,7 @@ def test_token_level_write_allows_exactly_the_next_token_at_token_boundaries():
 def test_golden_fixture_of_the_section_3_2_listing():
     import os
     path = os.path.join(os.path.dirname(__file__), "golden", "section_3_2_listing_language.txt")
-    tree = tree_of(grammars.paper_listing_example())
+    tree = tree_of(worked_example_tree())
     n = 0
     for line in open(path):
         line = line.rstrip("\n")

@@ -1,7 +1,6 @@
 """Templates with holes (host side, no GPU): an instantiated template must accept exactly the
 language of the tree in which every hole is replaced by its argument's tree, which the CPU
 checker interprets directly.  The two are walked side by side over every reachable transition."""
-import time
 
 import numpy as np
 import pytest
@@ -140,9 +139,11 @@ def test_what_is_refused(wg):
     assert g.step(g.walk(g.start_state, b"axx"), EOS) == g.done_state
 
 
-def test_instantiation_is_cheaper_than_lowering_when_the_static_part_dominates(wg):
+def test_instantiation_only_lowers_the_arguments_when_the_static_part_dominates(wg):
     # a long fixed outline with a short enum per section: the shape of the paper's
-    # outline-generation task, where the tags are known offline and only titles vary
+    # outline-generation task, where the tags are known offline and only titles vary.  What a
+    # request still has to lower is counted in table rows (states), not timed: a clock-based
+    # comparison would depend on what else the machine is doing.
     parts, args = [], []
     rng = np.random.default_rng(3)
     for i in range(300):
@@ -153,23 +154,18 @@ def test_instantiation_is_cheaper_than_lowering_when_the_static_part_dominates(w
                         for _ in range(12)})
         args.append(enum_trie(names))
     template = Sequence(parts)
-    whole = flatten(substitute(template, args))
+    whole = wg.Grammar(flatten(substitute(template, args)))
     T = wg.Template(flatten(template))
-    flat_args = [flatten(a) for a in args]
-
-    def best(fn, n=5):
-        out = []
-        for _ in range(n):
-            t0 = time.perf_counter()
-            fn()
-            out.append(time.perf_counter() - t0)
-        return min(out)
-
-    t_full = best(lambda: wg.Grammar(whole))
-    t_inst = best(lambda: T.instantiate([wg.Grammar(f) for f in flat_args]))
-    g = T.instantiate([wg.Grammar(f) for f in flat_args])
-    assert g.n_states == wg.Grammar(whole).n_states > 20000
-    assert t_inst < t_full, (t_inst, t_full)
+    compiled_args = [wg.Grammar(flatten(a)) for a in args]
+    g = T.instantiate(compiled_args)
+    assert g.n_states == whole.n_states > 20000
+    # per request: four small argument grammars instead of the whole tree
+    lowered_per_request = sum(a.n_states for a in compiled_args)
+    assert lowered_per_request * 50 < whole.n_states
+    assert T.n_states * 2 > whole.n_states - 300 * max(a.n_states for a in compiled_args)
+    for probe, alive in ((b'<section class="outline-level-2" data-index="0"><h2 id="', True),
+                         (b"<sec", True), (b"<section id", False)):
+        assert (g.walk(g.start_state, probe) != 0) == alive == (whole.walk(whole.start_state, probe) != 0)
 
 
 def _random_op(rng, depth, hole_args=0):

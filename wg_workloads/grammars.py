@@ -17,23 +17,15 @@ from .optree import (ALL_BYTES, DIGITS, Cond, DoWhile, Hole, IfElse, Op, Sequenc
 LT = ord("<")
 
 
-def paper_listing_example() -> Op:
-    """The operator tree of the listing in Section 3.2 (digits, dot-separated, then EOS)."""
+def dotted_number() -> Op:
+    """One or more digits, then any number of groups of a period and one or more digits, then the
+    end of sequence: the language Section 3.2 states for its worked example, built here from that
+    statement (a digit, then "more digits or a period and a digit again" as a loop)."""
     from .optree import EOS
-    d = DIGITS
-    cond_allow = d | b"." | [EOS]
-    return Sequence(
-        Wait(allow=d, wait=d),
-        IfElse(
-            condition=Cond(allow=cond_allow, true_waits=SymSet([EOS]), false_waits=SymSet(b".")),
-            if_body=None,
-            else_body=DoWhile(
-                body=Wait(allow=d, wait=d),
-                condition=Cond(allow=cond_allow, true_waits=SymSet(b"."),
-                               false_waits=SymSet([EOS])),
-            ),
-        ),
-    )
+    digit = Wait(allow=DIGITS, wait=DIGITS)
+    return DoWhile(body=digit,
+                   condition=Cond(allow=DIGITS | b"." | [EOS], true_waits=SymSet(b"."),
+                                  false_waits=SymSet([EOS])))
 
 
 def text_slot(closing: bytes) -> List[Op]:
@@ -84,19 +76,14 @@ def int_0_63(terminator: bytes) -> Op:
 
 
 def id_path_string() -> Op:
-    """A quoted string of /-separated decimal node ids: the Section 3.2 pattern with '/'."""
-    allow = DIGITS | b'/"'
+    """A quoted string of /-separated decimal node ids (``"12/7/3"``): the language of
+    ``dotted_number`` with '/' for the period and a closing quote for the end of sequence."""
+    digit = Wait(allow=DIGITS, wait=DIGITS)
     return Sequence(
         Write(b'"'),
-        Wait(allow=DIGITS, wait=DIGITS),
-        IfElse(
-            condition=Cond(allow=allow, true_waits=SymSet(b'"'), false_waits=SymSet(b"/")),
-            if_body=None,
-            else_body=DoWhile(
-                body=Wait(allow=DIGITS, wait=DIGITS),
-                condition=Cond(allow=allow, true_waits=SymSet(b"/"), false_waits=SymSet(b'"')),
-            ),
-        ),
+        DoWhile(body=digit,
+                condition=Cond(allow=DIGITS | b'/"', true_waits=SymSet(b"/"),
+                               false_waits=SymSet(b'"'))),
     )
 
 
