@@ -530,6 +530,7 @@ int32_t wg_ctx_create_ex(const wg_vocab *vocab, int32_t cache_capacity, int32_t 
     take(&d.build_next, 2);
     take(&d.argkey, (size_t)max_batch);
     take(&d.stats, (size_t)ST_COUNT);
+    take(&d.row_done, (size_t)max_batch);
     take(&c->d_stage_gid, (size_t)max_batch);
     take(&c->d_stage_sid, (size_t)max_batch);
     c->grammar_cap = 64;
@@ -544,7 +545,8 @@ int32_t wg_ctx_create_ex(const wg_vocab *vocab, int32_t cache_capacity, int32_t 
             cudaMemset(d.bl_count, 0, sizeof(int32_t)) != cudaSuccess ||
             cudaMemset(d.build_next, 0, 2 * sizeof(int32_t)) != cudaSuccess ||
             cudaMemset(d.argkey, 0, sizeof(unsigned long long) * (size_t)max_batch) != cudaSuccess ||
-            cudaMemset(d.stats, 0, sizeof(unsigned long long) * ST_COUNT) != cudaSuccess)
+            cudaMemset(d.stats, 0, sizeof(unsigned long long) * ST_COUNT) != cudaSuccess ||
+            cudaMemset(d.row_done, 0, sizeof(int32_t) * (size_t)max_batch) != cudaSuccess)
             rc = WG_ERR_CUDA;
         if (compact && rc == WG_OK &&
             (cudaMemset(d.arena_top, 0, sizeof(unsigned long long)) != cudaSuccess ||
@@ -868,6 +870,9 @@ int32_t launch_apply(int32_t dtype, const ApplyArgs &a, const CtxDev &ctx,
 
 bool batch_ok(const wg_ctx *c, int32_t B) { return c && B >= 1 && B <= c->max_batch; }
 
+// wg_decode_step over at most this many rows is one kernel launch
+constexpr int SMALL_STEP_ROWS = 32;
+
 }  // namespace
 
 extern "C" {
@@ -1028,6 +1033,24 @@ int32_t decode_step_impl(wg_ctx *c, const int32_t *gid, int32_t *sid, int32_t B,
     ApplyArgs a{row0, row_stride_elems, bitmask, bitmask, mask_stride_words, B, v_end, W_end, 0,
                 v_begin / 1024};
     const int32_t t_last = v_end == v.V ? v.W * 32 : v_end;
+    if (whole && !best_keys && B <= SMALL_STEP_ROWS && rows_aligned(logits, row_stride_elems, esize)) {
+        // A handful of rows: the whole step in one launch (see decode_step_small_kernel).
+        int32_t rc;
+        if ((rc = timing_mark(c, 0, st)) != WG_OK) return rc;
+        if ((rc = timing_mark(c, 1, st)) != WG_OK) return rc;
+        if ((rc = timing_mark(c, 2, st)) != WG_OK) return rc;
+        const dim3 grid = apply_grid(a);
+        const SmallStepArgs ss{gid, sid, token_out, status, (uint32_t)(flags & WG_RESTART_ON_DONE),
+                               no_cache ? 0 : 1};
+        if (dtype == WG_DTYPE_BF16)
+            WG_CUDA(launch_pdl(decode_step_small_kernel<uint16_t>, grid, dim3(APPLY_THREADS), st, a,
+                               c->dev, v, ss));
+        else
+            WG_CUDA(launch_pdl(decode_step_small_kernel<uint32_t>, grid, dim3(APPLY_THREADS), st, a,
+                               c->dev, v, ss));
+        WG_LAUNCHED();
+        return timing_mark(c, 3, st);
+    }
     // Every kernel of the step is launched with programmatic stream serialization and starts
     // with griddepcontrol.wait, so launch latency and block scheduling of a kernel overlap the
     // tail of the one before it (also across consecutive steps on one stream).

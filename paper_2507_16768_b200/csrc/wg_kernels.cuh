@@ -73,6 +73,8 @@ struct CtxDev {
                                        // both zero between launches
     unsigned long long *argkey;  // [max_batch] packed (value key, ~id) maxima
     unsigned long long *stats;   // [ST_COUNT]
+    int32_t *row_done;           // [max_batch] one-launch step: blocks of the row that have finished
+                                 // (the last one ends the step for the row); zero between launches
     // "what follows byte b" masks of the vocabulary, made for the bytes that close a free-text
     // slot of some added grammar (see after_masks_kernel); slot k holds AFTER_ROWS rows of W words
     const uint32_t *after_masks; // [AFTER_SLOTS][AFTER_ROWS][W], or NULL while no byte needed them
@@ -486,6 +488,241 @@ build_masks_kernel(VocabDev v, CtxDev ctx, BuildWork work) {
 }
 
 // ---------------------------------------------------------------------------------------
+// Warp-level building blocks of a mask build inside another kernel (the one-launch step below):
+// a warp decides whole spans 32 tokens per lane at a time, queues the undecided tokens in its own
+// slice of shared memory, walks them and ends with the spans' finished words in registers, one
+// word per lane -- the layout the apply sweeps take their mask words in.  The arithmetic is that
+// of build_masks_kernel (see the comment there).
+// ---------------------------------------------------------------------------------------
+constexpr int WARP_QUEUE = 1024;   // queued tokens per warp: one whole span always fits
+
+// The facts about the mask of one (grammar, state), gathered by one warp.
+struct MaskFacts {
+    const void *table;
+    const uint8_t *byte_class;
+    const uint4 *rec_class;
+    uint32_t *dst;
+    const uint32_t *after_rows;     // "what follows the closing byte" masks, or NULL
+    unsigned long long leaves, after_fold;
+    uint32_t s0, eos_next;
+    int32_t gid, n_classes, wide, n_ok, forced_tok, row;
+    int32_t n_first, n_fold;        // entries of the two lists below
+    uint8_t first_list[128];        // first bytes to OR (or to exclude, when complemented)
+    uint8_t fold_list[64];          // folds of the leaving bytes (unused when there are too many)
+};
+
+// Called by ONE warp: the grammar record and the state's sets for (gid, sid) into fx.
+__device__ __forceinline__ void gather_item_facts(const VocabDev &v, const CtxDev &ctx, int gid_, int sid_,
+                                                  uint32_t *dst, int row, bool first_chunk, MaskFacts &fx) {
+    const int lane = threadIdx.x & 31;
+    uint32_t s_ = (uint32_t)sid_;
+    const bool known_ = gid_ >= 0 && gid_ < ctx.n_grammars;
+    GrammarDev g = {};
+    if (known_) g = ctx.grammars[gid_];
+    if (!known_ || s_ >= (uint32_t)g.n_states) s_ = 0;  // unknown state: an all-zero row
+    const uint32_t ok_word_ = (s_ && lane < 8) ? g.first_ok[(size_t)s_ * 8 + lane] : 0u;
+    int n_ok_ = __popc(ok_word_);
+#pragma unroll
+    for (int o = 4; o > 0; o >>= 1) n_ok_ += __shfl_xor_sync(0xFFFFFFFFu, n_ok_, o);
+    n_ok_ = __shfl_sync(0xFFFFFFFFu, n_ok_, 0);
+    const bool complement = n_ok_ > 128;
+    // the list of first bytes: byte 32 * j + lane, taken when its bit differs from `complement`
+    int n_first_ = 0;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const uint32_t word = __shfl_sync(0xFFFFFFFFu, ok_word_, j);
+        const bool take = (((word >> lane) & 1u) != 0u) != complement;
+        const uint32_t m = __ballot_sync(0xFFFFFFFFu, take);
+        if (take) fx.first_list[n_first_ + __popc(m & ((1u << lane) - 1u))] = (uint8_t)(32 * j + lane);
+        n_first_ += __popc(m);
+    }
+    const unsigned long long leaves_ = s_ ? g.leaves[s_] : 0ull;
+    int n_fold_ = 0;
+    if (__popcll(leaves_) <= BUILD_MAX_FOLDS) {
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            const bool take = (leaves_ >> (32 * j + lane)) & 1ull;
+            const uint32_t m = __ballot_sync(0xFFFFFFFFu, take);
+            if (take) fx.fold_list[n_fold_ + __popc(m & ((1u << lane) - 1u))] = (uint8_t)(32 * j + lane);
+            n_fold_ += __popc(m);
+        }
+    }
+    if (lane == 0) {
+        fx.gid = known_ ? gid_ : -1;
+        fx.s0 = s_;
+        fx.dst = dst;
+        fx.row = row;
+        fx.table = g.table;
+        fx.byte_class = g.byte_class;
+        fx.rec_class = g.rec_class;
+        fx.n_classes = g.n_classes;
+        fx.wide = g.wide;
+        fx.n_ok = n_ok_;
+        fx.n_first = n_first_;
+        fx.n_fold = n_fold_;
+        fx.leaves = leaves_;
+        uint32_t eos_ = 0;
+        if (s_) eos_ = g.wide ? static_cast<const uint32_t *>(g.table)[(size_t)s_ * g.n_classes + g.eos_class]
+                             : static_cast<const uint16_t *>(g.table)[(size_t)s_ * g.n_classes + g.eos_class];
+        fx.eos_next = eos_;
+        fx.forced_tok = (s_ && g.forced) ? g.forced[s_].x : -1;  // token-level Write state
+        // A free-text slot has ONE byte that leads on (its closing byte); a token that
+        // holds it is dead unless that byte ends the token or the byte after its first
+        // occurrence survives in the next state.  The vocabulary masks for that byte turn
+        // this into word-wise work.
+        const uint32_t *rows_ = nullptr;
+        unsigned long long fold_ = 0ull;
+        if (s_ && ctx.after_masks) {
+            const int lv = g.leave1[s_];
+            if (lv >= 0) {
+                fold_ = g.leave_fold[s_];  // 0: not a state the masks were made for
+                const int k_ = fold_ != 0ull ? ctx.after_slot[lv] : -1;
+                if (k_ >= 0) rows_ = ctx.after_masks + (size_t)k_ * AFTER_ROWS * v.W;
+            }
+        }
+        fx.after_rows = rows_;
+        fx.after_fold = fold_;
+        if (first_chunk) {
+            atomicAdd(&ctx.stats[ST_BUILT], 1ull);
+            if (s_ == 0 && sid_ != 0) atomicAdd(&ctx.stats[ST_BAD_STATE], 1ull);
+        }
+    }
+}
+
+// Mask words w[0..K) of the state described by fx, as far as they can be decided 32 tokens at a
+// time: `alive` = tokens allowed without a walk, `todo` = tokens that need the table walk.  A
+// negative w[k] is skipped.  The loads of the K words are independent of one another and of every
+// branch, so they are all in flight together (one round trip to L2 for the lot).
+template <int K, bool COUNT>
+__device__ __forceinline__ void decide_words(const VocabDev &v, const MaskFacts &fx, const int (&w)[K],
+                                             uint32_t (&alive)[K], uint32_t (&todo)[K],
+                                             int &counted_words) {
+#pragma unroll
+    for (int k = 0; k < K; ++k) { alive[k] = 0; todo[k] = 0; }
+    if (fx.forced_tok >= 0) {
+#pragma unroll
+        for (int k = 0; k < K; ++k)
+            if ((fx.forced_tok >> 5) == w[k] && fx.forced_tok < v.V) alive[k] = 1u << (fx.forced_tok & 31);
+        return;
+    }
+    if (fx.s0 == 0) return;
+    const int nf = fx.n_first, nq = fx.n_fold;
+    const bool complement = fx.n_ok > 128;
+    const bool queue_all = __popcll(fx.leaves) > BUILD_MAX_FOLDS;
+    uint32_t p[K], q[K];
+    size_t at[K];   // a word that is skipped reads word 0 and throws the result away
+#pragma unroll
+    for (int k = 0; k < K; ++k) { p[k] = 0; q[k] = queue_all ? 0xFFFFFFFFu : 0u; at[k] = w[k] < 0 ? 0 : (size_t)w[k]; }
+    for (int i = 0; i < nf; ++i) {
+        const uint32_t *row = v.first_mask + (size_t)fx.first_list[i] * v.W;
+#pragma unroll
+        for (int k = 0; k < K; ++k) p[k] |= __ldg(&row[at[k]]);
+    }
+    if (complement) {
+#pragma unroll
+        for (int k = 0; k < K; ++k) p[k] = __ldg(&v.valid_mask[at[k]]) & ~p[k];
+    }
+    for (int i = 0; i < nq; ++i) {
+        const uint32_t *row = v.fold_mask + (size_t)fx.fold_list[i] * v.W;
+#pragma unroll
+        for (int k = 0; k < K; ++k) q[k] |= __ldg(&row[at[k]]);
+    }
+    const uint32_t *rows = fx.after_rows;
+    uint32_t has[K], worth[K];
+#pragma unroll
+    for (int k = 0; k < K; ++k) { has[k] = 0; worth[k] = 0; }
+    if (rows != nullptr) {   // uniform: loaded whether or not a word turns out to need them
+#pragma unroll
+        for (int k = 0; k < K; ++k) {
+            has[k] = __ldg(&rows[at[k]]);
+            worth[k] = __ldg(&rows[(size_t)v.W + at[k]]);
+        }
+        for (unsigned long long f = fx.after_fold; f; f &= f - 1) {
+            const uint32_t *row = rows + (size_t)(2 + __ffsll((long long)f) - 1) * v.W;
+#pragma unroll
+            for (int k = 0; k < K; ++k) worth[k] |= __ldg(&row[at[k]]);
+        }
+    }
+#pragma unroll
+    for (int k = 0; k < K; ++k) {
+        if (w[k] < 0) continue;
+        uint32_t a = p[k] & ~q[k], t = p[k] & q[k];
+        if (rows != nullptr) {
+            if (fx.n_ok == 256) {
+                // no byte kills the state and only the closing byte leaves it: a token
+                // without that byte is allowed without a walk (the folded sets also
+                // catch the other bytes of the closing byte's fold, e.g. 'b' for '"')
+                a |= t & ~has[k];
+                t &= has[k];
+            }
+            // a token that holds the closing byte is only worth a walk when that byte ends it
+            // or the byte after its first occurrence can survive in the next state
+            t &= ~has[k] | worth[k];
+        }
+        if ((v.eos_id >> 5) == w[k] && fx.eos_next != 0) a |= 1u << (v.eos_id & 31);
+        alive[k] = a;
+        todo[k] = t;
+        if (COUNT)
+            counted_words += nf + nq + (complement ? 1 : 0) +
+                             (rows != nullptr ? 2 + __popcll(fx.after_fold) : 0);
+    }
+}
+
+// Walks the tokens a warp has queued (entries: span slot k << 10 | token within the span) and
+// ORs the survivors into the warp's scratch words; called by the whole warp.
+template <bool COUNT>
+__device__ __forceinline__ void walk_queued(const VocabDev &v, const MaskFacts &fx, const uint16_t *queue,
+                                            int n, int t_base, int span_step, uint32_t *scratch,
+                                            int &counted_lookups) {
+    const int lane = threadIdx.x & 31;
+    __syncwarp();
+    for (int i = lane; i < n; i += 32) {
+        const int e = queue[i];
+        const int k = e >> 10, rel = e & 1023;
+        const int t = t_base + k * span_step + rel;
+        int *const counter = COUNT ? &counted_lookups : nullptr;
+        const uint32_t end = fx.wide
+            ? walk_token_classes<uint32_t>(v, fx.rec_class, static_cast<const uint32_t *>(fx.table),
+                                           fx.n_classes, fx.byte_class, fx.s0, t, counter)
+            : walk_token_classes<uint16_t>(v, fx.rec_class, static_cast<const uint16_t *>(fx.table),
+                                           fx.n_classes, fx.byte_class, fx.s0, t, counter);
+        if (end != 0) atomicOr(&scratch[k * 32 + (rel >> 5)], 1u << (rel & 31));
+    }
+    __syncwarp();
+}
+
+// Appends the set bits of todo[k], for the span slots k named in `slots`, to the warp's queue
+// (which holds `queued` entries); returns the new count.  Called by the whole warp.
+template <int K>
+__device__ __forceinline__ int push_queued(uint16_t *queue, int queued, const uint32_t (&todo)[K],
+                                           uint32_t slots) {
+    const int lane = threadIdx.x & 31;
+    int n_mine = 0;
+#pragma unroll
+    for (int k = 0; k < K; ++k)
+        if ((slots >> k) & 1u) n_mine += __popc(todo[k]);
+    int before = n_mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int x = __shfl_up_sync(0xFFFFFFFFu, before, o);
+        if (lane >= o) before += x;
+    }
+    const int total = __shfl_sync(0xFFFFFFFFu, before, 31);
+    int at = queued + before - n_mine;
+#pragma unroll
+    for (int k = 0; k < K; ++k) {
+        if (!((slots >> k) & 1u)) continue;
+        uint32_t bits = todo[k];
+        while (bits) {
+            const int bit = __ffs(bits) - 1;
+            bits &= bits - 1;
+            queue[at++] = (uint16_t)((k << 10) | (lane * 32 + bit));
+        }
+    }
+    return queued + total;
+}
+
+// ---------------------------------------------------------------------------------------
 // Set-up kernels of wg_ctx_add_grammar (a grammar that is instantiated per request is added on
 // the request's critical path, so its derived arrays are made here rather than on the host).
 // ---------------------------------------------------------------------------------------
@@ -624,6 +861,26 @@ __device__ __forceinline__ uint32_t cache_hash(unsigned long long k) {
 }
 
 constexpr int32_t ENT_NEW = 0x40000000;  // marks the row that inserted its key in this call
+
+// Read-only probe for (g, s): the pool row; -1 when the key is absent; -2 when it is present
+// without a usable row (taken while the pool was full, being filed at this moment, or a compact
+// entry that found no room in the arena).
+__device__ __forceinline__ int32_t cache_probe(const CtxDev &ctx, int g, int s) {
+    if (ctx.hash_size <= 0) return -1;
+    const unsigned long long key = cache_key(g, s);
+    const uint32_t mask = (uint32_t)ctx.hash_size - 1;
+    uint32_t h = cache_hash(key) & mask;
+    for (int probe = 0; probe < ctx.hash_size; ++probe, h = (h + 1) & mask) {
+        const unsigned long long k = ctx.keys[h];
+        if (k == key) {
+            const int32_t row = *(volatile int32_t *)&ctx.vals[h];
+            if (row < 0 || (ctx.compact && ctx.ent_fail[row])) return -2;
+            return row;
+        }
+        if (k == 0) break;
+    }
+    return -1;
+}
 
 // Read-only probe: slot[r] = pool row or -1.
 __global__ void cache_lookup_kernel(CtxDev ctx, const int32_t *gid, const int32_t *sid, int B,
@@ -895,42 +1152,21 @@ __device__ __forceinline__ void pdl_enter() {
     asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
-// grid = (blocks per row, B).  Requires 16-byte aligned rows (pointer and stride).
-template <typename E, bool ARGMAX, bool GATHER>
-// (every variant fits 64 registers, four blocks per SM; one of them has to be told)
-__global__ void __launch_bounds__(APPLY_THREADS, (sizeof(E) == 4 && ARGMAX && !GATHER) ? 4 : 0)
-apply_mask_kernel(ApplyArgs a, CtxDev ctx, unsigned long long *argkey) {
+// The two sweeps of the apply kernels over the spans [span_begin, span_end) of one row, for the
+// calling block: this warp's spans are span_begin + warp, + APPLY_WARPS, ...; words[k] holds mask
+// word `lane` of the k-th of them.  Returns the packed (value, token) maximum of this thread's
+// allowed elements (0 when it saw none).
+template <typename E, bool ARGMAX>
+__device__ __forceinline__ unsigned long long apply_spans(E *row, const uint32_t (&words)[APPLY_SPANS_PER_WARP],
+                                                          int span_begin, int span_end, int V) {
     constexpr int EPC = ElemTraits<E>::PER_CHUNK;  // elements per chunk: bits per lane
     constexpr int CHUNKS_PER_WORD = 32 / EPC;      // 4 (bf16) or 8 (fp32)
     constexpr int PASSES = CHUNKS_PER_WORD;        // 16-byte accesses per lane and span
     constexpr int GROUP = 4;                       // accesses issued together
     constexpr uint32_t FULL = (1u << EPC) - 1;
     constexpr uint32_t SKIP = 0xFFFFFFFFu;
-    pdl_enter();
-    const int r = blockIdx.y;
-    E *row = static_cast<E *>(a.logits) + (int64_t)r * a.row_stride;
-    const uint32_t *own = a.bitmask + (int64_t)r * a.mask_stride;
-    const uint32_t *mrow = own;
-    const uint2 *entry = nullptr;  // header row of the state's compact cache entry, if any
-    bool entry_failed = false;     // no room in the arena: the staging row holds the mask
-    if (GATHER) {
-        const int32_t slot = ctx.slot[r];
-        if (slot >= 0 && !ctx.compact) {
-            mrow = ctx.pool + (int64_t)slot * ctx.pool_stride;
-        } else if (slot >= 0) {
-            // The entry is read without waiting for its failure flag (the header row of a cache
-            // row in use only ever names stored words); a failed entry is read again below.
-            entry = ctx.ent_hdr + (int64_t)slot * ctx.hdr_stride;
-            entry_failed = ctx.ent_fail[slot] != 0;
-            mrow = nullptr;
-        }
-    }
-    const bool copy_out = GATHER && mrow != own;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int n_spans = (a.W + 31) / 32;
-    const int span_begin = a.span_first + blockIdx.x * a.spans_per_block;
-    const int span_end = min(span_begin + a.spans_per_block, n_spans);
-    const int full_chunks = a.V / EPC;  // chunks that lie wholly inside the row
+    const int full_chunks = V / EPC;  // chunks that lie wholly inside the row
     // Per-lane running maximum: a strict float compare keeps the first of equal values and
     // treats -0.0 and +0.0 as equal; !(m <= best_v) also takes the very first candidate chunk,
     // whatever its value (best_v starts as NaN).
@@ -938,37 +1174,6 @@ apply_mask_kernel(ApplyArgs a, CtxDev ctx, unsigned long long *argkey) {
     int best_chunk = -1;
     uint32_t best_bits = 0, best_w[4] = {0, 0, 0, 0};
 
-    // The mask words of every span this warp will handle are fetched first, so their L2
-    // latency is paid once and not once per span (the spans themselves are store streams).
-    uint32_t words[APPLY_SPANS_PER_WARP];
-#pragma unroll
-    for (int k = 0; k < APPLY_SPANS_PER_WARP; ++k) {
-        const int w = (span_begin + warp + k * APPLY_WARPS) * 32 + lane;
-        words[k] = 0;
-        if (span_begin + warp + k * APPLY_WARPS < span_end) {
-            if (GATHER && entry)
-                words[k] = entry_word(entry, ctx.arena, span_begin + warp + k * APPLY_WARPS, lane,
-                                      a.V, a.W);
-            else if (w < a.W)
-                words[k] = mrow[w];
-        }
-    }
-    if (GATHER && entry_failed) {  // built in this call, no room in the arena (uniform per block)
-        const uint32_t *srow = ctx.stage + (int64_t)ctx.ent_stage[ctx.slot[r]] * ctx.pool_stride;
-#pragma unroll
-        for (int k = 0; k < APPLY_SPANS_PER_WARP; ++k) {
-            const int w = (span_begin + warp + k * APPLY_WARPS) * 32 + lane;
-            if (span_begin + warp + k * APPLY_WARPS < span_end && w < a.W) words[k] = srow[w];
-        }
-    }
-    if (copy_out) {
-#pragma unroll
-        for (int k = 0; k < APPLY_SPANS_PER_WARP; ++k) {
-            const int w = (span_begin + warp + k * APPLY_WARPS) * 32 + lane;
-            if (span_begin + warp + k * APPLY_WARPS < span_end && w < a.W)
-                a.bitmask_out[(int64_t)r * a.mask_stride + w] = words[k];
-        }
-    }
     // Sweep 1: every chunk whose bits are all clear is a pure store; chunks that will have to
     // be read (mixed bits, or any allowed element when the argmax is wanted) are only
     // prefetched into L2 here, so no warp waits on DRAM while its stores could be going out.
@@ -1079,6 +1284,72 @@ apply_mask_kernel(ApplyArgs a, CtxDev ctx, unsigned long long *argkey) {
         }
         packed = pack_best(order_key(__float_as_uint(best_v)), idx);
     }
+    return packed;
+}
+
+// grid = (blocks per row, B).  Requires 16-byte aligned rows (pointer and stride).
+template <typename E, bool ARGMAX, bool GATHER>
+// (every variant fits 64 registers, four blocks per SM; one of them has to be told)
+__global__ void __launch_bounds__(APPLY_THREADS, (sizeof(E) == 4 && ARGMAX && !GATHER) ? 4 : 0)
+apply_mask_kernel(ApplyArgs a, CtxDev ctx, unsigned long long *argkey) {
+    constexpr int EPC = ElemTraits<E>::PER_CHUNK;  // elements per 16-byte chunk
+    pdl_enter();
+    const int r = blockIdx.y;
+    E *row = static_cast<E *>(a.logits) + (int64_t)r * a.row_stride;
+    const uint32_t *own = a.bitmask + (int64_t)r * a.mask_stride;
+    const uint32_t *mrow = own;
+    const uint2 *entry = nullptr;  // header row of the state's compact cache entry, if any
+    bool entry_failed = false;     // no room in the arena: the staging row holds the mask
+    if (GATHER) {
+        const int32_t slot = ctx.slot[r];
+        if (slot >= 0 && !ctx.compact) {
+            mrow = ctx.pool + (int64_t)slot * ctx.pool_stride;
+        } else if (slot >= 0) {
+            // The entry is read without waiting for its failure flag (the header row of a cache
+            // row in use only ever names stored words); a failed entry is read again below.
+            entry = ctx.ent_hdr + (int64_t)slot * ctx.hdr_stride;
+            entry_failed = ctx.ent_fail[slot] != 0;
+            mrow = nullptr;
+        }
+    }
+    const bool copy_out = GATHER && mrow != own;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int n_spans = (a.W + 31) / 32;
+    const int span_begin = a.span_first + blockIdx.x * a.spans_per_block;
+    const int span_end = min(span_begin + a.spans_per_block, n_spans);
+    const int full_chunks = a.V / EPC;  // chunks that lie wholly inside the row
+    // The mask words of every span this warp will handle are fetched first, so their L2
+    // latency is paid once and not once per span (the spans themselves are store streams).
+    uint32_t words[APPLY_SPANS_PER_WARP];
+#pragma unroll
+    for (int k = 0; k < APPLY_SPANS_PER_WARP; ++k) {
+        const int w = (span_begin + warp + k * APPLY_WARPS) * 32 + lane;
+        words[k] = 0;
+        if (span_begin + warp + k * APPLY_WARPS < span_end) {
+            if (GATHER && entry)
+                words[k] = entry_word(entry, ctx.arena, span_begin + warp + k * APPLY_WARPS, lane,
+                                      a.V, a.W);
+            else if (w < a.W)
+                words[k] = mrow[w];
+        }
+    }
+    if (GATHER && entry_failed) {  // built in this call, no room in the arena (uniform per block)
+        const uint32_t *srow = ctx.stage + (int64_t)ctx.ent_stage[ctx.slot[r]] * ctx.pool_stride;
+#pragma unroll
+        for (int k = 0; k < APPLY_SPANS_PER_WARP; ++k) {
+            const int w = (span_begin + warp + k * APPLY_WARPS) * 32 + lane;
+            if (span_begin + warp + k * APPLY_WARPS < span_end && w < a.W) words[k] = srow[w];
+        }
+    }
+    if (copy_out) {
+#pragma unroll
+        for (int k = 0; k < APPLY_SPANS_PER_WARP; ++k) {
+            const int w = (span_begin + warp + k * APPLY_WARPS) * 32 + lane;
+            if (span_begin + warp + k * APPLY_WARPS < span_end && w < a.W)
+                a.bitmask_out[(int64_t)r * a.mask_stride + w] = words[k];
+        }
+    }
+    unsigned long long packed = apply_spans<E, ARGMAX>(row, words, span_begin, span_end, a.V);
     // elements after the last whole chunk (V not a multiple of the chunk size)
     if (blockIdx.x == gridDim.x - 1 && full_chunks * EPC < a.V) {
         if (GATHER && entry) {  // the row's last words were written out by this very block
@@ -1159,6 +1430,48 @@ __global__ void export_keys_kernel(CtxDev ctx, long long *out, int B) {
     ctx.argkey[r] = 0ull;
 }
 
+// Row r takes token t: the new state into sid[r], the row's status out.  `chosen`: the token is
+// the step's own greedy choice (-1 = nothing was allowed).
+__device__ __forceinline__ void advance_row(const VocabDev &v, const CtxDev &ctx, const GrammarDev &gr,
+                                            bool known, int32_t *sid, int32_t *status, uint32_t flags,
+                                            int r, int t, bool chosen) {
+    const uint32_t s = (uint32_t)sid[r];
+    int32_t st = WG_OK;
+    if (!known || s >= (uint32_t)gr.n_states) {
+        st = WG_ERR_STATE;
+        atomicAdd(&ctx.stats[ST_BAD_STATE], 1ull);
+    } else if (chosen && t < 0) {
+        st = WG_ERR_EMPTY_MASK;
+        atomicAdd(&ctx.stats[ST_EMPTY], 1ull);
+    } else {
+        uint32_t next = 0;
+        if (gr.forced && s != 0 && gr.forced[s].x >= 0) {  // token-level Write: that token only
+            const int2 f = gr.forced[s];
+            if (t == f.x && t < v.V) next = (uint32_t)f.y;
+        } else if (t >= 0 && t < v.V && s != 0) {
+            // the class-mapped record of the token: one dependent look-up per byte instead of
+            // two (this is a chain of dependent loads at the very end of every step)
+            if (t == v.eos_id)
+                next = gr.wide ? static_cast<const uint32_t *>(gr.table)[(size_t)s * gr.n_classes + gr.eos_class]
+                               : static_cast<const uint16_t *>(gr.table)[(size_t)s * gr.n_classes + gr.eos_class];
+            else
+                next = gr.wide
+                    ? walk_token_classes<uint32_t>(v, gr.rec_class, static_cast<const uint32_t *>(gr.table),
+                                                   gr.n_classes, gr.byte_class, s, t)
+                    : walk_token_classes<uint16_t>(v, gr.rec_class, static_cast<const uint16_t *>(gr.table),
+                                                   gr.n_classes, gr.byte_class, s, t);
+        }
+        if (next == 0) {
+            st = WG_ERR_TOKEN_REJECTED;
+            atomicAdd(&ctx.stats[ST_REJECTED], 1ull);
+        } else {
+            if ((flags & WG_RESTART_ON_DONE) && next == (uint32_t)gr.done) next = (uint32_t)gr.start;
+            sid[r] = (int32_t)next;
+        }
+    }
+    if (status) status[r] = st;
+}
+
 // from_keys: 0 = the tokens come in token_in; 1 = from the fused step's packed maxima; 2 = from
 // ext_keys (signed packed maxima, e.g. after an all-reduce over vocabulary shards).
 __global__ void advance_kernel(VocabDev v, CtxDev ctx, const int32_t *gid, int32_t *sid,
@@ -1187,39 +1500,199 @@ __global__ void advance_kernel(VocabDev v, CtxDev ctx, const int32_t *gid, int32
     } else {
         t = token_in[r];
     }
-    const uint32_t s = (uint32_t)sid[r];
-    int32_t st = WG_OK;
-    if (!known || s >= (uint32_t)gr.n_states) {
-        st = WG_ERR_STATE;
-        atomicAdd(&ctx.stats[ST_BAD_STATE], 1ull);
-    } else if (from_keys && t < 0) {
-        st = WG_ERR_EMPTY_MASK;
-        atomicAdd(&ctx.stats[ST_EMPTY], 1ull);
-    } else {
-        uint32_t next = 0;
-        if (gr.forced && s != 0 && gr.forced[s].x >= 0) {  // token-level Write: that token only
-            const int2 f = gr.forced[s];
-            if (t == f.x && t < v.V) next = (uint32_t)f.y;
-        } else if (t >= 0 && t < v.V && s != 0) {
-            // the class-mapped record of the token: one dependent look-up per byte instead of
-            // two (this kernel is a chain of dependent loads at the very end of every step)
-            if (t == v.eos_id)
-                next = gr.wide ? static_cast<const uint32_t *>(gr.table)[(size_t)s * gr.n_classes + gr.eos_class]
-                               : static_cast<const uint16_t *>(gr.table)[(size_t)s * gr.n_classes + gr.eos_class];
-            else
-                next = gr.wide
-                    ? walk_token_classes<uint32_t>(v, gr.rec_class, static_cast<const uint32_t *>(gr.table),
-                                                   gr.n_classes, gr.byte_class, s, t)
-                    : walk_token_classes<uint16_t>(v, gr.rec_class, static_cast<const uint16_t *>(gr.table),
-                                                   gr.n_classes, gr.byte_class, s, t);
-        }
-        if (next == 0) {
-            st = WG_ERR_TOKEN_REJECTED;
-            atomicAdd(&ctx.stats[ST_REJECTED], 1ull);
-        } else {
-            if ((flags & WG_RESTART_ON_DONE) && next == (uint32_t)gr.done) next = (uint32_t)gr.start;
-            sid[r] = (int32_t)next;
+    advance_row(v, ctx, gr, known, sid, status, flags, r, t, from_keys != 0);
+}
+
+// ---------------------------------------------------------------------------------------
+// The whole decode step of a SMALL batch in one launch.  With a handful of rows the four kernels
+// of the step cost more in launches and in the waits between them than in work, so here every
+// block does everything for its part of a row: it probes the cache itself (all blocks of a row
+// make the same read-only probe), takes the mask words from the cached row or, on a miss, builds
+// the words of its own spans (the warp-level build above), masks and scans its logits, and the
+// block that finishes a row LAST (a per-row arrival counter) advances the row's state and, after
+// a miss, files the finished mask row in the cache.  Rows that meet the same new state in one
+// step each build it (there are few rows); one of them files it.
+// grid = (blocks per row, B); needs 16-byte aligned rows.
+// ---------------------------------------------------------------------------------------
+struct SmallStepArgs {
+    const int32_t *gid;
+    int32_t *sid;        // in / out
+    int32_t *token_out;
+    int32_t *status;     // or NULL
+    uint32_t flags;      // WG_RESTART_ON_DONE or 0
+    int32_t use_cache;   // 0: WG_NO_CACHE (every row is built, nothing is probed or filed)
+};
+
+template <typename E>
+__global__ void __launch_bounds__(APPLY_THREADS)
+decode_step_small_kernel(ApplyArgs a, CtxDev ctx, VocabDev v, SmallStepArgs st) {
+    constexpr int EPC = ElemTraits<E>::PER_CHUNK;
+    constexpr int K = APPLY_SPANS_PER_WARP;
+    __shared__ MaskFacts facts;
+    __shared__ uint16_t queues[APPLY_WARPS][WARP_QUEUE];
+    __shared__ uint32_t scratch[APPLY_WARPS][K * 32];
+    __shared__ int32_t sh_slot, sh_last, sh_new_row;
+    pdl_enter();
+    const int r = blockIdx.y;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    E *row = static_cast<E *>(a.logits) + (int64_t)r * a.row_stride;
+    uint32_t *own = a.bitmask_out + (int64_t)r * a.mask_stride;
+    const int g = st.gid[r], s = st.sid[r];
+    // ---- where the row's mask comes from
+    if (threadIdx.x == 0) {
+        int32_t slot = -1;
+        if (st.use_cache && g >= 0 && g < ctx.n_grammars && s > 0 && s < ctx.grammars[g].n_states)
+            slot = cache_probe(ctx, g, s);          // -1: not cached, -2: cached without a row
+        sh_slot = slot;
+        if (blockIdx.x == 0) {
+            if (slot >= 0) atomicAdd(&ctx.stats[ST_HITS], 1ull);
+            else if (st.use_cache) atomicAdd(&ctx.stats[ST_MISSES], 1ull);
         }
     }
-    if (status) status[r] = st;
+    __syncthreads();
+    const int32_t slot = sh_slot;
+    const int n_spans = (a.W + 31) / 32;
+    const int span_begin = a.span_first + blockIdx.x * a.spans_per_block;
+    const int span_end = min(span_begin + a.spans_per_block, n_spans);
+    uint32_t words[K];
+    if (slot >= 0) {
+        const bool failed = ctx.compact && ctx.ent_fail[slot] != 0;   // (never true: probed above)
+        const uint2 *entry = ctx.compact ? ctx.ent_hdr + (int64_t)slot * ctx.hdr_stride : nullptr;
+        const uint32_t *mrow = ctx.compact ? nullptr : ctx.pool + (int64_t)slot * ctx.pool_stride;
+#pragma unroll
+        for (int k = 0; k < K; ++k) {
+            const int span = span_begin + warp + k * APPLY_WARPS;
+            const int w = span * 32 + lane;
+            words[k] = 0;
+            if (span < span_end && !failed) {
+                if (entry) words[k] = entry_word(entry, ctx.arena, span, lane, a.V, a.W);
+                else if (w < a.W) words[k] = mrow[w];
+            }
+        }
+    } else {
+        // ---- build this block's spans of the mask
+        if (warp == 0) gather_item_facts(v, ctx, g, s, own, -1, blockIdx.x == 0, facts);
+        __syncthreads();
+        uint16_t *queue = queues[warp];
+        uint32_t *mine = scratch[warp];
+#pragma unroll
+        for (int k = 0; k < K; ++k) mine[k * 32 + lane] = 0u;
+        int w[K];
+#pragma unroll
+        for (int k = 0; k < K; ++k) {
+            const int span = span_begin + warp + k * APPLY_WARPS;
+            w[k] = (span < span_end && span * 32 + lane < a.W) ? span * 32 + lane : -1;
+        }
+        uint32_t alive[K], todo[K];
+        int unused_a = 0, unused_b = 0;
+        decide_words<K, false>(v, facts, w, alive, todo, unused_a);
+        const int t_base = (span_begin + warp) << 10;
+        int n_todo = 0;
+#pragma unroll
+        for (int k = 0; k < K; ++k) n_todo += __popc(todo[k]);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) n_todo += __shfl_xor_sync(0xFFFFFFFFu, n_todo, o);
+        if (n_todo > WARP_QUEUE) {   // a state that walks most tokens: span by span
+#pragma unroll
+            for (int k = 0; k < K; ++k) {
+                const int n = push_queued<K>(queue, 0, todo, 1u << k);
+                walk_queued<false>(v, facts, queue, n, t_base, APPLY_WARPS << 10, mine, unused_b);
+            }
+        } else if (n_todo > 0) {
+            const int n = push_queued<K>(queue, 0, todo, (1u << K) - 1u);
+            walk_queued<false>(v, facts, queue, n, t_base, APPLY_WARPS << 10, mine, unused_b);
+        } else {
+            __syncwarp();
+        }
+#pragma unroll
+        for (int k = 0; k < K; ++k) words[k] = alive[k] | mine[k * 32 + lane];
+    }
+    // ---- the row's mask words out, then mask and scan the logits
+#pragma unroll
+    for (int k = 0; k < K; ++k) {
+        const int span = span_begin + warp + k * APPLY_WARPS;
+        const int w = span * 32 + lane;
+        if (span < span_end && w < a.W) own[w] = words[k];
+    }
+    unsigned long long packed = apply_spans<E, true>(row, words, span_begin, span_end, a.V);
+    const int full_chunks = a.V / EPC;
+    if (blockIdx.x == gridDim.x - 1 && full_chunks * EPC < a.V) {
+        __syncthreads();   // the row's last words were written out by this very block
+        apply_scalar<E, true>(row, own, full_chunks * EPC, a.V, packed);
+    }
+    block_argmax_commit<true>(packed, ctx.argkey + r);
+    // ---- the last block of the row ends the step for it
+    if (threadIdx.x == 0) {
+        __threadfence();
+        sh_last = atomicAdd(&ctx.row_done[r], 1) == (int)gridDim.x - 1;
+    }
+    __syncthreads();
+    if (!sh_last) return;
+    __threadfence();
+    if (threadIdx.x == 0) {
+        ctx.row_done[r] = 0;
+        const int t = unpack_best(atomicExch(&ctx.argkey[r], 0ull));   // zero again for the next step
+        st.token_out[r] = t;
+        const bool known = g >= 0 && g < ctx.n_grammars;
+        GrammarDev gr = {};
+        if (known) gr = ctx.grammars[g];
+        // File the mask first: the key is claimed here, the row index published after the copy.
+        // A built row that nobody files (no cache, no room, a state the grammar does not have)
+        // counts as uncached.
+        int32_t new_row = -1;
+        if (st.use_cache && slot < 0) {
+            bool filed = false;   // by this row, or by another row that met the same state
+            if (ctx.hash_size > 0 && known && s > 0 && s < gr.n_states) {
+                const unsigned long long key = cache_key(g, s);
+                const uint32_t mask = (uint32_t)ctx.hash_size - 1;
+                uint32_t h = cache_hash(key) & mask;
+                for (int probe = 0; probe < ctx.hash_size; ++probe, h = (h + 1) & mask) {
+                    unsigned long long k = ctx.keys[h];
+                    if (k == 0) {
+                        if (*(volatile int32_t *)ctx.n_slots >= ctx.capacity) break;   // full
+                        k = atomicCAS(&ctx.keys[h], 0ull, key);
+                        if (k == 0) {
+                            const int32_t got = atomicAdd(ctx.n_slots, 1);
+                            if (got < ctx.capacity) {
+                                new_row = got;
+                                filed = true;
+                                if (ctx.compact) ctx.ent_fail[got] = 0;
+                            } else {
+                                atomicSub(ctx.n_slots, 1);   // the key stays, without a row
+                            }
+                            ctx.ent[r] = (int32_t)h;
+                            break;
+                        }
+                    }
+                    if (k == key) {
+                        // another row files it in this step (or did, with a compact entry that
+                        // found no room); a key left without a row by a full pool is not filed
+                        filed = *(volatile int32_t *)ctx.n_slots < ctx.capacity ||
+                                *(volatile int32_t *)&ctx.vals[h] >= 0;
+                        break;
+                    }
+                }
+            }
+            if (!filed) atomicAdd(&ctx.stats[ST_UNCACHED], 1ull);
+        }
+        sh_new_row = new_row;
+        advance_row(v, ctx, gr, known, st.sid, st.status, st.flags, r, t, true);
+    }
+    __syncthreads();
+    const int32_t new_row = sh_new_row;
+    if (new_row < 0) return;
+    if (!ctx.compact) {
+        uint32_t *dst = ctx.pool + (int64_t)new_row * ctx.pool_stride;
+        for (int w = threadIdx.x; w < a.W; w += APPLY_THREADS) dst[w] = __ldcg(&own[w]);
+    } else {
+        for (int span = warp; span < n_spans; span += APPLY_WARPS) {
+            const int w = span * 32 + lane;
+            store_span(ctx.ent_hdr + (int64_t)new_row * ctx.hdr_stride, ctx.arena, ctx.arena_top,
+                       ctx.arena_words, ctx.ent_fail + new_row, ctx.stats + ST_UNCACHED, span,
+                       w < a.W ? __ldcg(&own[w]) : 0u, lane, a.V, a.W);
+        }
+    }
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) ctx.vals[ctx.ent[r]] = new_row;   // from now on a probe finds the row
 }

@@ -68,7 +68,9 @@ def test_json_lookup_every_step_on_all_32_rows(wg, torch):
     run(sim, w.steps, set(range(w.steps)))
     st = sim.ctx.stats()
     assert st["cache_hits"] + st["cache_misses"] == w.steps * w.batch
-    assert st["masks_built"] == st["cache_entries"] and len(sim.visited) > 200
+    # (rows that meet a new state in the same step each build it; one of them files it)
+    assert st["masks_built"] >= st["cache_entries"] > 100 and len(sim.visited) > 200
+    assert st["rows_uncached"] == 0
 
 
 def test_cold_templates_batch_256_no_cache(wg, torch):
