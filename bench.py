@@ -36,6 +36,32 @@ import numpy as np  # noqa: E402
 
 from wg_workloads import BY_NAME, flatten, has_structural_byte, make_logits, make_vocab  # noqa: E402
 
+# dram__bytes_read.sum + dram__bytes_write.sum of ONE launch of the dominant kernel, taken with ncu
+# on the same launch shape, together with the SHA-256 of the kernel source at the time of the
+# capture: a figure is only reported while the kernels are still the ones that were measured.
+NCU_TRAFFIC = {
+    # workload: (bytes per launch, sha256 of paper_2507_16768_b200/csrc/wg_kernels.cuh)
+    "json_warm": (224.7e6, "0d0b65a7487b772b11933209b2fa03f1513e095f8c4031bde9fb8cc984d917aa"),            # 2.7 MB read + 222.0 MB written
+    "html_warm_free_text": (401.1e6, "0d0b65a7487b772b11933209b2fa03f1513e095f8c4031bde9fb8cc984d917aa"),  # 258.3 MB read + 142.8 MB written
+}
+
+
+def kernel_source_hash() -> str:
+    import hashlib
+    path = os.path.join(ROOT, "paper_2507_16768_b200", "csrc", "wg_kernels.cuh")
+    with open(path, "rb") as f:
+        return hashlib.sha256(f.read()).hexdigest()
+
+
+def measured_traffic(workload: str, full_batch: bool):
+    """The ncu DRAM traffic of the workload's dominant kernel, or None when there is no capture of
+    the kernels as they are now."""
+    entry = NCU_TRAFFIC.get(workload)
+    if not entry or not full_batch or entry[1] != kernel_source_hash():
+        return None
+    return entry[0]
+
+
 METRIC = "masked logit rows/s (mask build+apply)"
 UNIT = "rows/s"
 FALLBACK_HBM_GBS = 6650.0
@@ -501,7 +527,8 @@ class Workbench:
             step_gbs = algo / (m["ms"] / m["steps"] * 1e-3) / 1e9
             return {"kernel": "apply_mask_kernel (gather + apply + argmax)", "bound": "hbm",
                     "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                    "peak_kind": f"of {peak_kind}", "traffic": None,
+                    "peak_kind": f"of {peak_kind}",
+                    "traffic": measured_traffic(self.w.name, self.B == self.w.batch),
                     "algorithmic_bytes_per_launch": algo, "avg_launch_ms": apply_ms,
                     "whole_step": {"achieved": step_gbs, "frac": step_gbs / peak,
                                    "what": "the same bytes over the whole step's time"},

@@ -417,7 +417,12 @@ int32_t wg_advance(wg_ctx *ctx, const int32_t *gid, int32_t *sid, const int32_t 
 /* One whole decode step on device buffers: cache lookup, build of the misses, mask rows out,
  * apply with greedy argmax, state advance.  Same results as the four calls above in that
  * order, in fewer kernel launches (the rows are copied from the cache pool inside the apply
- * kernel).  flags: WG_USE_CACHE or WG_NO_CACHE, optionally | WG_RESTART_ON_DONE.
+ * kernel).  Up to 64 rows with 16-byte aligned logits rows the step is ONE launch: every block
+ * probes the cache for its row, builds its own part of the mask on a miss, and the last block of
+ * a row advances the row's state and files a newly built mask in the cache.  On that path rows
+ * that meet the same new state in the same step each build it (masks_built counts every built
+ * row, cache_misses every row that missed) and one of them files it.
+ * flags: WG_USE_CACHE or WG_NO_CACHE, optionally | WG_RESTART_ON_DONE.
  *   token_out  device, B entries (the greedy choice, -1 for an empty mask)
  *   status     device, B entries, or NULL (WG_OK, WG_ERR_EMPTY_MASK, WG_ERR_STATE) */
 int32_t wg_decode_step(wg_ctx *ctx, const int32_t *gid, int32_t *sid, int32_t B, void *logits,
@@ -459,9 +464,9 @@ int32_t wg_advance_keys(wg_ctx *ctx, const int32_t *gid, int32_t *sid, const int
                         int32_t B, int32_t *token_out, int32_t *status, uint32_t flags,
                         void *stream);
 
-/* A decode step recorded once as a CUDA graph and replayed: for small batches the four kernel
- * launches of wg_decode_step cost more host time than the kernels take on the GPU, and a
- * graph launch replaces them with one call.  All arguments are those of wg_decode_step and
+/* A decode step recorded once as a CUDA graph and replayed: where wg_decode_step takes several
+ * kernel launches (more than 64 rows) a graph launch replaces them with one call.  (Up to 64
+ * rows the step is a single kernel already and a plain call is cheaper than a graph launch.)  All arguments are those of wg_decode_step and
  * are frozen into the graph: the caller keeps writing each step's logits into the same
  * buffer (as an LM head does) and reads tokens and states from the same arrays.  Grammars
  * added to the context after creation are not seen by the graph while the context's grammar
