@@ -718,3 +718,36 @@ def test_equal_tables_over_different_class_maps_are_different_grammars(wg, torch
     bits = np.unpackbits(out.cpu().numpy().view(np.uint8), axis=1, bitorder="little")
     assert np.flatnonzero(bits[0]).tolist() == [ord("a")]
     assert np.flatnonzero(bits[1]).tolist() == [ord("b")]
+
+
+@pytest.mark.parametrize("cache_mode,capacity,arena", [(0, 3, 0), (0, 40, 0), (1, 40, 4096), (1, 6, 0)])
+def test_one_launch_step_with_a_cache_that_fills_up(wg, torch, cache_mode, capacity, arena):
+    """Small batches take the one-launch step, which files new masks itself.  A pool (or a compact
+    arena) that is too small must leave the later states uncached -- built on every visit, with
+    the same masks, tokens and states as ever."""
+    vocab = make_vocab(8192, seed=17)
+    ops = [grammars.html_template(), grammars.json_reference_lookup(doc_nodes=60)]
+    rows = [0, 1, 1, 0, 1, 0, 1]
+    sim = Sim(wg, torch, vocab, ops, rows, "bf16", cache_capacity=capacity, seed=12, steer=6.0,
+              cache_mode=cache_mode, arena_bytes=arena)
+    for _ in range(60):
+        sim.step()
+    st = sim.ctx.stats()
+    assert len(sim.visited) > capacity, "the run must meet more states than the cache holds"
+    assert st["rows_uncached"] > 0 and st["cache_entries"] <= capacity
+    assert st["cache_hits"] + st["cache_misses"] == 60 * len(rows)
+    assert st["masks_built"] >= st["cache_misses"] - 0 and st["cache_hits"] > 0
+
+
+def test_one_launch_step_at_its_largest_batch_and_the_first_batch_beyond(wg, torch):
+    vocab = make_vocab(8192, seed=18)
+    ops = [grammars.json_reference_lookup(doc_nodes=80), grammars.random_template(5)]
+    for B in (64, 65):
+        rows = [r % 2 for r in range(B)]
+        sim = Sim(wg, torch, vocab, ops, rows, "fp32", cache_capacity=1024, seed=B, steer=5.0)
+        launches = wg.kernel_launch_count()
+        for _ in range(12):
+            sim.step()
+        per_step = (wg.kernel_launch_count() - launches) / 12
+        assert per_step == (1 if B == 64 else 4)
+        assert sim.ctx.stats()["rows_uncached"] == 0 and len(sim.visited) > 10
