@@ -497,8 +497,9 @@ class Workbench:
         kt = ctx.get_timing()
         ctx.set_timing(False)
         work = None
-        if stats["masks_built"]:
-            # what the build kernel had to do, from its counting variant over a few steps
+        if not self.w.prewarm:
+            # what the build kernel had to do, from its counting variant over a few steps (decided
+            # by the workload, not by this rank's counters: every rank must make the same calls)
             ctx.reset_stats()
             ctx.count_build_work(True)
             self.region(min(steps, 16))

@@ -607,12 +607,12 @@ def test_forced_token_beyond_the_vocabulary_gives_an_empty_mask(wg, torch):
     assert status.item() == wg.binding.WG_ERR_EMPTY_MASK and sid.item() == g.start_state
 
 
-def test_large_batch_stats_reset_and_kernel_timing(wg, torch):
+@pytest.mark.parametrize("B", [3000, 20000])      # several passes of the one-block lookup kernel
+def test_large_batch_stats_reset_and_kernel_timing(wg, torch, B):
     vocab = make_vocab(2048, seed=15)
     flat = flatten(grammars.json_reference_lookup(doc_nodes=40))
     tree, g = oracle.Tree(flat), wg.Grammar(flat)
     dv = wg.Vocab(vocab.offsets, vocab.data, vocab.eos_id)
-    B = 3000                                       # several passes of the one-block lookup kernel
     ctx = wg.Context(dv, 512, B)
     gid = torch.full((B,), ctx.add_grammar(g), dtype=torch.int32, device="cuda")
     cursor_of = co_reachable(tree, g, mentioned_symbols(flat))
@@ -751,3 +751,12 @@ def test_one_launch_step_at_its_largest_batch_and_the_first_batch_beyond(wg, tor
         per_step = (wg.kernel_launch_count() - launches) / 12
         assert per_step == (1 if B == 64 else 4)
         assert sim.ctx.stats()["rows_uncached"] == 0 and len(sim.visited) > 10
+
+
+def test_batches_beyond_the_row_limit_are_refused(wg, torch):
+    vocab = make_vocab(1024, seed=4)
+    dv = wg.Vocab(vocab.offsets, vocab.data, vocab.eos_id)
+    with pytest.raises(wg.WgError) as e:
+        wg.Context(dv, 4, 65536)                   # WG_MAX_ROWS is 65535
+    assert e.value.status == wg.binding.WG_ERR_ARG
+    wg.Context(dv, 4, 65535).close()
