@@ -196,305 +196,11 @@ __device__ __forceinline__ void store_span(uint2 *hdr_row, uint32_t *arena,
 }
 
 // ---------------------------------------------------------------------------------------
-// K1: mask build.  Work item = (mask m, chunk of tokens); a fixed-size grid strides over the
-// items, so a launch with nothing to build costs a few empty blocks.
-//
-// Most tokens are decided 32 at a time, without walking the table.  The vocabulary holds
-// V-bit masks "token starts with byte b" (256 of them) and "token contains a byte that folds
-// to c = b & 63" (64 of them); a state holds the set of first bytes that do not kill it and
-// the folded set of bytes that LEAVE it.  For a word of 32 tokens:
-//   P = tokens whose first byte keeps the state alive   (OR of a few first-byte masks, or the
-//                                                         complement when most bytes are fine)
-//   Q = tokens that contain a byte which may leave       (OR of a few fold masks)
-//   P & ~Q  are allowed: every byte loops on the state   (free-text states: ~all tokens)
-//   ~P      are not allowed                              (literal states: ~all tokens)
-//   P & Q   are queued in shared memory and walked afterwards, densely, one per thread.
+// What the mask of one (grammar, state) is decided from, and the word-wise decision itself; used
+// by the build kernel and by the one-launch step.  The arithmetic is described at the build
+// kernel below.
 // ---------------------------------------------------------------------------------------
-constexpr int BUILD_THREADS = 256;
-constexpr int BUILD_CHUNK_MAX = 8192;  // tokens per work item (the launch picks 2048 or 8192)
 constexpr int BUILD_MAX_FOLDS = 20;    // more leaving folds than this: queue every P token
-
-// The spans of one finished chunk (n_words mask words in shared memory, beginning at span
-// first_span) into a cache row.
-__device__ __forceinline__ void store_chunk_spans(uint2 *hdr_row, uint32_t *arena,
-                                               unsigned long long *arena_top, long long arena_words,
-                                               int32_t *fail_flag, unsigned long long *uncached_stat,
-                                               int first_span, int n_words, const uint32_t *words,
-                                               int V, int W) {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    for (int sl = warp; sl * 32 < n_words; sl += (int)(blockDim.x >> 5)) {
-        const int wl = sl * 32 + lane;
-        store_span(hdr_row, arena, arena_top, arena_words, fail_flag, uncached_stat, first_span + sl,
-                   wl < n_words ? words[wl] : 0u, lane, V, W);
-    }
-}
-
-struct BuildWork {
-    const int32_t *gid, *sid;   // per entry
-    uint32_t *const *dst_list;  // per entry destination, or NULL: use dst_base + m * dst_stride
-    uint32_t *dst_base;
-    int64_t dst_stride;
-    const int32_t *count_ptr;   // number of entries on the device, or NULL: use count
-    int32_t count;
-    int32_t chunk;              // tokens per work item: a multiple of 32, <= BUILD_CHUNK_MAX
-    int32_t t_first, t_last;    // tokens [t_first, t_last) are built: whole chunks, or up to W * 32
-};
-
-// COMPACT: the cache keeps allows / denies entries; finished chunks are also stored as spans.
-// COUNT: the variant that also counts its work (queued tokens, table look-ups, vocabulary-mask
-// words read) for the benchmark's bound; never used for a timed launch.
-template <bool COMPACT, bool COUNT = false>
-__global__ void __launch_bounds__(BUILD_THREADS, (COMPACT || COUNT) ? 5 : 8)
-build_masks_kernel(VocabDev v, CtxDev ctx, BuildWork work) {
-    // the facts about one work item's mask, gathered by warp 0 (two copies: the next item's are
-    // gathered while the other warps walk the current item's tokens)
-    struct ItemFacts {
-        const void *table;
-        const uint8_t *byte_class;
-        const uint4 *rec_class;
-        uint32_t *dst;
-        unsigned long long leaves, after_fold;
-        uint32_t first_ok[8];
-        uint32_t s0, eos_next;
-        int32_t gid, n_classes, wide, n_ok, forced_tok, after_k;
-    };
-    __shared__ ItemFacts facts[2];
-    __shared__ uint8_t cls[256];
-    __shared__ int cls_gid;
-    __shared__ uint8_t first_list[128];  // first bytes to OR (or to exclude, when complemented)
-    __shared__ uint8_t fold_list[64];
-    __shared__ int n_first, n_fold;
-    __shared__ uint32_t words[BUILD_CHUNK_MAX / 32];
-    __shared__ uint16_t todo[BUILD_CHUNK_MAX];
-    __shared__ int n_todo;
-    __shared__ uint32_t next_item;
-    pdl_enter();
-    const int lane = threadIdx.x & 31;
-    const int n_entries = work.count_ptr ? *work.count_ptr : work.count;
-    const int n_chunks = (work.t_last - work.t_first + work.chunk - 1) / work.chunk;
-    // (item numbers stay in 32 bits: the launch refuses more than 2^31 of them; the division by
-    // the chunk count below would otherwise be a 64-bit one, a hundred instructions per item)
-    const uint32_t n_items = (uint32_t)n_entries * (uint32_t)n_chunks;
-    // Nothing to build (every row of a warm step hit the cache): leave at once.  Nobody has
-    // touched the work counters, so they need no reset either -- and the launch is then a few
-    // hundred blocks that read one word and exit, on the critical path of every warm step.
-    if (n_items == 0) return;
-
-    // Called by warp 0: the grammar record and the state's sets of item `it` into fx.
-    auto gather = [&](uint32_t it, ItemFacts &fx) {
-        const int m = (int)(it / (uint32_t)n_chunks);
-        const int t_begin_ = work.t_first + (int)(it - (uint32_t)m * (uint32_t)n_chunks) * work.chunk;
-        const int gid_ = work.gid[m];
-        uint32_t s_ = (uint32_t)work.sid[m];
-        const bool known_ = gid_ >= 0 && gid_ < ctx.n_grammars;
-        GrammarDev g = {};
-        if (known_) g = ctx.grammars[gid_];
-        if (!known_ || s_ >= (uint32_t)g.n_states) s_ = 0;  // unknown state: an all-zero row
-        const uint32_t ok_word_ = (s_ && lane < 8) ? g.first_ok[(size_t)s_ * 8 + lane] : 0u;
-        int n_ok_ = __popc(ok_word_);
-#pragma unroll
-        for (int o = 4; o > 0; o >>= 1) n_ok_ += __shfl_xor_sync(0xFFFFFFFFu, n_ok_, o);
-        if (lane < 8) fx.first_ok[lane] = ok_word_;
-        if (lane == 0) {
-            fx.gid = known_ ? gid_ : -1;
-            fx.s0 = s_;
-            fx.dst = work.dst_list ? work.dst_list[m] : work.dst_base + (int64_t)m * work.dst_stride;
-            fx.table = g.table;
-            fx.byte_class = g.byte_class;
-            fx.rec_class = g.rec_class;
-            fx.n_classes = g.n_classes;
-            fx.wide = g.wide;
-            fx.n_ok = n_ok_;
-            fx.leaves = s_ ? g.leaves[s_] : 0ull;
-            uint32_t eos_ = 0;
-            if (s_) eos_ = g.wide ? static_cast<const uint32_t *>(g.table)[(size_t)s_ * g.n_classes + g.eos_class]
-                                 : static_cast<const uint16_t *>(g.table)[(size_t)s_ * g.n_classes + g.eos_class];
-            fx.eos_next = eos_;
-            fx.forced_tok = (s_ && g.forced) ? g.forced[s_].x : -1;  // token-level Write state
-            // A free-text slot has ONE byte that leads on (its closing byte); a token that
-            // holds it is dead unless that byte ends the token or the byte after its first
-            // occurrence survives in the next state.  The vocabulary masks for that byte turn
-            // this into word-wise work.
-            int k_ = -1;
-            unsigned long long fold_ = 0ull;
-            if (s_ && ctx.after_masks) {
-                const int lv = g.leave1[s_];
-                if (lv >= 0) {
-                    fold_ = g.leave_fold[s_];  // 0: not a state the masks were made for
-                    if (fold_ != 0ull) k_ = ctx.after_slot[lv];
-                }
-            }
-            fx.after_k = k_;
-            fx.after_fold = fold_;
-            if (t_begin_ == work.t_first) {
-                atomicAdd(&ctx.stats[ST_BUILT], 1ull);
-                if (s_ == 0 && work.sid[m] != 0) atomicAdd(&ctx.stats[ST_BAD_STATE], 1ull);
-            }
-        }
-    };
-
-    if (threadIdx.x == 0) { cls_gid = -1; n_todo = 0; n_first = 0; n_fold = 0; }
-    if (threadIdx.x < 32 && blockIdx.x < n_items) gather(blockIdx.x, facts[0]);
-    __syncthreads();
-    // Items differ a lot in cost (a literal state decides nearly everything word-wise, a
-    // free-text state walks thousands of tokens), so after its first item a block takes the next
-    // one from a device counter instead of a fixed stride.  Warp 0 does that, and gathers the
-    // next item's facts, while the other seven warps walk the current item's queued tokens.
-    int cur = 0;
-    for (uint32_t item = blockIdx.x; item < n_items; item = next_item, cur ^= 1) {
-        const ItemFacts &info = facts[cur];
-        const int m = (int)(item / (uint32_t)n_chunks);
-        const int t_begin = work.t_first + (int)(item - (uint32_t)m * (uint32_t)n_chunks) * work.chunk;
-        const int t_end = min(t_begin + work.chunk, work.t_last);
-        const int gid = info.gid;
-        const bool known = gid >= 0;
-        const uint32_t s0 = info.s0;
-        uint32_t *dst = info.dst;
-        if (known && cls_gid != gid) cls[threadIdx.x] = info.byte_class[threadIdx.x];
-        // the state's first-byte set; complemented when more than half of the bytes are fine
-        const uint32_t ok_word = info.first_ok[threadIdx.x >> 5];
-        const int n_ok = info.n_ok;
-        const bool complement = n_ok > 128;
-        const unsigned long long leaves = info.leaves;
-        const bool queue_all = __popcll(leaves) > BUILD_MAX_FOLDS;
-        const uint32_t eos_next = info.eos_next;
-        const int forced_tok = info.forced_tok;
-        const int after_k = info.after_k;
-        const unsigned long long after_fold = info.after_fold;
-        {
-            const bool is_ok = (ok_word >> lane) & 1u;   // thread b looks at byte b
-            if (is_ok != complement) first_list[atomicAdd(&n_first, 1)] = (uint8_t)threadIdx.x;
-            if (threadIdx.x < 64 && !queue_all && ((leaves >> threadIdx.x) & 1ull))
-                fold_list[atomicAdd(&n_fold, 1)] = (uint8_t)threadIdx.x;
-        }
-        __syncthreads();
-        if (threadIdx.x == 0 && known) cls_gid = gid;  // read again only after the next barrier
-        // phase 1: one word of 32 tokens per thread
-        const int n_words = (t_end - t_begin) >> 5;
-        const int nf = n_first, nq = n_fold;
-        int counted_words = 0, counted_lookups = 0;
-        for (int wl = threadIdx.x; wl < ((n_words + 31) & ~31); wl += BUILD_THREADS) {
-            uint32_t alive = 0, queue = 0;
-            const int w = (t_begin >> 5) + wl;
-            if (wl < n_words && forced_tok >= 0) {
-                if ((forced_tok >> 5) == w && forced_tok < v.V) alive = 1u << (forced_tok & 31);
-            } else if (wl < n_words && s0 != 0) {
-                uint32_t p = 0;
-                for (int i = 0; i < nf; ++i) p |= __ldg(&v.first_mask[(size_t)first_list[i] * v.W + w]);
-                if (complement) p = __ldg(&v.valid_mask[w]) & ~p;
-                uint32_t q = queue_all ? 0xFFFFFFFFu : 0u;
-                for (int i = 0; i < nq; ++i) q |= __ldg(&v.fold_mask[(size_t)fold_list[i] * v.W + w]);
-                alive = p & ~q;
-                queue = p & q;
-                if (COUNT) counted_words += nf + nq + (complement ? 1 : 0);
-                if (after_k >= 0 && queue != 0) {
-                    const uint32_t *rows = ctx.after_masks + (size_t)after_k * AFTER_ROWS * v.W;
-                    const uint32_t has = __ldg(&rows[w]);
-                    if (n_ok == 256) {
-                        // no byte kills the state and only the closing byte leaves it: a token
-                        // without that byte is allowed without a walk (the folded sets also
-                        // catch the other bytes of the closing byte's fold, e.g. 'b' for '"')
-                        alive |= queue & ~has;
-                        queue &= has;
-                    }
-                    if (COUNT) counted_words += 1;
-                    if (queue & has) {
-                        uint32_t worth = __ldg(&rows[(size_t)v.W + w]);
-                        for (unsigned long long f = after_fold; f; f &= f - 1)
-                            worth |= __ldg(&rows[(size_t)(2 + __ffsll((long long)f) - 1) * v.W + w]);
-                        queue &= ~has | worth;
-                        if (COUNT) counted_words += 1 + __popcll(after_fold);
-                    }
-                }
-                if ((v.eos_id >> 5) == w && eos_next != 0) alive |= 1u << (v.eos_id & 31);
-            }
-            if (wl < n_words) words[wl] = alive;
-            // queue the undecided tokens: one shared-memory atomic per warp
-            const int mine = __popc(queue);
-            int before = mine;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const int x = __shfl_up_sync(0xFFFFFFFFu, before, o);
-                if (lane >= o) before += x;
-            }
-            int base = 0;
-            if (lane == 31 && before > 0) base = atomicAdd(&n_todo, before);
-            base = __shfl_sync(0xFFFFFFFFu, base, 31) + before - mine;
-            while (queue) {
-                const int bit = __ffs(queue) - 1;
-                queue &= queue - 1;
-                todo[base++] = (uint16_t)(wl * 32 + bit);
-            }
-        }
-        __syncthreads();
-        if (threadIdx.x == 0) { n_first = 0; n_fold = 0; }  // everybody has read them
-        // phase 2: warp 0 takes the block's next item and gathers its facts; the other warps
-        // walk the queued tokens, one per thread (the EOS token is never queued: it has no bytes)
-        const int n = n_todo;
-        if (threadIdx.x < 32) {
-            uint32_t nxt = 0;
-            if (lane == 0) nxt = gridDim.x + (uint32_t)atomicAdd(ctx.build_next, 1);
-            nxt = __shfl_sync(0xFFFFFFFFu, nxt, 0);
-            if (lane == 0) next_item = nxt;
-            if (nxt < n_items) gather(nxt, facts[cur ^ 1]);
-        } else {
-            for (int i = threadIdx.x - 32; i < n; i += BUILD_THREADS - 32) {
-                const int rel = todo[i];
-                int *const counter = COUNT ? &counted_lookups : nullptr;
-                const uint32_t end = info.wide
-                    ? walk_token_classes<uint32_t>(v, info.rec_class, static_cast<const uint32_t *>(info.table),
-                                                   info.n_classes, cls, s0, t_begin + rel, counter)
-                    : walk_token_classes<uint16_t>(v, info.rec_class, static_cast<const uint16_t *>(info.table),
-                                                   info.n_classes, cls, s0, t_begin + rel, counter);
-                if (end != 0) atomicOr(&words[rel >> 5], 1u << (rel & 31));
-            }
-        }
-        if (COUNT) {
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
-                counted_words += __shfl_xor_sync(0xFFFFFFFFu, counted_words, o);
-                counted_lookups += __shfl_xor_sync(0xFFFFFFFFu, counted_lookups, o);
-            }
-            if (lane == 0) {
-                atomicAdd(&ctx.stats[ST_MASK_WORDS], (unsigned long long)counted_words);
-                atomicAdd(&ctx.stats[ST_WALKED], (unsigned long long)counted_lookups);
-            }
-            if (threadIdx.x == 32) atomicAdd(&ctx.stats[ST_QUEUED], (unsigned long long)n);
-        }
-        __syncthreads();
-        if (threadIdx.x == 0) n_todo = 0;  // everybody has read it
-        // phase 3: whole words out
-        for (int wl = threadIdx.x; wl < n_words; wl += BUILD_THREADS)
-            dst[(t_begin >> 5) + wl] = words[wl];
-        // Compact cache: the chunk's spans go into the cache entry straight from shared memory
-        // (chunks are whole spans; the dense words above only serve the call that built them).
-        if (COMPACT && work.dst_list) {
-            const int row = ctx.bl_row[m];
-            if (row >= 0)
-                store_chunk_spans(ctx.ent_hdr + (int64_t)row * ctx.hdr_stride, ctx.arena, ctx.arena_top,
-                                  ctx.arena_words, ctx.ent_fail + row, ctx.stats + ST_UNCACHED,
-                                  t_begin >> 10, n_words, words, v.V, v.W);
-        }
-        __syncthreads();  // the shared arrays are free for the next item
-    }
-    // the last block to leave puts the counters back to zero for the next launch
-    if (threadIdx.x == 0) {
-        __threadfence();
-        if (atomicAdd(ctx.build_done, 1) == (int)gridDim.x - 1) {
-            *ctx.build_next = 0;
-            *ctx.build_done = 0;
-        }
-    }
-}
-
-// ---------------------------------------------------------------------------------------
-// Warp-level building blocks of a mask build inside another kernel (the one-launch step below):
-// a warp decides whole spans 32 tokens per lane at a time, queues the undecided tokens in its own
-// slice of shared memory, walks them and ends with the spans' finished words in registers, one
-// word per lane -- the layout the apply sweeps take their mask words in.  The arithmetic is that
-// of build_masks_kernel (see the comment there).
-// ---------------------------------------------------------------------------------------
-constexpr int WARP_QUEUE = 1024;   // queued tokens per warp: one whole span always fits
 
 // The facts about the mask of one (grammar, state), gathered by one warp.
 struct MaskFacts {
@@ -667,6 +373,189 @@ __device__ __forceinline__ void decide_words(const VocabDev &v, const MaskFacts 
                              (rows != nullptr ? 2 + __popcll(fx.after_fold) : 0);
     }
 }
+
+// ---------------------------------------------------------------------------------------
+// K1: mask build.  Work item = (mask m, chunk of tokens); a fixed-size grid strides over the
+// items, so a launch with nothing to build costs a few empty blocks.
+//
+// Most tokens are decided 32 at a time, without walking the table.  The vocabulary holds
+// V-bit masks "token starts with byte b" (256 of them) and "token contains a byte that folds
+// to c = b & 63" (64 of them); a state holds the set of first bytes that do not kill it and
+// the folded set of bytes that LEAVE it.  For a word of 32 tokens:
+//   P = tokens whose first byte keeps the state alive   (OR of a few first-byte masks, or the
+//                                                         complement when most bytes are fine)
+//   Q = tokens that contain a byte which may leave       (OR of a few fold masks)
+//   P & ~Q  are allowed: every byte loops on the state   (free-text states: ~all tokens)
+//   ~P      are not allowed                              (literal states: ~all tokens)
+//   P & Q   are queued in shared memory and walked afterwards, densely, one per thread.
+// ---------------------------------------------------------------------------------------
+constexpr int BUILD_THREADS = 256;
+constexpr int BUILD_CHUNK_MAX = 8192;  // tokens per work item (the launch picks 2048 or 8192)
+
+// The spans of one finished chunk (n_words mask words in shared memory, beginning at span
+// first_span) into a cache row.
+__device__ __forceinline__ void store_chunk_spans(uint2 *hdr_row, uint32_t *arena,
+                                               unsigned long long *arena_top, long long arena_words,
+                                               int32_t *fail_flag, unsigned long long *uncached_stat,
+                                               int first_span, int n_words, const uint32_t *words,
+                                               int V, int W) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int sl = warp; sl * 32 < n_words; sl += (int)(blockDim.x >> 5)) {
+        const int wl = sl * 32 + lane;
+        store_span(hdr_row, arena, arena_top, arena_words, fail_flag, uncached_stat, first_span + sl,
+                   wl < n_words ? words[wl] : 0u, lane, V, W);
+    }
+}
+
+struct BuildWork {
+    const int32_t *gid, *sid;   // per entry
+    uint32_t *const *dst_list;  // per entry destination, or NULL: use dst_base + m * dst_stride
+    uint32_t *dst_base;
+    int64_t dst_stride;
+    const int32_t *count_ptr;   // number of entries on the device, or NULL: use count
+    int32_t count;
+    int32_t chunk;              // tokens per work item: a multiple of 32, <= BUILD_CHUNK_MAX
+    int32_t t_first, t_last;    // tokens [t_first, t_last) are built: whole chunks, or up to W * 32
+};
+
+// COMPACT: the cache keeps allows / denies entries; finished chunks are also stored as spans.
+// COUNT: the variant that also counts its work (queued tokens, table look-ups, vocabulary-mask
+// words read) for the benchmark's bound; never used for a timed launch.
+template <bool COMPACT, bool COUNT = false>
+__global__ void __launch_bounds__(BUILD_THREADS, (COMPACT || COUNT) ? 5 : 8)
+build_masks_kernel(VocabDev v, CtxDev ctx, BuildWork work) {
+    // the facts about one work item's mask, gathered by warp 0 (two copies: the next item's are
+    // gathered while the other warps walk the current item's tokens)
+    __shared__ MaskFacts facts[2];
+    __shared__ uint32_t words[BUILD_CHUNK_MAX / 32];
+    __shared__ uint16_t todo[BUILD_CHUNK_MAX];
+    __shared__ int n_todo;
+    __shared__ uint32_t next_item;
+    pdl_enter();
+    const int lane = threadIdx.x & 31;
+    const int n_entries = work.count_ptr ? *work.count_ptr : work.count;
+    const int n_chunks = (work.t_last - work.t_first + work.chunk - 1) / work.chunk;
+    // (item numbers stay in 32 bits: the launch refuses more than 2^31 of them; the division by
+    // the chunk count below would otherwise be a 64-bit one, a hundred instructions per item)
+    const uint32_t n_items = (uint32_t)n_entries * (uint32_t)n_chunks;
+    // Nothing to build (every row of a warm step hit the cache): leave at once.  Nobody has
+    // touched the work counters, so they need no reset either -- and the launch is then a few
+    // hundred blocks that read one word and exit, on the critical path of every warm step.
+    if (n_items == 0) return;
+
+    // Called by warp 0: the facts of item `it` into fx.
+    auto gather = [&](uint32_t it, MaskFacts &fx) {
+        const int m = (int)(it / (uint32_t)n_chunks);
+        const int chunk = (int)(it - (uint32_t)m * (uint32_t)n_chunks);
+        uint32_t *dst = work.dst_list ? work.dst_list[m] : work.dst_base + (int64_t)m * work.dst_stride;
+        const int row = (COMPACT && work.dst_list) ? ctx.bl_row[m] : -1;
+        gather_item_facts(v, ctx, work.gid[m], work.sid[m], dst, row, chunk == 0, fx);
+    };
+
+    if (threadIdx.x == 0) n_todo = 0;
+    if (threadIdx.x < 32 && blockIdx.x < n_items) gather(blockIdx.x, facts[0]);
+    __syncthreads();
+    // Items differ a lot in cost (a literal state decides nearly everything word-wise, a
+    // free-text state walks thousands of tokens), so after its first item a block takes the next
+    // one from a device counter instead of a fixed stride.  Warp 0 does that, and gathers the
+    // next item's facts, while the other seven warps walk the current item's queued tokens.
+    int cur = 0;
+    for (uint32_t item = blockIdx.x; item < n_items; item = next_item, cur ^= 1) {
+        const MaskFacts &info = facts[cur];
+        const int m = (int)(item / (uint32_t)n_chunks);
+        const int t_begin = work.t_first + (int)(item - (uint32_t)m * (uint32_t)n_chunks) * work.chunk;
+        const int t_end = min(t_begin + work.chunk, work.t_last);
+        // phase 1: one word of 32 tokens per thread
+        const int n_words = (t_end - t_begin) >> 5;
+        int counted_words = 0, counted_lookups = 0;
+        for (int wl = threadIdx.x; wl < ((n_words + 31) & ~31); wl += BUILD_THREADS) {
+            const int w[1] = {wl < n_words ? (t_begin >> 5) + wl : -1};
+            uint32_t alive[1], queue[1];
+            decide_words<1, COUNT>(v, info, w, alive, queue, counted_words);
+            if (wl < n_words) words[wl] = alive[0];
+            // queue the undecided tokens: one shared-memory atomic per warp
+            const int mine = __popc(queue[0]);
+            int before = mine;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int x = __shfl_up_sync(0xFFFFFFFFu, before, o);
+                if (lane >= o) before += x;
+            }
+            int base = 0;
+            if (lane == 31 && before > 0) base = atomicAdd(&n_todo, before);
+            base = __shfl_sync(0xFFFFFFFFu, base, 31) + before - mine;
+            uint32_t bits = queue[0];
+            while (bits) {
+                const int bit = __ffs(bits) - 1;
+                bits &= bits - 1;
+                todo[base++] = (uint16_t)(wl * 32 + bit);
+            }
+        }
+        __syncthreads();
+        // phase 2: warp 0 takes the block's next item and gathers its facts; the other warps
+        // walk the queued tokens, one per thread (the EOS token is never queued: it has no bytes)
+        const int n = n_todo;
+        if (threadIdx.x < 32) {
+            uint32_t nxt = 0;
+            if (lane == 0) nxt = gridDim.x + (uint32_t)atomicAdd(ctx.build_next, 1);
+            nxt = __shfl_sync(0xFFFFFFFFu, nxt, 0);
+            if (lane == 0) next_item = nxt;
+            if (nxt < n_items) gather(nxt, facts[cur ^ 1]);
+        } else {
+            for (int i = threadIdx.x - 32; i < n; i += BUILD_THREADS - 32) {
+                const int rel = todo[i];
+                int *const counter = COUNT ? &counted_lookups : nullptr;
+                const uint32_t end = info.wide
+                    ? walk_token_classes<uint32_t>(v, info.rec_class, static_cast<const uint32_t *>(info.table),
+                                                   info.n_classes, info.byte_class, info.s0, t_begin + rel, counter)
+                    : walk_token_classes<uint16_t>(v, info.rec_class, static_cast<const uint16_t *>(info.table),
+                                                   info.n_classes, info.byte_class, info.s0, t_begin + rel, counter);
+                if (end != 0) atomicOr(&words[rel >> 5], 1u << (rel & 31));
+            }
+        }
+        if (COUNT) {
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                counted_words += __shfl_xor_sync(0xFFFFFFFFu, counted_words, o);
+                counted_lookups += __shfl_xor_sync(0xFFFFFFFFu, counted_lookups, o);
+            }
+            if (lane == 0) {
+                atomicAdd(&ctx.stats[ST_MASK_WORDS], (unsigned long long)counted_words);
+                atomicAdd(&ctx.stats[ST_WALKED], (unsigned long long)counted_lookups);
+            }
+            if (threadIdx.x == 32) atomicAdd(&ctx.stats[ST_QUEUED], (unsigned long long)n);
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) n_todo = 0;  // everybody has read it
+        // phase 3: whole words out
+        uint32_t *dst = info.dst;
+        for (int wl = threadIdx.x; wl < n_words; wl += BUILD_THREADS)
+            dst[(t_begin >> 5) + wl] = words[wl];
+        // Compact cache: the chunk's spans go into the cache entry straight from shared memory
+        // (chunks are whole spans; the dense words above only serve the call that built them).
+        if (COMPACT && info.row >= 0)
+            store_chunk_spans(ctx.ent_hdr + (int64_t)info.row * ctx.hdr_stride, ctx.arena, ctx.arena_top,
+                              ctx.arena_words, ctx.ent_fail + info.row, ctx.stats + ST_UNCACHED,
+                              t_begin >> 10, n_words, words, v.V, v.W);
+        __syncthreads();  // the shared arrays are free for the next item
+    }
+    // the last block to leave puts the counters back to zero for the next launch
+    if (threadIdx.x == 0) {
+        __threadfence();
+        if (atomicAdd(ctx.build_done, 1) == (int)gridDim.x - 1) {
+            *ctx.build_next = 0;
+            *ctx.build_done = 0;
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// Warp-level queue of undecided tokens for a mask build inside another kernel (the one-launch
+// step): a warp decides whole spans 32 tokens per lane at a time, queues the undecided tokens in
+// its own slice of shared memory, walks them and ends with the spans' finished words in registers,
+// one word per lane -- the layout the apply sweeps take their mask words in.
+// ---------------------------------------------------------------------------------------
+constexpr int WARP_QUEUE = 1024;   // queued tokens per warp: one whole span always fits
 
 // Walks the tokens a warp has queued (entries: span slot k << 10 | token within the span) and
 // ORs the survivors into the warp's scratch words; called by the whole warp.
