@@ -760,3 +760,46 @@ def test_batches_beyond_the_row_limit_are_refused(wg, torch):
         wg.Context(dv, 4, 65536)                   # WG_MAX_ROWS is 65535
     assert e.value.status == wg.binding.WG_ERR_ARG
     wg.Context(dv, 4, 65535).close()
+
+
+def test_one_launch_step_on_random_trees_with_a_dense_small_alphabet_vocabulary(wg, torch):
+    """The in-kernel mask build of the one-launch step on grammars nobody designed: random operator
+    trees over a six-letter alphabet and a vocabulary that holds every string of up to three
+    letters, so that most tokens are decided by the walk and many survive it."""
+    import itertools
+    from test_oracle_pins import _random_tree
+    rng = np.random.default_rng(41)
+    alphabet = b"abcd,;"
+    tokens = [b""]                                                   # id 0 = EOS
+    for n in (1, 2, 3):
+        tokens += [bytes(t) for t in itertools.product(alphabet, repeat=n)]
+    tokens += [bytes(rng.choice(list(alphabet), size=int(rng.integers(4, 24))).tolist())
+               for _ in range(1500)]
+    vocab = vocab_from_tokens(tokens, eos_id=0)
+    n_visited = 0
+    for _ in range(12):
+        ops = [_random_tree(rng, 3) for _ in range(3)]
+        rows = [0, 1, 2, 0, 1, 2, 2, 1, 0]
+        for cache_mode in (0, 1):
+            sim = Sim(wg, torch, vocab, ops, rows, "fp32", cache_capacity=256, seed=int(rng.integers(1 << 20)),
+                      steer=0.0, cache_mode=cache_mode)
+            for _ in range(10):
+                sim.step()
+            n_visited += len(sim.visited)
+    assert n_visited > 150
+
+
+def test_one_launch_step_when_a_warp_queues_more_tokens_than_its_queue_holds(wg, torch):
+    """At 64 rows and more than about 600 000 tokens a warp of the one-launch step takes two spans
+    at a time.  In a state that leaves on any of forty bytes every token is walked, 2 048 per warp
+    and pass, more than the warp's queue of 1 024 holds: the spans are then walked one by one."""
+    vocab = make_vocab(620000, seed=19)
+    leaving = SymSet(b"0123456789abcdefghijklmnopqrstuvwxyzABCD")
+    op = Sequence(Wait(allow=ALL_BYTES, wait=leaving), Write(b"!"), Wait(allow=ALL_BYTES, wait=SymSet(b"<")))
+    B = 64
+    sim = Sim(wg, torch, vocab, [op], [0] * B, "fp32", cache_capacity=0, use_cache=False, seed=23, steer=0.0)
+    launches = wg.kernel_launch_count()
+    for _ in range(2):
+        sim.step()
+    assert wg.kernel_launch_count() - launches == 2          # the one-launch step
+    assert sim.ctx.stats()["masks_built"] == 2 * B
