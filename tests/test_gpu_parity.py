@@ -163,7 +163,7 @@ class Sim:
 
     def __init__(self, wg, torch, vocab, ops, row_grammar, dtype, cache_capacity, use_cache=True,
                  seed=0, steer=6.0, delays=None, minimize=False, cache_mode=0, arena_bytes=0,
-                 grams=None, starts=None):
+                 grams=None, starts=None, row_pad=0):
         self.wg, self.torch, self.vocab, self.dtype = wg, torch, vocab, dtype
         self.flats = [op if hasattr(op, "nodes") else flatten(op) for op in ops]
         self.trees = [oracle.Tree(f) for f in self.flats]
@@ -178,6 +178,7 @@ class Sim:
         self.row_grammar = list(row_grammar)
         self.flags = (wg.WG_USE_CACHE if use_cache else wg.WG_NO_CACHE) | wg.WG_RESTART_ON_DONE
         self.seed, self.steer = seed, steer
+        self.row_pad = row_pad        # extra elements between logits rows (aligned rows, ragged V)
         self.bonus = has_structural_byte(vocab)
         self.delays = delays or [0] * self.B
         # a row that starts one step late sits in DONE first: it emits EOS and restarts
@@ -232,6 +233,10 @@ class Sim:
         oracle.apply_mask(want_logits, want_mask, vocab.size)
         # ---- library
         dl = dev_logits(torch, host, self.dtype)
+        if self.row_pad:
+            wide = torch.zeros((self.B, vocab.size + self.row_pad), dtype=dl.dtype, device="cuda")
+            wide[:, :vocab.size] = dl
+            dl = wide[:, :vocab.size]
         self._remember_inputs(dl)
         if fused:
             wg.wg_decode_step(self.ctx, self.d_gid, self.d_sid, dl, self.d_mask, self.d_tok,
@@ -803,3 +808,18 @@ def test_one_launch_step_when_a_warp_queues_more_tokens_than_its_queue_holds(wg,
         sim.step()
     assert wg.kernel_launch_count() - launches == 2          # the one-launch step
     assert sim.ctx.stats()["masks_built"] == 2 * B
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "fp32"])
+def test_one_launch_step_on_a_vocabulary_whose_size_is_no_multiple_of_anything(wg, torch, dtype):
+    vocab = odd_vocab()                      # V % 32 != 0, V % 8 != 0: ragged last word and chunk
+    assert vocab.size % 8 != 0
+    ops = [grammars.html_template(), grammars.json_reference_lookup(doc_nodes=60)]
+    pad = 16 - vocab.size % 16               # rows 32 or 64 bytes apart modulo 16: aligned rows
+    sim = Sim(wg, torch, vocab, ops, [0, 1, 0, 1, 1], dtype, cache_capacity=512, seed=31, steer=6.0,
+              row_pad=pad)
+    launches = wg.kernel_launch_count()
+    for _ in range(40):
+        sim.step()
+    assert wg.kernel_launch_count() - launches == 40          # aligned rows: the one-launch step
+    assert len(sim.visited) > 30 and sim.ctx.stats()["cache_hits"] > 0
