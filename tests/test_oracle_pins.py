@@ -694,3 +694,33 @@ def test_random_trees_agree_with_their_regular_expression():
             assert (cursor == oracle.DONE) == member, (op, text)
             n_members += member
     assert n_members > 200
+
+
+def test_masks_of_many_rows_equal_the_masks_taken_one_by_one():
+    """The multi-row call (threads over rows, strided output) against the single-row call, on
+    different trees and cursors per row, with an output whose rows are further apart than W."""
+    vocab = make_vocab(4096, seed=7)
+    ops = [grammars.html_template(), grammars.json_reference_lookup(doc_nodes=30), grammars.dotted_number()]
+    trees = [tree_of(op) for op in ops]
+    rng = np.random.default_rng(5)
+    row_tree, cursors = [], []
+    for r in range(11):
+        t = trees[r % 3]
+        cur = t.start()
+        for _ in range(int(rng.integers(0, 6))):          # a few random live steps
+            live = [s for s in range(257) if not oracle.is_dead(t.step(cur, s))]
+            if not live:
+                break
+            nxt = t.step(cur, int(rng.choice(live)))
+            if nxt == oracle.DONE:
+                break
+            cur = nxt
+        row_tree.append(t)
+        cursors.append(cur)
+    W = (vocab.size + 31) // 32
+    wide = np.full((11, W + 3), 0xABCDEF01, np.uint32)
+    got = oracle.masks(row_tree, vocab, cursors, n_threads=4, out=wide[:, :W])
+    for r in range(11):
+        assert (got[r] == oracle.mask(row_tree[r], vocab, cursors[r])).all(), r
+    assert (wide[:, W:] == 0xABCDEF01).all(), "words between the rows were written"
+    assert len({bytes(got[r]) for r in range(11)}) > 3
