@@ -118,9 +118,11 @@ __device__ __forceinline__ uint32_t walk_token_classes(const VocabDev &v, const 
                                                        const T *__restrict__ tab, int C,
                                                        const uint8_t *cls, uint32_t s, int t,
                                                        int *lookups = nullptr) {
+    // (both loads are issued before the length is looked at: one round trip instead of two;
+    // the record of a token without bytes exists and is not used)
+    const uint4 rec = __ldg(&rec_class[t]);
     const int n = v.len[t];
     if (n == 0) return 0;
-    const uint4 rec = __ldg(&rec_class[t]);
     const uint32_t w[4] = {rec.x, rec.y, rec.z, rec.w};
     // (the index stays in 32 bits: a table has fewer than 2^32 cells, and the address then takes
     // one wide multiply-add instead of a 64-bit multiply, add and shift)
