@@ -798,24 +798,49 @@ __global__ void cache_lookup_kernel(CtxDev ctx, const int32_t *gid, const int32_
 // state is new append one build-list entry per distinct state; when the pool or the table is
 // full the row is listed for an uncached build straight into its bitmask row.
 // bitmask may be NULL (prewarm): uncached rows are then dropped.
+//
+// The kernel sits between the previous step's advance and this step's apply with nothing to hide
+// its latency, so the usual case -- the state is cached and found at its first probe position --
+// is kept to two round trips after the wait: the state id, then key and pool row together.  What
+// never changes while steps are in flight (the row's grammar id, that grammar's state count) is
+// read before the wait, for the first row of every thread.
 __global__ void __launch_bounds__(1024)
 cache_lookup_insert_kernel(CtxDev ctx, const int32_t *gid, const int32_t *sid, int B,
                            uint32_t *bitmask, int64_t mask_stride) {
-    pdl_enter();
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    const int g_first = (int)threadIdx.x < B ? gid[threadIdx.x] : -1;
+    const int n_first = (g_first >= 0 && g_first < ctx.n_grammars) ? ctx.grammars[g_first].n_states : 0;
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     if (threadIdx.x == 0) *ctx.bl_count = 0;
     __syncthreads();
     const uint32_t mask = (uint32_t)ctx.hash_size - 1;
-    for (int r = threadIdx.x; r < B; r += blockDim.x) {
+    int hits = 0, misses = 0, uncached = 0;
+    unsigned long long settled = 0ull;  // bit i: the i-th row of this thread was served below
+    int it = 0;
+    for (int r = threadIdx.x; r < B; r += blockDim.x, ++it) {
         ctx.argkey[r] = 0ull;
-        const int g = gid[r], s = sid[r];
+        const int s = sid[r];
+        const int g = it == 0 ? g_first : gid[r];
+        const int n_states = it == 0 ? n_first : ((g >= 0 && g < ctx.n_grammars) ? ctx.grammars[g].n_states : 0);
         int32_t entry = -1;
         bool inserted = false;
         // a state id that the grammar does not have (or DEAD) gets no cache entry: the row is
         // built uncached, as a row of zeros, and counted as a bad state on every step
-        if (ctx.hash_size > 0 && g >= 0 && g < ctx.n_grammars && s > 0 &&
-            s < ctx.grammars[g].n_states) {
+        if (ctx.hash_size > 0 && s > 0 && s < n_states) {
             const unsigned long long key = cache_key(g, s);
             uint32_t h = cache_hash(key) & mask;
+            {
+                // key and pool row of the first probe position, requested together.  A row >= 0
+                // under the right key is final: rows are written once, after the key.
+                const unsigned long long k0 = ctx.keys[h];
+                const int32_t row0 = *(volatile int32_t *)&ctx.vals[h];
+                if (k0 == key && row0 >= 0 && !(ctx.compact && ctx.ent_fail[row0]) && it < 64) {
+                    ctx.slot[r] = row0;
+                    ++hits;
+                    settled |= 1ull << it;
+                    continue;
+                }
+            }
             for (int probe = 0; probe < ctx.hash_size; ++probe, h = (h + 1) & mask) {
                 unsigned long long k = ctx.keys[h];
                 if (k == 0) {
@@ -853,8 +878,9 @@ cache_lookup_insert_kernel(CtxDev ctx, const int32_t *gid, const int32_t *sid, i
         ctx.ent[r] = (entry >= 0 && inserted) ? (entry | ENT_NEW) : entry;
     }
     __syncthreads();
-    int hits = 0, misses = 0, uncached = 0;
-    for (int r = threadIdx.x; r < B; r += blockDim.x) {
+    it = 0;
+    for (int r = threadIdx.x; r < B; r += blockDim.x, ++it) {
+        if (it < 64 && ((settled >> it) & 1ull)) continue;
         const int32_t e = ctx.ent[r];
         int32_t row = e >= 0 ? ctx.vals[e & ~ENT_NEW] : -1;
         // a state whose entry found no room in the arena is rebuilt on every step (a row
