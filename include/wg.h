@@ -423,8 +423,13 @@ int32_t wg_advance(wg_ctx *ctx, const int32_t *gid, int32_t *sid, const int32_t 
  * that meet the same new state in the same step each build it (masks_built counts every built
  * row, cache_misses every row that missed) and one of them files it.
  * flags: WG_USE_CACHE or WG_NO_CACHE, optionally | WG_RESTART_ON_DONE.
- *   token_out  device, B entries (the greedy choice, -1 for an empty mask)
- *   status     device, B entries, or NULL (WG_OK, WG_ERR_EMPTY_MASK, WG_ERR_STATE) */
+ *   token_out  device, B entries (the greedy choice, -1 for an empty mask), or NULL
+ *   status     device, B entries, or NULL (WG_OK, WG_ERR_EMPTY_MASK, WG_ERR_STATE)
+ * With token_out NULL the step only masks, for an engine that samples by itself (paper Section 2:
+ * the mask is applied to the logits before sampling): lookup, build of the misses, mask rows out
+ * and apply run as above, no token is chosen and sid is left as it is; the caller samples from the
+ * masked logits and hands its tokens to wg_advance.  status must then be NULL and
+ * WG_RESTART_ON_DONE unset (WG_ERR_ARG otherwise). */
 int32_t wg_decode_step(wg_ctx *ctx, const int32_t *gid, int32_t *sid, int32_t B, void *logits,
                        int32_t dtype, int64_t row_stride_elems, uint32_t *bitmask,
                        int64_t mask_stride_words, int32_t *token_out, int32_t *status,

@@ -553,10 +553,12 @@ def _step_args(ctx: Context, gid, sid, logits, n_cols: int, bitmask, token_out, 
 
 def wg_decode_step(ctx: Context, gid, sid, logits, bitmask, token_out, status=None,
                    flags: int = WG_USE_CACHE, stream=None) -> None:
+    """One decode step.  With ``token_out`` None the step only masks (no argmax, no advance): the
+    caller samples from the masked logits and calls ``wg_advance``."""
     g, s, B, lp, dtype, stride, mp, mstride, tok, st = _step_args(
         ctx, gid, sid, logits, ctx.vocab.V, bitmask, token_out, status)
-    if tok is None:
-        raise ValueError("token_out is required")
+    if tok is None and (st is not None or int(flags) & WG_RESTART_ON_DONE):
+        raise ValueError("a step without token_out advances nothing: no status, no WG_RESTART_ON_DONE")
     _check(_lib.wg_decode_step(ctx.handle, g, s, B, lp, dtype, stride, mp, mstride, tok, st,
                                int(flags), _stream_ptr(stream)), "wg_decode_step")
 

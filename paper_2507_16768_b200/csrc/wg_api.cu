@@ -1035,7 +1035,11 @@ int32_t decode_step_impl(wg_ctx *c, const int32_t *gid, int32_t *sid, int32_t B,
     ApplyArgs a{row0, row_stride_elems, bitmask, bitmask, mask_stride_words, B, v_end, W_end, 0,
                 v_begin / 1024};
     const int32_t t_last = v_end == v.V ? v.W * 32 : v_end;
-    if (whole && !best_keys && B <= SMALL_STEP_ROWS && rows_aligned(logits, row_stride_elems, esize)) {
+    // Without token_out and best_keys the step only masks: no argmax, no advance (the caller
+    // samples and calls wg_advance).
+    const bool mask_only = !token_out && !best_keys;
+    if (whole && !best_keys && !mask_only && B <= SMALL_STEP_ROWS &&
+        rows_aligned(logits, row_stride_elems, esize)) {
         // A handful of rows: the whole step in one launch (see decode_step_small_kernel).
         int32_t rc;
         if ((rc = timing_mark(c, 0, st)) != WG_OK) return rc;
@@ -1075,10 +1079,15 @@ int32_t decode_step_impl(wg_ctx *c, const int32_t *gid, int32_t *sid, int32_t B,
     if (rc != WG_OK) return rc;
     if ((rc = timing_mark(c, 1, st)) != WG_OK) return rc;
     if ((rc = timing_mark(c, 2, st)) != WG_OK) return rc;
-    rc = no_cache ? launch_apply<true, false>(dtype, a, c->dev, c->dev.argkey, st, true)
-                  : launch_apply<true, true>(dtype, a, c->dev, c->dev.argkey, st, true);
+    if (mask_only)
+        rc = no_cache ? launch_apply<false, false>(dtype, a, c->dev, nullptr, st, true)
+                      : launch_apply<false, true>(dtype, a, c->dev, nullptr, st, true);
+    else
+        rc = no_cache ? launch_apply<true, false>(dtype, a, c->dev, c->dev.argkey, st, true)
+                      : launch_apply<true, true>(dtype, a, c->dev, c->dev.argkey, st, true);
     if (rc != WG_OK) return rc;
     if ((rc = timing_mark(c, 3, st)) != WG_OK) return rc;
+    if (mask_only) return WG_OK;
     if (best_keys) {
         WG_CUDA(launch_pdl(export_keys_kernel, dim3((B + 127) / 128), dim3(128), st, c->dev,
                            best_keys, B));
@@ -1100,9 +1109,10 @@ int32_t wg_decode_step(wg_ctx *c, const int32_t *gid, int32_t *sid, int32_t B, v
                        int64_t mask_stride_words, int32_t *token_out, int32_t *status,
                        uint32_t flags, void *stream) {
     NvtxRange nvtx_range("wg_decode_step");
-    if (!batch_ok(c, B) || !gid || !sid || !logits || !bitmask || !token_out) return WG_ERR_ARG;
+    if (!batch_ok(c, B) || !gid || !sid || !logits || !bitmask) return WG_ERR_ARG;
     if (dtype != WG_DTYPE_BF16 && dtype != WG_DTYPE_FP32) return WG_ERR_ARG;
     if (flags & ~(uint32_t)(WG_NO_CACHE | WG_RESTART_ON_DONE)) return WG_ERR_ARG;
+    if (!token_out && (status || (flags & WG_RESTART_ON_DONE))) return WG_ERR_ARG;  // nothing advances
     const VocabDev &v = c->vocab->dev;
     if (row_stride_elems < v.V || mask_stride_words < v.W) return WG_ERR_ARG;
     return decode_step_impl(c, gid, sid, B, logits, dtype, row_stride_elems, bitmask,

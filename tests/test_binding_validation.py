@@ -184,3 +184,12 @@ def test_host_step_refuses(no_library):
         call(tok_host=torch.zeros(B - 1, dtype=torch.int32))
     with pytest.raises(ValueError):
         call(tok=FakeTensor([B - 1]))
+
+
+def test_mask_only_step_takes_no_status_and_no_restart_flag(no_library):
+    a = good()
+    with pytest.raises(ValueError):
+        wg.wg_decode_step(FakeContext(), a["gid"], a["sid"], a["logits"], a["bitmask"], None, a["status"])
+    with pytest.raises(ValueError):
+        wg.wg_decode_step(FakeContext(), a["gid"], a["sid"], a["logits"], a["bitmask"], None, None,
+                          wg.WG_USE_CACHE | wg.WG_RESTART_ON_DONE)

@@ -823,3 +823,57 @@ def test_one_launch_step_on_a_vocabulary_whose_size_is_no_multiple_of_anything(w
         sim.step()
     assert wg.kernel_launch_count() - launches == 40          # aligned rows: the one-launch step
     assert len(sim.visited) > 30 and sim.ctx.stats()["cache_hits"] > 0
+
+
+@pytest.mark.parametrize("B,dtype,cache_mode,use_cache", [(5, "fp32", 0, True), (96, "bf16", 0, True),
+                                                          (96, "bf16", 1, True), (70, "fp32", 0, False)])
+def test_mask_only_step_for_an_engine_that_samples_itself(wg, torch, B, dtype, cache_mode, use_cache):
+    """wg_decode_step without token_out: masks and masked logits as the checker's, states left
+    alone; the test then "samples" a random allowed token per row and hands it to wg_advance."""
+    vocab = make_vocab(12000 + 7, seed=41)
+    ops = [grammars.html_template(), grammars.json_reference_lookup(doc_nodes=60)]
+    rows = [r % 2 for r in range(B)]
+    sim = Sim(wg, torch, vocab, ops, rows, dtype, cache_capacity=2048, seed=B, steer=4.0,
+              cache_mode=cache_mode, use_cache=use_cache)
+    rng = np.random.default_rng(B)
+    flags = wg.WG_USE_CACHE if use_cache else wg.WG_NO_CACHE
+    V = vocab.size
+    for step in range(40):
+        host = sim.logits()
+        trees = [sim.trees[g] for g in rows]
+        want_mask = oracle.masks(trees, vocab, sim.cursors, n_threads=oracle.max_threads())
+        want_logits = host.copy()
+        oracle.apply_mask(want_logits, want_mask, V)
+        dl = dev_logits(torch, host, dtype)
+        before = sim.d_sid.clone()
+        wg.wg_decode_step(sim.ctx, sim.d_gid, sim.d_sid, dl, sim.d_mask, None, None, flags)
+        assert (sim.d_sid == before).all(), "a step that chooses no token advances nothing"
+        got_mask = sim.d_mask.cpu().numpy().view(np.uint32)
+        assert (got_mask == want_mask).all(), step
+        raw_want = want_logits.view(np.uint32) if dtype == "fp32" else want_logits
+        assert (raw_bits(torch, dl) == raw_want).all(), step
+        # the engine's sampler: any allowed token
+        bits = np.unpackbits(want_mask.view(np.uint8), axis=1, bitorder="little")[:, :V]
+        toks = np.array([rng.choice(np.flatnonzero(bits[r])) for r in range(B)], np.int32)
+        d_tok = to_dev(torch, toks)
+        wg.wg_advance(sim.ctx, sim.d_gid, sim.d_sid, d_tok, sim.d_status, wg.WG_RESTART_ON_DONE)
+        assert (sim.d_status.cpu().numpy() == 0).all()
+        got_sid = sim.d_sid.cpu().numpy()
+        for r in range(B):
+            gi, t = rows[r], int(toks[r])
+            rc, cur = oracle.advance(sim.trees[gi], vocab, sim.cursors[r], t)
+            assert rc == 0
+            host_sid = sim.grams[gi].step_token(int(sim.h_sid[r]), t, token_symbols(vocab, t))
+            if cur == oracle.DONE:
+                cur, host_sid = sim.trees[gi].start(), sim.grams[gi].start_state
+            sim.cursors[r] = cur
+            assert got_sid[r] == host_sid, (step, r)
+            sim.visited.add((gi, host_sid))
+        sim.h_sid = got_sid.copy()
+        sim.step_no += 1
+    assert len(sim.visited) > 40
+    with pytest.raises(ValueError):                 # nothing advances: a status array has no meaning
+        wg.wg_decode_step(sim.ctx, sim.d_gid, sim.d_sid, dl, sim.d_mask, None, sim.d_status, flags)
+    with pytest.raises(ValueError):
+        wg.wg_decode_step(sim.ctx, sim.d_gid, sim.d_sid, dl, sim.d_mask, None, None,
+                          flags | wg.WG_RESTART_ON_DONE)
