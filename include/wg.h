@@ -322,9 +322,23 @@ int32_t wg_cache_entry_read(wg_ctx *ctx, int32_t grammar_id, int32_t state, int3
  * instantiated with the same arguments share cache entries.  Synchronous: the table is
  * copied and a few set-up kernels run on the legacy default stream, which the call waits for
  * (so it must not be made while a stream capture is under way).
- * Errors: WG_ERR_ARG, WG_ERR_CAPACITY (more than 65535 grammars, or a table of 2^32 cells or
- * more), WG_ERR_CUDA. */
+ * The id may be one that wg_ctx_remove_grammar set free.
+ * Errors: WG_ERR_ARG, WG_ERR_CAPACITY (more than 65535 grammars at a time, or a table of 2^32
+ * cells or more), WG_ERR_CUDA. */
 int32_t wg_ctx_add_grammar(wg_ctx *ctx, const wg_grammar *grammar, int32_t *grammar_id);
+
+/* Takes grammar `grammar_id` out of the context again (paper Section 3.1: a state machine is
+ * made per request from the request's arguments, so a serving process adds grammars for as long
+ * as it runs).  The grammar's device tables are freed, its cached masks stop matching and their
+ * pool rows are handed out to later states (the words a compact entry took in the arena come
+ * back only with wg_cache_clear), and the id is given to a grammar added later -- at most 65535
+ * grammars are held AT A TIME.  From the call on, a row that still names the id is treated as a
+ * row in a state the grammar does not have: an all-zero mask, WG_ERR_STATE, bad_states counted.
+ * Synchronous: waits for everything queued on the device first (no stream capture may be under
+ * way); a step recorded with wg_step_graph_create for rows of this grammar must not be launched
+ * afterwards.  When removed entries hold a quarter of the hash table it is rebuilt without them.
+ * Errors: WG_ERR_ARG (no such grammar), WG_ERR_CUDA. */
+int32_t wg_ctx_remove_grammar(wg_ctx *ctx, int32_t grammar_id);
 
 /* Builds and caches the mask of every state of grammar `grammar_id` (states 1..n_states-1),
  * max_batch states at a time.  Returns WG_ERR_CAPACITY after the first batch that found the

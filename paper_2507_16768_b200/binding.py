@@ -83,6 +83,7 @@ _SIGNATURES = {
     "wg_cache_entry_read": (_i32, [_vp, _i32, _i32, C.POINTER(_i32), C.POINTER(_i32), _vp, _i32,
                                    C.POINTER(_i64), _vp]),
     "wg_ctx_add_grammar": (_i32, [_vp, _vp, C.POINTER(_i32)]),
+    "wg_ctx_remove_grammar": (_i32, [_vp, _i32]),
     "wg_cache_prewarm": (_i32, [_vp, _i32, _vp]),
     "wg_cache_clear": (_i32, [_vp, _vp]),
     "wg_get_stats": (_i32, [_vp, C.POINTER(WgStats), _vp]),
@@ -410,6 +411,10 @@ class Context:
         _check(_lib.wg_ctx_add_grammar(self.handle, grammar.handle, C.byref(gid)),
                "wg_ctx_add_grammar")
         return gid.value
+
+    def remove_grammar(self, grammar_id: int) -> None:
+        """Frees the grammar's tables and cached masks; the id goes to a grammar added later."""
+        _check(_lib.wg_ctx_remove_grammar(self.handle, int(grammar_id)), "wg_ctx_remove_grammar")
 
     def cache_prewarm(self, grammar_id: int, stream=None) -> None:
         _check(_lib.wg_cache_prewarm(self.handle, int(grammar_id), _stream_ptr(stream)),

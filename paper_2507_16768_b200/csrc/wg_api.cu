@@ -95,9 +95,10 @@ struct GrammarSlot {
     // (Write("a") and Write("b")) are different grammars
     uint8_t byte_class[256];
     int32_t start, done, eos_class;
+    bool removed = false;  // wg_ctx_remove_grammar: the id waits to be given to another grammar
 
     bool same_as(const wg_grammar &g) const {
-        return hash == g.hash && n_states == g.n_states && n_classes == g.n_classes &&
+        return !removed && hash == g.hash && n_states == g.n_states && n_classes == g.n_classes &&
                start == g.start && done == g.done && eos_class == g.eos_class &&
                memcmp(byte_class, g.byte_class, 256) == 0 && table == g.table &&
                forced_tok == g.forced_tok && forced_next == g.forced_next;
@@ -107,6 +108,7 @@ struct GrammarSlot {
 struct ClassMappedRecords {
     uint8_t byte_class[256];
     void *d_rec;  // uint4[V]
+    int users;    // grammars of the context that walk these records
 };
 
 struct wg_ctx {
@@ -132,6 +134,8 @@ struct wg_ctx {
     std::vector<void *> owned;  // every other device allocation
     std::mutex mu;
     bool count_build_work = false;  // launch the counting variant of the build kernel
+    int64_t removed_keys = 0;       // hash-table entries of removed grammars still in the table
+    int32_t *d_counts = nullptr;    // scratch of wg_ctx_remove_grammar
     // optional per-kernel timing: events[4 * i + {0,1,2,3}] = build begin/end, apply begin/end
     bool timing = false;
     std::vector<cudaEvent_t> events;
@@ -521,6 +525,9 @@ int32_t wg_ctx_create_ex(const wg_vocab *vocab, int32_t cache_capacity, int32_t 
         take(&d.pool, (size_t)d.capacity * (size_t)d.pool_stride);
     }
     take(&d.n_slots, 1);
+    take(&d.free_rows, (size_t)d.capacity);
+    take(&d.n_free, 1);
+    take(&c->d_counts, 1);
     take(&d.ent, (size_t)max_batch);
     take(&d.slot, (size_t)max_batch);
     take(&d.bl_gid, (size_t)max_batch);
@@ -542,6 +549,7 @@ int32_t wg_ctx_create_ex(const wg_vocab *vocab, int32_t cache_capacity, int32_t 
         if (cudaMemset(d.keys, 0, sizeof(unsigned long long) * (size_t)(d.hash_size ? d.hash_size : 1)) != cudaSuccess ||
             cudaMemset(d.vals, 0xFF, sizeof(int32_t) * (size_t)(d.hash_size ? d.hash_size : 1)) != cudaSuccess ||
             cudaMemset(d.n_slots, 0, sizeof(int32_t)) != cudaSuccess ||
+            cudaMemset(d.n_free, 0, sizeof(int32_t)) != cudaSuccess ||
             cudaMemset(d.bl_count, 0, sizeof(int32_t)) != cudaSuccess ||
             cudaMemset(d.build_next, 0, 2 * sizeof(int32_t)) != cudaSuccess ||
             cudaMemset(d.argkey, 0, sizeof(unsigned long long) * (size_t)max_batch) != cudaSuccess ||
@@ -592,7 +600,9 @@ int32_t wg_ctx_add_grammar(wg_ctx *c, const wg_grammar *g, int32_t *grammar_id) 
             return WG_OK;
         }
     }
-    if (c->slots.size() >= 65535) return WG_ERR_CAPACITY;
+    bool id_waiting = false;  // the id of a removed grammar can be used again
+    for (const GrammarSlot &sl : c->slots) id_waiting = id_waiting || sl.removed;
+    if (c->slots.size() >= 65535 && !id_waiting) return WG_ERR_CAPACITY;
     // the kernels index table cells with 32 bits
     if ((uint64_t)g->n_states * (uint64_t)g->n_classes >= (1ull << 32)) return WG_ERR_CAPACITY;
     const bool wide = g->n_states > 65535;
@@ -686,13 +696,18 @@ int32_t wg_ctx_add_grammar(wg_ctx *c, const wg_grammar *g, int32_t *grammar_id) 
     // the vocabulary's records with bytes replaced by this grammar's classes (shared between
     // grammars whose class maps are equal)
     const void *d_rec_class = nullptr;
-    for (const ClassMappedRecords &r : c->class_records)
-        if (memcmp(r.byte_class, g->byte_class, 256) == 0) d_rec_class = r.d_rec;
+    for (ClassMappedRecords &r : c->class_records)
+        if (r.d_rec && memcmp(r.byte_class, g->byte_class, 256) == 0) {
+            d_rec_class = r.d_rec;
+            ++r.users;
+            break;
+        }
     if (!d_rec_class) {
         const int V = c->vocab->dev.V;
         ClassMappedRecords r;
         memcpy(r.byte_class, g->byte_class, 256);
         r.d_rec = nullptr;
+        r.users = 1;
         WG_CUDA(cudaMalloc(&r.d_rec, (size_t)V * WG_REC_BYTES));
         map_records_kernel<<<(unsigned)((V + 255) / 256), 256, 0, cudaStreamLegacy>>>(
             c->vocab->dev.rec, static_cast<const uint8_t *>(slot.d_cls), static_cast<uint4 *>(r.d_rec), V);
@@ -714,7 +729,9 @@ int32_t wg_ctx_add_grammar(wg_ctx *c, const wg_grammar *g, int32_t *grammar_id) 
                   static_cast<const int16_t *>(slot.d_leave1),
                   static_cast<const unsigned long long *>(slot.d_leave_fold), g->n_states,
                   g->n_classes, g->start, g->done, g->eos_class, wide ? 1 : 0};
-    const int32_t id = (int32_t)c->slots.size();
+    int32_t id = (int32_t)c->slots.size();
+    for (size_t i = 0; i < c->slots.size(); ++i)  // the id of a removed grammar is used again
+        if (c->slots[i].removed) { id = (int32_t)i; break; }
     if (id >= c->grammar_cap) {  // grow the registry; queued kernels still read the old one
         WG_CUDA(cudaDeviceSynchronize());
         const int32_t cap = c->grammar_cap * 2;
@@ -728,11 +745,79 @@ int32_t wg_ctx_add_grammar(wg_ctx *c, const wg_grammar *g, int32_t *grammar_id) 
         c->dev.grammars = bigger;
     }
     WG_CUDA(cudaMemcpy(c->d_grammars + id, &gd, sizeof(GrammarDev), cudaMemcpyHostToDevice));
-    c->grammars.push_back(gd);
     guard.s = nullptr;  // the context owns the uploads from here on
-    c->slots.push_back(std::move(slot));
-    c->dev.n_grammars = id + 1;
+    if (id < (int32_t)c->slots.size()) {
+        c->grammars[id] = gd;
+        c->slots[id] = std::move(slot);
+    } else {
+        c->grammars.push_back(gd);
+        c->slots.push_back(std::move(slot));
+        c->dev.n_grammars = id + 1;
+    }
     *grammar_id = id;
+    return WG_OK;
+}
+
+int32_t wg_ctx_remove_grammar(wg_ctx *c, int32_t grammar_id) {
+    NvtxRange nvtx_range("wg_ctx_remove_grammar");
+    if (!c) return WG_ERR_ARG;
+    std::lock_guard<std::mutex> lock(c->mu);
+    if (grammar_id < 0 || grammar_id >= (int32_t)c->slots.size() || c->slots[grammar_id].removed)
+        return WG_ERR_ARG;
+    // every queued kernel may still read the grammar's tables and the cache
+    WG_CUDA(cudaDeviceSynchronize());
+    GrammarSlot &slot = c->slots[grammar_id];
+    // 1. rows that still name the id get an all-zero mask and a bad-state count from now on
+    GrammarDev none{};
+    WG_CUDA(cudaMemcpy(c->d_grammars + grammar_id, &none, sizeof(GrammarDev), cudaMemcpyHostToDevice));
+    c->grammars[grammar_id] = none;
+    // 2. its cached masks stop matching and their pool rows are handed out again
+    if (c->dev.hash_size > 0) {
+        WG_CUDA(cudaMemset(c->d_counts, 0, sizeof(int32_t)));
+        remove_grammar_entries_kernel<<<(c->dev.hash_size + 255) / 256, 256, 0, cudaStreamLegacy>>>(
+            c->dev, grammar_id, c->d_counts);
+        WG_LAUNCHED();
+        int32_t dropped = 0;
+        WG_CUDA(cudaMemcpy(&dropped, c->d_counts, sizeof(dropped), cudaMemcpyDeviceToHost));
+        c->removed_keys += dropped;
+        // 3. once a quarter of the table is held by removed entries it is rebuilt without them
+        if (c->removed_keys * 4 > c->dev.hash_size) {
+            unsigned long long *old_keys = nullptr;
+            int32_t *old_vals = nullptr;
+            const size_t n = (size_t)c->dev.hash_size;
+            if (cudaMalloc((void **)&old_keys, n * sizeof(unsigned long long)) != cudaSuccess ||
+                cudaMalloc((void **)&old_vals, n * sizeof(int32_t)) != cudaSuccess) {
+                cudaFree(old_keys);
+                cudaGetLastError();   // (the table stays as it is: longer probes, same results)
+            } else {
+                cudaMemcpy(old_keys, c->dev.keys, n * sizeof(unsigned long long), cudaMemcpyDeviceToDevice);
+                cudaMemcpy(old_vals, c->dev.vals, n * sizeof(int32_t), cudaMemcpyDeviceToDevice);
+                cudaMemset(c->dev.keys, 0, n * sizeof(unsigned long long));
+                cudaMemset(c->dev.vals, 0xFF, n * sizeof(int32_t));
+                rehash_kernel<<<(unsigned)((n + 255) / 256), 256, 0, cudaStreamLegacy>>>(c->dev, old_keys, old_vals);
+                WG_LAUNCHED();
+                const cudaError_t err = cudaDeviceSynchronize();
+                cudaFree(old_keys);
+                cudaFree(old_vals);
+                if (err != cudaSuccess) return WG_ERR_CUDA;
+                c->removed_keys = 0;
+            }
+        }
+    }
+    WG_CUDA(cudaDeviceSynchronize());
+    // 4. the grammar's own device arrays
+    cudaFree(slot.d_table); cudaFree(slot.d_cls); cudaFree(slot.d_first_ok); cudaFree(slot.d_leaves);
+    cudaFree(slot.d_forced); cudaFree(slot.d_leave1); cudaFree(slot.d_leave_fold);
+    slot.d_table = slot.d_cls = slot.d_first_ok = slot.d_leaves = nullptr;
+    slot.d_forced = slot.d_leave1 = slot.d_leave_fold = nullptr;
+    for (ClassMappedRecords &r : c->class_records)
+        if (r.d_rec && memcmp(r.byte_class, slot.byte_class, 256) == 0 && --r.users == 0) {
+            cudaFree(r.d_rec);
+            r.d_rec = nullptr;
+        }
+    slot.table.clear(); slot.table.shrink_to_fit();
+    slot.forced_tok.clear(); slot.forced_next.clear();
+    slot.removed = true;
     return WG_OK;
 }
 
@@ -743,6 +828,7 @@ int32_t wg_cache_clear(wg_ctx *c, void *stream) {
     const int n = c->dev.hash_size > 0 ? c->dev.hash_size : 1;
     cache_clear_kernel<<<(n + 255) / 256, 256, 0, st>>>(c->dev);
     WG_LAUNCHED();
+    c->removed_keys = 0;
     return WG_OK;
 }
 
@@ -750,10 +836,11 @@ int32_t wg_get_stats(wg_ctx *c, wg_stats *out, void *stream) {
     if (!c || !out) return WG_ERR_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     unsigned long long h[ST_COUNT];
-    int32_t n_slots = 0;
+    int32_t n_slots = 0, n_free = 0;
     unsigned long long arena_top = 0;
     WG_CUDA(cudaMemcpyAsync(h, c->dev.stats, sizeof(h), cudaMemcpyDeviceToHost, st));
     WG_CUDA(cudaMemcpyAsync(&n_slots, c->dev.n_slots, sizeof(n_slots), cudaMemcpyDeviceToHost, st));
+    WG_CUDA(cudaMemcpyAsync(&n_free, c->dev.n_free, sizeof(n_free), cudaMemcpyDeviceToHost, st));
     if (c->dev.compact)
         WG_CUDA(cudaMemcpyAsync(&arena_top, c->dev.arena_top, sizeof(arena_top),
                                 cudaMemcpyDeviceToHost, st));
@@ -765,6 +852,7 @@ int32_t wg_get_stats(wg_ctx *c, wg_stats *out, void *stream) {
     out->tokens_rejected = (int64_t)h[ST_REJECTED];
     out->empty_masks = (int64_t)h[ST_EMPTY];
     out->bad_states = (int64_t)h[ST_BAD_STATE];
+    n_slots -= n_free > 0 ? n_free : 0;  // rows that a removed grammar gave back hold nothing
     out->cache_entries = n_slots;
     if (arena_top > (unsigned long long)c->dev.arena_words) arena_top = (unsigned long long)c->dev.arena_words;
     out->cache_bytes = c->dev.compact

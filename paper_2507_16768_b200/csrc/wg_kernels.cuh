@@ -62,7 +62,9 @@ struct CtxDev {
     int32_t hash_size;         // power of two (0 when capacity == 0)
     int32_t capacity;
     int64_t pool_stride;       // words
-    int32_t *n_slots;          // pool rows handed out so far
+    int32_t *n_slots;          // pool rows handed out so far (the high-water mark)
+    int32_t *free_rows;        // [capacity] pool rows given back when a grammar was removed
+    int32_t *n_free;           // how many of them wait to be handed out again
     // per-call scratch
     int32_t *ent;              // [max_batch] hash entry of each row
     int32_t *slot;             // [max_batch] resolved pool row of each row, or -1
@@ -752,6 +754,27 @@ __device__ __forceinline__ uint32_t cache_hash(unsigned long long k) {
 }
 
 constexpr int32_t ENT_NEW = 0x40000000;  // marks the row that inserted its key in this call
+// The key of an entry whose grammar was removed: it matches no state and does not end a probe
+// sequence (grammar ids stay below 65 535, so no real key has all bits set).
+constexpr unsigned long long KEY_REMOVED = ~0ull;
+
+// No pool row left to hand out (neither a returned one nor a fresh one).
+__device__ __forceinline__ bool pool_full(const CtxDev &ctx) {
+    return *(volatile int32_t *)ctx.n_slots >= ctx.capacity && *(volatile int32_t *)ctx.n_free <= 0;
+}
+
+// A pool row for a new entry: one that a removed grammar gave back, else a fresh one; -1 when
+// the pool is full.  (Rows are only given back by remove_grammar_entries_kernel, which never
+// runs beside a kernel that takes rows.)
+__device__ __forceinline__ int32_t take_pool_row(const CtxDev &ctx) {
+    const int32_t waiting = atomicSub(ctx.n_free, 1);
+    if (waiting > 0) return ctx.free_rows[waiting - 1];
+    atomicAdd(ctx.n_free, 1);
+    const int32_t row = atomicAdd(ctx.n_slots, 1);
+    if (row < ctx.capacity) return row;
+    atomicSub(ctx.n_slots, 1);
+    return -1;
+}
 
 // Read-only probe for (g, s): the pool row; -1 when the key is absent; -2 when it is present
 // without a usable row (taken while the pool was full, being filed at this moment, or a compact
@@ -846,11 +869,11 @@ cache_lookup_insert_kernel(CtxDev ctx, const int32_t *gid, const int32_t *sid, i
                 if (k == 0) {
                     // a full pool takes no new keys, so the table never fills up with states
                     // it cannot serve (the row is then built uncached)
-                    if (*(volatile int32_t *)ctx.n_slots >= ctx.capacity) break;
+                    if (pool_full(ctx)) break;
                     k = atomicCAS(&ctx.keys[h], 0ull, key);
                     if (k == 0) {  // this thread owns the new entry
-                        const int32_t row = atomicAdd(ctx.n_slots, 1);
-                        if (row < ctx.capacity) {
+                        const int32_t row = take_pool_row(ctx);
+                        if (row >= 0) {
                             ctx.vals[h] = row;
                             const int i = atomicAdd(ctx.bl_count, 1);
                             ctx.bl_gid[i] = g;
@@ -864,7 +887,6 @@ cache_lookup_insert_kernel(CtxDev ctx, const int32_t *gid, const int32_t *sid, i
                                 ctx.bl_dst[i] = ctx.pool + (int64_t)row * ctx.pool_stride;
                             }
                         } else {
-                            atomicSub(ctx.n_slots, 1);
                             ctx.vals[h] = -1;
                         }
                         entry = (int32_t)h;
@@ -926,7 +948,40 @@ __global__ void cache_clear_kernel(CtxDev ctx) {
     if (i < ctx.hash_size) { ctx.keys[i] = 0ull; ctx.vals[i] = -1; }
     if (i == 0) {
         *ctx.n_slots = 0;
+        *ctx.n_free = 0;
         if (ctx.compact) *ctx.arena_top = 0ull;
+    }
+}
+
+// wg_ctx_remove_grammar: every cache entry of grammar g stops matching (its key becomes
+// KEY_REMOVED, so probe sequences that pass over it stay whole) and its pool row goes onto the list
+// of rows to hand out again.  counts[0] += entries dropped.  Runs alone on an idle device.
+__global__ void remove_grammar_entries_kernel(CtxDev ctx, int g, int32_t *counts) {
+    const int h = blockIdx.x * blockDim.x + threadIdx.x;
+    if (h >= ctx.hash_size) return;
+    if ((uint32_t)(ctx.keys[h] >> 32) != (uint32_t)(g + 1)) return;
+    const int32_t row = ctx.vals[h];
+    ctx.keys[h] = KEY_REMOVED;
+    ctx.vals[h] = -1;
+    if (row >= 0) ctx.free_rows[atomicAdd(ctx.n_free, 1)] = row;
+    atomicAdd(&counts[0], 1);
+}
+
+// Rebuilds the hash table from a copy of itself without the removed entries (they would
+// otherwise lengthen every probe sequence for good).  old_keys / old_vals: the copy; the
+// table itself has been cleared before.
+__global__ void rehash_kernel(CtxDev ctx, const unsigned long long *old_keys, const int32_t *old_vals) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= ctx.hash_size) return;
+    const unsigned long long key = old_keys[i];
+    if (key == 0ull || key == KEY_REMOVED) return;
+    const uint32_t mask = (uint32_t)ctx.hash_size - 1;
+    uint32_t h = cache_hash(key) & mask;
+    for (int probe = 0; probe < ctx.hash_size; ++probe, h = (h + 1) & mask) {
+        if (atomicCAS(&ctx.keys[h], 0ull, key) == 0ull) {
+            ctx.vals[h] = old_vals[i];
+            return;
+        }
     }
 }
 
@@ -1566,16 +1621,14 @@ decode_step_small_kernel(ApplyArgs a, CtxDev ctx, VocabDev v, SmallStepArgs st) 
                 for (int probe = 0; probe < ctx.hash_size; ++probe, h = (h + 1) & mask) {
                     unsigned long long k = ctx.keys[h];
                     if (k == 0) {
-                        if (*(volatile int32_t *)ctx.n_slots >= ctx.capacity) break;   // full
+                        if (pool_full(ctx)) break;
                         k = atomicCAS(&ctx.keys[h], 0ull, key);
                         if (k == 0) {
-                            const int32_t got = atomicAdd(ctx.n_slots, 1);
-                            if (got < ctx.capacity) {
+                            const int32_t got = take_pool_row(ctx);
+                            if (got >= 0) {        // (else the key stays, without a row)
                                 new_row = got;
                                 filed = true;
                                 if (ctx.compact) ctx.ent_fail[got] = 0;
-                            } else {
-                                atomicSub(ctx.n_slots, 1);   // the key stays, without a row
                             }
                             ctx.ent[r] = (int32_t)h;
                             break;
@@ -1584,8 +1637,7 @@ decode_step_small_kernel(ApplyArgs a, CtxDev ctx, VocabDev v, SmallStepArgs st) 
                     if (k == key) {
                         // another row files it in this step (or did, with a compact entry that
                         // found no room); a key left without a row by a full pool is not filed
-                        filed = *(volatile int32_t *)ctx.n_slots < ctx.capacity ||
-                                *(volatile int32_t *)&ctx.vals[h] >= 0;
+                        filed = !pool_full(ctx) || *(volatile int32_t *)&ctx.vals[h] >= 0;
                         break;
                     }
                 }
